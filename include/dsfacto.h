@@ -1,0 +1,142 @@
+/*
+ * dsfacto.h - C ABI of the DS-FACTO training hot path (doubly-separable factorization machines,
+ * arXiv 2004.13940) for one NVIDIA B200 (sm_100a).
+ *
+ * Model (Section 3.2, eq. (fm_model2)): f(x_i) = w0 + sum_j w_j x_ij
+ *     + 1/2 sum_k [ (sum_j v_jk x_ij)^2 - sum_j v_jk^2 x_ij^2 ],  w in R^D, V in R^{D x K}.
+ * Objective (eq. (fm_obj)): L = (1/N) sum_i l(f(x_i), y_i) + lambda_w/2 |w|^2 + lambda_v/2 |V|^2.
+ * Auxiliaries (Table "Notations", eq. (compute_a_jk)): a_ik = sum_j v_jk x_ij and the multiplier
+ *     G_i = dl/df (f - y for the squared loss, -y / (1 + exp(y f)) for the logistic loss).
+ *
+ * One epoch = one outer iteration of Algorithm 1 in its synchronous (DSGD-style) form:
+ *   X is cut into a p x p grid of (row-block, column-block) tiles (figure "communication
+ *   pattern"); in inner round s the tiles (r, (r+s) mod p), r = 0..p-1, are processed; every
+ *   stored entry applies the stochastic updates (dsfacto_sgdupdatew)/(dsfacto_sgdupdatev) once,
+ *   with G and A frozen; afterwards G and A are recomputed from the new parameters
+ *   (Section 4.2, "Handling the staleness ...") and the objective is evaluated.
+ *
+ * Conventions
+ *   - Every pointer argument is HOST memory, borrowed for the duration of the call; outputs are
+ *     caller-allocated.  The library owns all device memory.
+ *   - Return value: DSFACTO_OK (0) or a negative DSFACTO_ERR_* code; nothing is thrown.
+ *   - Calls on one handle must not overlap in time.  Every call returns after its device work
+ *     has completed.  There is no CPU fallback: without a usable CUDA device calls fail with
+ *     DSFACTO_ERR_CUDA.
+ *   - All device state is fp32 (X, y, w, V, A, G); sums that form the objective are fp64.
+ */
+#ifndef DSFACTO_H
+#define DSFACTO_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dsfacto dsfacto_t; /* opaque, owned by the library */
+
+enum { DSFACTO_SQUARED = 0, DSFACTO_LOGISTIC = 1 }; /* l = 1/2 (f-y)^2 ; l = log(1+exp(-y f)), y = +-1 */
+
+enum {
+    DSFACTO_OK = 0,
+    DSFACTO_ERR_INVALID_ARG = -1, /* null pointer, size or hyper-parameter out of range */
+    DSFACTO_ERR_INVALID_CSR = -2, /* indptr not monotone, column ids not strictly increasing or out
+                                     of [0,d), non-finite value or label */
+    DSFACTO_ERR_NO_DATA = -3,     /* call needs dsfacto_load_csr first */
+    DSFACTO_ERR_OOM = -4,         /* host or device allocation failed */
+    DSFACTO_ERR_CUDA = -5,        /* CUDA runtime error (see dsfacto_last_error) */
+    DSFACTO_ERR_DIVERGED = -6     /* objective is NaN or infinite */
+};
+
+/* Problem statement of Section 3.2 plus the partition of Section 4.2.
+ *   n rows (1 <= n < 2^31), d columns (1 <= d), K latent factors (1 <= K <= 256), p tiles per side
+ *   (1 <= p <= 4096; p may exceed d or n, the surplus blocks are empty), loss DSFACTO_SQUARED or
+ *   DSFACTO_LOGISTIC, regularisers lambda_w, lambda_v >= 0, learning rate eta > 0.
+ * The per-entry step is eta / n (the objective carries 1/N, the printed updates do not).
+ * Initialisation (Algorithm 1, initialisation line): w0 = 0, w = 0, v_jk = 0.01 * z with z standard
+ * normal: element e = j*K+k takes outputs 2e and 2e+1 of SplitMix64 seeded with `seed`, maps each
+ * to (u>>11 + 0.5)/2^53 and applies Box-Muller (cosine branch); the product is rounded to fp32.
+ * On success *out holds a new handle (release with dsfacto_destroy). */
+int dsfacto_create(dsfacto_t **out, int64_t n, int32_t d, int32_t K, int32_t p, int32_t loss,
+                   float lambda_w, float lambda_v, float eta, uint64_t seed);
+
+/* Loads the training set X (CSR: indptr int64[n+1] with indptr[0] = 0, indices int32[nnz] strictly
+ * increasing inside each row and in [0,d), values fp32[nnz] finite; stored zeros count as entries)
+ * and labels y fp32[n] (finite).  Builds the p x p tile lists on the host (figure "communication
+ * pattern": row block of row i is floor(i*p/n), column block of column j is floor(j*p/d); tile
+ * (r,c) belongs to round s = (c-r) mod p; tiles ordered by (s, r); inside a tile entries ordered
+ * by (column, row)), copies CSR and tiles to the device and runs the recompute pass once, so that
+ * A, G and the objective of the initial parameters exist.  Replaces any earlier data set. */
+int dsfacto_load_csr(dsfacto_t *h, const int64_t *indptr, const int32_t *indices,
+                     const float *values, const float *y);
+
+/* One epoch (Algorithm 1, body of the loop over t):
+ *   w0 <- w0 - (eta/n) sum_i G_i                        (frozen G; df/dw0 = 1)
+ *   for s = 0..p-1, for the tiles (r,(r+s) mod p), for each stored (i,j,x) in tile order:
+ *       w_j  <- w_j  - (eta/n) (G_i x + lambda_w w_j)                          eq. (dsfacto_sgdupdatew)
+ *       v_jk <- v_jk - (eta/n) (G_i (x a_ik - v_jk x^2) + lambda_v v_jk)       eq. (dsfacto_sgdupdatev)
+ *   recompute a_ik (eq. (compute_a_jk)), f_i (eq. (fm_model2)), G_i and the objective (eq. (fm_obj)).
+ * Returns DSFACTO_ERR_DIVERGED if the new objective is not finite (state is kept). */
+int dsfacto_epoch(dsfacto_t *h);
+
+/* Raw scores f(x_i), eq. (fm_model2), of m rows given as CSR (same rules as dsfacto_load_csr) with
+ * the current parameters; scores_out fp32[m].  indptr == NULL scores the loaded training rows
+ * (m must then equal n). */
+int dsfacto_predict(dsfacto_t *h, int64_t m, const int64_t *indptr, const int32_t *indices,
+                    const float *values, float *scores_out);
+
+/* Objective eq. (fm_obj) as of the last recompute pass (after load_csr, epoch or set_params). */
+int dsfacto_objective(dsfacto_t *h, double *out);
+
+/* Copies out w0 (1), w (d) and V (d*K, row-major: V[j*K+k] = v_jk).  Any pointer may be NULL. */
+int dsfacto_get_params(dsfacto_t *h, float *w0, float *w, float *V);
+
+/* Overwrites the parameters (same layout as dsfacto_get_params; NULL keeps the current value) and,
+ * if data is loaded, reruns the recompute pass.  Checkpoint/restore and test injection; the paper
+ * has no counterpart. */
+int dsfacto_set_params(dsfacto_t *h, const float *w0, const float *w, const float *V);
+
+void dsfacto_destroy(dsfacto_t *h);
+
+/* ---- inspection (tests, tooling) ---- */
+
+/* Tile lists as built by dsfacto_load_csr, in the canonical order described there:
+ * tile_ptr int64[p*p+1] (tile t = s*p + r), rows int32[nnz], cols int32[nnz] (global ids),
+ * vals fp32[nnz]. */
+int dsfacto_get_tiles(dsfacto_t *h, int64_t *tile_ptr, int32_t *rows, int32_t *cols, float *vals);
+
+/* The host tile bucketer of dsfacto_load_csr on its own: same inputs (n rows, d columns, p tiles per
+ * side, CSR arrays), same checks, same output layout as dsfacto_get_tiles.  Touches no GPU. */
+int dsfacto_bucket_host(int64_t n, int32_t d, int32_t p, const int64_t *indptr, const int32_t *indices,
+                        const float *values, int64_t *tile_ptr, int32_t *rows, int32_t *cols, float *vals);
+
+/* Frozen auxiliaries of the last recompute pass: A fp32[n*K] row-major (a_ik), G fp32[n].
+ * Either pointer may be NULL. */
+int dsfacto_get_aux(dsfacto_t *h, float *A, float *G);
+
+/* Mean loss (1/N) sum_i l_i and sum_i G_i of the last recompute pass.  Either pointer may be NULL. */
+int dsfacto_get_stats(dsfacto_t *h, double *mean_loss, double *sum_G);
+
+/* ---- plumbing ---- */
+
+/* Runs all later device work of this handle on `cuda_stream` (a cudaStream_t passed as void*;
+ * NULL = the legacy default stream).  The stream stays owned by the caller. */
+int dsfacto_set_stream(dsfacto_t *h, void *cuda_stream);
+
+/* Device time of the last dsfacto_epoch from CUDA events on the handle's stream, in milliseconds:
+ * ms[0] whole epoch, ms[1] the p strata (update loop), ms[2] recompute pass (refresh + residual +
+ * loss sums), ms[3] parameter norms + final reduction. */
+int dsfacto_last_epoch_ms(dsfacto_t *h, float ms[4]);
+
+/* Number of kernels this handle has launched since creation. */
+int dsfacto_launch_count(dsfacto_t *h, int64_t *out);
+
+/* Text of the last CUDA/host error recorded on this handle ("" if none); valid until the next call. */
+const char *dsfacto_last_error(dsfacto_t *h);
+
+const char *dsfacto_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DSFACTO_H */

@@ -1,0 +1,706 @@
+// Host side of the DS-FACTO C ABI (include/dsfacto.h): handle, validation, seeded initialisation,
+// the tile bucketer, device memory, the epoch driver and the copy-out calls.
+#include "dsfacto.h"
+#include "dsfacto_kernels.cuh"
+
+#include <omp.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+namespace {
+
+using namespace dsf;
+
+struct DevBuf {
+    void *p = nullptr;
+    size_t bytes = 0;
+};
+
+}  // namespace
+
+struct dsfacto {
+    int64_t n = 0, nnz = 0;
+    int32_t d = 0, K = 0, Kp = 0, p = 0, loss = 0, LG = 1, NV = 1;
+    float lambda_w = 0, lambda_v = 0, eta = 0;
+    float h = 0;  // per-entry step eta / n
+    uint64_t seed = 0;
+    float w0 = 0.f;
+    bool loaded = false, wide = false;
+    int ibits = 0, jbits = 0;
+    cudaStream_t stream = nullptr;
+    cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
+    float ms[4] = {0, 0, 0, 0};
+    int64_t launches = 0;
+    int sm_count = 148;
+    std::string err;
+
+    std::vector<int64_t> row_start;  // p+1
+    std::vector<int32_t> col_start;  // p+1
+    std::vector<int64_t> tile_ptr;   // p*p+1
+
+    // device
+    float *d_w = nullptr, *d_V = nullptr, *d_A = nullptr, *d_G = nullptr, *d_y = nullptr, *d_val = nullptr, *d_xw = nullptr;
+    int64_t *d_indptr = nullptr, *d_tile_ptr = nullptr, *d_row_start = nullptr;
+    int32_t *d_idx = nullptr, *d_col_start = nullptr;
+    uint2 *d_ent = nullptr;
+    double *d_partials = nullptr, *d_scal = nullptr;
+    int refresh_grid = 0, norm_grid = 0;
+
+    double loss_sum = 0, g_sum = 0, w2 = 0, v2 = 0, objective = 0;
+};
+
+namespace {
+
+#define CU_TRY(h, call)                                                                     \
+    do {                                                                                    \
+        cudaError_t e_ = (call);                                                            \
+        if (e_ != cudaSuccess) {                                                            \
+            (h)->err = std::string(#call) + ": " + cudaGetErrorString(e_);                 \
+            return e_ == cudaErrorMemoryAllocation ? DSFACTO_ERR_OOM : DSFACTO_ERR_CUDA;    \
+        }                                                                                   \
+    } while (0)
+
+template <typename T>
+int dev_alloc(dsfacto *h, T **ptr, size_t count) {
+    *ptr = nullptr;
+    if (count == 0) count = 1;
+    CU_TRY(h, cudaMalloc((void **)ptr, count * sizeof(T)));
+    return DSFACTO_OK;
+}
+template <typename T>
+void dev_free(T *&ptr) {
+    if (ptr) cudaFree(ptr);
+    ptr = nullptr;
+}
+
+// ---- SplitMix64 (Steele, Lea, Flood 2014), random access to the c-th output ----
+inline uint64_t splitmix64_output(uint64_t seed, uint64_t c) {
+    uint64_t z = seed + (c + 1) * 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+inline double open_unit(uint64_t u) { return ((double)(u >> 11) + 0.5) * (1.0 / 9007199254740992.0); }
+inline float init_factor(uint64_t seed, uint64_t e) {
+    const double u1 = open_unit(splitmix64_output(seed, 2 * e));
+    const double u2 = open_unit(splitmix64_output(seed, 2 * e + 1));
+    const double z = std::sqrt(-2.0 * std::log(u1)) * std::cos(2.0 * 3.14159265358979323846 * u2);
+    return (float)(0.01 * z);
+}
+
+inline int bits_for(int64_t count) {  // bits needed for values in [0, count)
+    int b = 0;
+    while (((int64_t)1 << b) < count) ++b;
+    return b;
+}
+
+// partition: row block r = rows [ceil(r n / p), ceil((r+1) n / p)), i.e. floor(i p / n) = r; same for
+// columns.  Also chooses the packed (32-bit key) or wide entry layout.
+int setup_partition(dsfacto *h) {
+    const int64_t n = h->n;
+    const int32_t d = h->d, p = h->p;
+    try {
+        h->row_start.resize((size_t)p + 1);
+        h->col_start.resize((size_t)p + 1);
+    } catch (const std::bad_alloc &) { return DSFACTO_ERR_OOM; }
+    int64_t max_rows = 0, max_cols = 0;
+    for (int32_t r = 0; r <= p; ++r) {
+        h->row_start[r] = (int64_t)(((__int128)r * n + p - 1) / p);
+        h->col_start[r] = (int32_t)(((__int128)r * d + p - 1) / p);
+    }
+    for (int32_t r = 0; r < p; ++r) {
+        max_rows = std::max(max_rows, h->row_start[r + 1] - h->row_start[r]);
+        max_cols = std::max<int64_t>(max_cols, h->col_start[r + 1] - h->col_start[r]);
+    }
+    h->ibits = bits_for(max_rows);
+    h->jbits = bits_for(max_cols);
+    h->wide = (h->ibits + h->jbits) > 32;
+    if (h->wide) h->jbits = 32;
+    return DSFACTO_OK;
+}
+
+// canonical (global row, global column, value) lists from the packed device layout
+void unpack_tiles(const dsfacto *h, const uint2 *ent, const float *xw, int32_t *rows, int32_t *cols, float *vals) {
+    const int64_t nt = (int64_t)h->p * h->p;
+    const uint32_t jmask = h->jbits >= 32 ? 0xFFFFFFFFu : ((1u << h->jbits) - 1u);
+#pragma omp parallel for schedule(dynamic, 8)
+    for (int64_t t = 0; t < nt; ++t) {
+        const int64_t s = t / h->p, r = t % h->p, c = (r + s) % h->p;
+        for (int64_t q = h->tile_ptr[t]; q < h->tile_ptr[t + 1]; ++q) {
+            uint32_t il, jl;
+            float x;
+            if (h->wide) { il = ent[q].x; jl = ent[q].y; x = xw[q]; }
+            else { il = ent[q].x >> h->jbits; jl = ent[q].x & jmask; std::memcpy(&x, &ent[q].y, 4); }
+            if (rows) rows[q] = (int32_t)(h->row_start[r] + il);
+            if (cols) cols[q] = (int32_t)(h->col_start[c] + jl);
+            if (vals) vals[q] = x;
+        }
+    }
+}
+
+void free_data(dsfacto *h) {
+    dev_free(h->d_A); dev_free(h->d_G); dev_free(h->d_y); dev_free(h->d_val); dev_free(h->d_xw);
+    dev_free(h->d_indptr); dev_free(h->d_tile_ptr); dev_free(h->d_idx); dev_free(h->d_ent);
+    dev_free(h->d_partials);
+    h->loaded = false;
+    h->nnz = 0;
+}
+
+// ---------------------------------------------------------------------------------------------
+// kernel dispatch over the factor-row layout
+// ---------------------------------------------------------------------------------------------
+template <int LG, int NV>
+void launch_sgd(dsfacto *h, const SgdArgs &a) {
+    if (h->wide) sgd_round_kernel<LG, NV, true><<<h->p, kThreads, 0, h->stream>>>(a);
+    else sgd_round_kernel<LG, NV, false><<<h->p, kThreads, 0, h->stream>>>(a);
+}
+template <int LG, int NV>
+void launch_refresh(dsfacto *h, const RefreshArgs &a, bool train, int grid) {
+    if (train) refresh_kernel<LG, NV, true><<<grid, kThreads, 0, h->stream>>>(a);
+    else refresh_kernel<LG, NV, false><<<grid, kThreads, 0, h->stream>>>(a);
+}
+
+#define DSF_DISPATCH(h, FN, ...)                                   \
+    do {                                                           \
+        switch ((h)->LG * 10 + (h)->NV) {                          \
+        case 11: FN<1, 1>(__VA_ARGS__); break;                     \
+        case 21: FN<2, 1>(__VA_ARGS__); break;                     \
+        case 41: FN<4, 1>(__VA_ARGS__); break;                     \
+        case 81: FN<8, 1>(__VA_ARGS__); break;                     \
+        case 161: FN<16, 1>(__VA_ARGS__); break;                   \
+        case 321: FN<32, 1>(__VA_ARGS__); break;                   \
+        case 322: FN<32, 2>(__VA_ARGS__); break;                   \
+        default: break;                                            \
+        }                                                          \
+    } while (0)
+
+int refresh_grid_for(const dsfacto *h, int64_t rows) {
+    const int G = kThreads / h->LG;
+    int64_t want = (rows + G - 1) / G;
+    const int64_t cap = (int64_t)h->sm_count * 16;
+    if (want > cap) want = cap;
+    if (want < 1) want = 1;
+    return (int)want;
+}
+
+// recompute pass + norms + objective; ends with a stream sync and the four sums on the host
+int run_refresh(dsfacto *h, bool timed) {
+    RefreshArgs a{};
+    a.n = h->n; a.indptr = h->d_indptr; a.idx = h->d_idx; a.val = h->d_val; a.y = h->d_y;
+    a.w = h->d_w; a.V = h->d_V; a.A = h->d_A; a.G = h->d_G; a.f_out = nullptr;
+    a.partials = h->d_partials; a.w0 = h->w0; a.loss = h->loss;
+    DSF_DISPATCH(h, launch_refresh, h, a, true, h->refresh_grid);
+    reduce2_kernel<<<1, kThreads, 0, h->stream>>>(h->d_partials, h->refresh_grid, h->d_scal);
+    if (timed) cudaEventRecord(h->ev[2], h->stream);
+    double *np = h->d_partials + 2 * (size_t)h->refresh_grid;
+    sqnorm_kernel<<<h->norm_grid, kThreads, 0, h->stream>>>(h->d_w, h->d, h->d_V, (int64_t)h->d * h->Kp, np);
+    reduce2_kernel<<<1, kThreads, 0, h->stream>>>(np, h->norm_grid, h->d_scal + 2);
+    h->launches += 4;
+    if (timed) cudaEventRecord(h->ev[3], h->stream);
+    double s[4];
+    CU_TRY(h, cudaMemcpyAsync(s, h->d_scal, sizeof s, cudaMemcpyDeviceToHost, h->stream));
+    CU_TRY(h, cudaStreamSynchronize(h->stream));
+    CU_TRY(h, cudaGetLastError());
+    h->loss_sum = s[0]; h->g_sum = s[1]; h->w2 = s[2]; h->v2 = s[3];
+    h->objective = s[0] / (double)h->n + 0.5 * (double)h->lambda_w * s[2] + 0.5 * (double)h->lambda_v * s[3];
+    return DSFACTO_OK;
+}
+
+// V padded (d x Kp) <-> caller layout (d x K)
+int upload_V(dsfacto *h, const float *V) {
+    if (h->Kp == h->K) {
+        CU_TRY(h, cudaMemcpyAsync(h->d_V, V, sizeof(float) * (size_t)h->d * h->K, cudaMemcpyHostToDevice, h->stream));
+    } else {
+        CU_TRY(h, cudaMemsetAsync(h->d_V, 0, sizeof(float) * (size_t)h->d * h->Kp, h->stream));
+        CU_TRY(h, cudaMemcpy2DAsync(h->d_V, sizeof(float) * h->Kp, V, sizeof(float) * h->K, sizeof(float) * h->K,
+                                    (size_t)h->d, cudaMemcpyHostToDevice, h->stream));
+    }
+    CU_TRY(h, cudaStreamSynchronize(h->stream));
+    return DSFACTO_OK;
+}
+int download_rows(dsfacto *h, float *dst, const float *src_dev, int64_t rows) {
+    if (h->Kp == h->K) {
+        CU_TRY(h, cudaMemcpyAsync(dst, src_dev, sizeof(float) * (size_t)rows * h->K, cudaMemcpyDeviceToHost, h->stream));
+    } else {
+        CU_TRY(h, cudaMemcpy2DAsync(dst, sizeof(float) * h->K, src_dev, sizeof(float) * h->Kp, sizeof(float) * h->K,
+                                    (size_t)rows, cudaMemcpyDeviceToHost, h->stream));
+    }
+    CU_TRY(h, cudaStreamSynchronize(h->stream));
+    return DSFACTO_OK;
+}
+
+// CSR checks shared by load_csr and predict.  Returns DSFACTO_OK or DSFACTO_ERR_INVALID_CSR.
+int validate_csr(int64_t m, int32_t d, const int64_t *indptr, const int32_t *indices, const float *values) {
+    if (indptr[0] != 0) return DSFACTO_ERR_INVALID_CSR;
+    int bad = 0;
+#pragma omp parallel for schedule(static) reduction(| : bad)
+    for (int64_t i = 0; i < m; ++i) {
+        const int64_t b = indptr[i], e = indptr[i + 1];
+        if (e < b) { bad |= 1; continue; }
+        int32_t prev = -1;
+        for (int64_t t = b; t < e; ++t) {
+            const int32_t j = indices[t];
+            if (j <= prev || j >= d) bad |= 1;
+            prev = j;
+            if (!std::isfinite(values[t])) bad |= 1;
+        }
+    }
+    return bad ? DSFACTO_ERR_INVALID_CSR : DSFACTO_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host tile bucketer.  Output order: tiles by (round s, row block r); inside a tile by (column,
+// row).  Three passes over the stored entries: count per (thread, tile), scatter (keeps rows
+// ascending inside a tile because threads own ascending row ranges), then a stable counting sort
+// by local column inside every tile.
+// ---------------------------------------------------------------------------------------------
+int bucket_tiles(dsfacto *h, const int64_t *indptr, const int32_t *indices, const float *values,
+                 std::vector<uint2> &ent, std::vector<float> &xw) {
+    const int64_t n = h->n, nnz = indptr[n];
+    const int32_t d = h->d, p = h->p;
+    const int64_t nt = (int64_t)p * p;
+    const bool wide = h->wide;
+    const int jbits = h->jbits;
+    int T = omp_get_max_threads();
+    if (T > 64) T = 64;
+    if ((int64_t)T > n) T = (int)std::max<int64_t>(1, n);
+
+    std::vector<int32_t> cb(d);  // column block of every column
+    for (int32_t c = 0; c < p; ++c)
+        for (int32_t j = h->col_start[c]; j < h->col_start[c + 1]; ++j) cb[j] = c;
+
+    // thread k owns rows [rs[k], rs[k+1]) chosen to balance stored entries
+    std::vector<int64_t> rs(T + 1);
+    rs[0] = 0;
+    for (int k = 1; k < T; ++k) {
+        const int64_t target = (int64_t)((__int128)nnz * k / T);
+        rs[k] = std::lower_bound(indptr, indptr + n + 1, target) - indptr;
+        if (rs[k] > n) rs[k] = n;
+        if (rs[k] < rs[k - 1]) rs[k] = rs[k - 1];
+    }
+    rs[T] = n;
+
+    std::vector<uint32_t> counts;
+    std::vector<uint2> tmp_e;
+    std::vector<float> tmp_x;
+    try {
+        counts.assign((size_t)T * nt, 0u);
+        tmp_e.resize((size_t)std::max<int64_t>(nnz, 1));
+        if (wide) tmp_x.resize((size_t)std::max<int64_t>(nnz, 1));
+        ent.resize((size_t)std::max<int64_t>(nnz, 1));
+        if (wide) xw.resize((size_t)std::max<int64_t>(nnz, 1));
+    } catch (const std::bad_alloc &) {
+        return DSFACTO_ERR_OOM;
+    }
+    h->tile_ptr.assign((size_t)nt + 1, 0);
+
+#pragma omp parallel num_threads(T)
+    {
+        const int k = omp_get_thread_num();
+        uint32_t *cnt = counts.data() + (size_t)k * nt;
+        int64_t r = 0;
+        for (int64_t i = rs[k]; i < rs[k + 1]; ++i) {
+            while (i >= h->row_start[r + 1]) ++r;
+            for (int64_t e = indptr[i]; e < indptr[i + 1]; ++e) {
+                int64_t s = cb[indices[e]] - r;
+                if (s < 0) s += p;
+                cnt[s * p + r] += 1;
+            }
+        }
+    }
+    // offsets: tile-major, thread-minor
+    {
+        int64_t run = 0;
+        std::vector<int64_t> off((size_t)T);
+        for (int64_t t = 0; t < nt; ++t) {
+            h->tile_ptr[t] = run;
+            for (int k = 0; k < T; ++k) run += counts[(size_t)k * nt + t];
+        }
+        h->tile_ptr[nt] = run;
+    }
+    std::vector<int64_t> offs;
+    try { offs.resize((size_t)T * nt); } catch (const std::bad_alloc &) { return DSFACTO_ERR_OOM; }
+#pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < nt; ++t) {
+        int64_t run = h->tile_ptr[t];
+        for (int k = 0; k < T; ++k) { offs[(size_t)k * nt + t] = run; run += counts[(size_t)k * nt + t]; }
+    }
+#pragma omp parallel num_threads(T)
+    {
+        const int k = omp_get_thread_num();
+        int64_t *off = offs.data() + (size_t)k * nt;
+        int64_t r = 0;
+        for (int64_t i = rs[k]; i < rs[k + 1]; ++i) {
+            while (i >= h->row_start[r + 1]) ++r;
+            const uint32_t il = (uint32_t)(i - h->row_start[r]);
+            for (int64_t e = indptr[i]; e < indptr[i + 1]; ++e) {
+                const int32_t j = indices[e];
+                const int32_t c = cb[j];
+                int64_t s = c - r;
+                if (s < 0) s += p;
+                const int64_t at = off[s * p + r]++;
+                const uint32_t jl = (uint32_t)(j - h->col_start[c]);
+                if (wide) { tmp_e[at] = make_uint2(il, jl); tmp_x[at] = values[e]; }
+                else {
+                    uint32_t xb;
+                    std::memcpy(&xb, &values[e], 4);
+                    tmp_e[at] = make_uint2((il << jbits) | jl, xb);
+                }
+            }
+        }
+    }
+    // stable counting sort by local column inside each tile
+    const uint32_t jmask = jbits >= 32 ? 0xFFFFFFFFu : ((1u << jbits) - 1u);
+#pragma omp parallel
+    {
+        std::vector<int64_t> hist;
+#pragma omp for schedule(dynamic, 8)
+        for (int64_t t = 0; t < nt; ++t) {
+            const int64_t b = h->tile_ptr[t], e = h->tile_ptr[t + 1];
+            if (b == e) continue;
+            const int64_t s = t / p, r = t % p;
+            const int64_t c = (r + s) % p;
+            const int64_t width = h->col_start[c + 1] - h->col_start[c];
+            hist.assign((size_t)width + 1, 0);
+            for (int64_t q = b; q < e; ++q) {
+                const uint32_t jl = wide ? tmp_e[q].y : (tmp_e[q].x & jmask);
+                hist[jl + 1] += 1;
+            }
+            for (int64_t j = 0; j < width; ++j) hist[j + 1] += hist[j];
+            for (int64_t q = b; q < e; ++q) {
+                const uint32_t jl = wide ? tmp_e[q].y : (tmp_e[q].x & jmask);
+                const int64_t at = b + hist[jl]++;
+                ent[at] = tmp_e[q];
+                if (wide) xw[at] = tmp_x[q];
+            }
+        }
+    }
+    return DSFACTO_OK;
+}
+
+}  // namespace
+
+// =============================================================================================
+// C ABI
+// =============================================================================================
+extern "C" {
+
+const char *dsfacto_strerror(int status) {
+    switch (status) {
+    case DSFACTO_OK: return "ok";
+    case DSFACTO_ERR_INVALID_ARG: return "invalid argument";
+    case DSFACTO_ERR_INVALID_CSR: return "invalid CSR data or labels";
+    case DSFACTO_ERR_NO_DATA: return "no data loaded";
+    case DSFACTO_ERR_OOM: return "out of memory";
+    case DSFACTO_ERR_CUDA: return "CUDA error";
+    case DSFACTO_ERR_DIVERGED: return "objective is not finite";
+    default: return "unknown status";
+    }
+}
+
+const char *dsfacto_last_error(dsfacto_t *h) { return h ? h->err.c_str() : ""; }
+
+int dsfacto_create(dsfacto_t **out, int64_t n, int32_t d, int32_t K, int32_t p, int32_t loss, float lambda_w,
+                   float lambda_v, float eta, uint64_t seed) {
+    if (!out) return DSFACTO_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (n < 1 || n >= ((int64_t)1 << 31) || d < 1 || K < 1 || K > 256 || p < 1 || p > 4096) return DSFACTO_ERR_INVALID_ARG;
+    if (loss != DSFACTO_SQUARED && loss != DSFACTO_LOGISTIC) return DSFACTO_ERR_INVALID_ARG;
+    if (!(lambda_w >= 0.f) || !(lambda_v >= 0.f) || !(eta > 0.f) || !std::isfinite(lambda_w) ||
+        !std::isfinite(lambda_v) || !std::isfinite(eta))
+        return DSFACTO_ERR_INVALID_ARG;
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) return DSFACTO_ERR_CUDA;
+
+    dsfacto *h = new (std::nothrow) dsfacto();
+    if (!h) return DSFACTO_ERR_OOM;
+    h->n = n; h->d = d; h->K = K; h->p = p; h->loss = loss;
+    h->lambda_w = lambda_w; h->lambda_v = lambda_v; h->eta = eta; h->seed = seed;
+    h->h = (float)((double)eta / (double)n);
+    // factor-row layout: Kp = 4 * LG * NV >= K
+    const int q4 = (K + 3) / 4;
+    int LG = 1;
+    while (LG < q4 && LG < 32) LG <<= 1;
+    h->LG = LG;
+    h->NV = (q4 + LG - 1) / LG;
+    h->Kp = 4 * h->LG * h->NV;
+
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, dev);
+    if (h->sm_count < 1) h->sm_count = 148;
+
+    auto fail = [&](int rc) { dsfacto_destroy(h); return rc; };
+    if (setup_partition(h)) return fail(DSFACTO_ERR_OOM);
+
+    for (auto &e : h->ev)
+        if (cudaEventCreate(&e) != cudaSuccess) return fail(DSFACTO_ERR_CUDA);
+    int rc;
+    if ((rc = dev_alloc(h, &h->d_w, (size_t)d)) || (rc = dev_alloc(h, &h->d_V, (size_t)d * h->Kp)) ||
+        (rc = dev_alloc(h, &h->d_row_start, (size_t)p + 1)) || (rc = dev_alloc(h, &h->d_col_start, (size_t)p + 1)) ||
+        (rc = dev_alloc(h, &h->d_scal, 4)))
+        return fail(rc);
+
+    std::vector<float> V;
+    try { V.resize((size_t)d * K); } catch (const std::bad_alloc &) { return fail(DSFACTO_ERR_OOM); }
+#pragma omp parallel for schedule(static)
+    for (int64_t e = 0; e < (int64_t)d * K; ++e) V[(size_t)e] = init_factor(seed, (uint64_t)e);
+    h->w0 = 0.f;
+    if (cudaMemset(h->d_w, 0, sizeof(float) * (size_t)d) != cudaSuccess) return fail(DSFACTO_ERR_CUDA);
+    if ((rc = upload_V(h, V.data()))) return fail(rc);
+    if (cudaMemcpy(h->d_row_start, h->row_start.data(), sizeof(int64_t) * ((size_t)p + 1), cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(h->d_col_start, h->col_start.data(), sizeof(int32_t) * ((size_t)p + 1), cudaMemcpyHostToDevice) != cudaSuccess)
+        return fail(DSFACTO_ERR_CUDA);
+    h->norm_grid = h->sm_count * 8;
+    *out = h;
+    return DSFACTO_OK;
+}
+
+void dsfacto_destroy(dsfacto_t *h) {
+    if (!h) return;
+    cudaStreamSynchronize(h->stream);
+    free_data(h);
+    dev_free(h->d_w); dev_free(h->d_V); dev_free(h->d_row_start); dev_free(h->d_col_start); dev_free(h->d_scal);
+    for (auto &e : h->ev)
+        if (e) cudaEventDestroy(e);
+    delete h;
+}
+
+int dsfacto_set_stream(dsfacto_t *h, void *cuda_stream) {
+    if (!h) return DSFACTO_ERR_INVALID_ARG;
+    CU_TRY(h, cudaStreamSynchronize(h->stream));
+    h->stream = (cudaStream_t)cuda_stream;
+    return DSFACTO_OK;
+}
+
+int dsfacto_load_csr(dsfacto_t *h, const int64_t *indptr, const int32_t *indices, const float *values, const float *y) {
+    if (!h || !indptr || !y) return DSFACTO_ERR_INVALID_ARG;
+    const int64_t n = h->n;
+    if (indptr[0] != 0 || indptr[n] < 0) return DSFACTO_ERR_INVALID_CSR;
+    const int64_t nnz = indptr[n];
+    if (nnz > 0 && (!indices || !values)) return DSFACTO_ERR_INVALID_ARG;
+    int rc = validate_csr(n, h->d, indptr, indices, values);
+    if (rc) return rc;
+    int bad = 0;
+#pragma omp parallel for schedule(static) reduction(| : bad)
+    for (int64_t i = 0; i < n; ++i)
+        if (!std::isfinite(y[i])) bad |= 1;
+    if (bad) return DSFACTO_ERR_INVALID_CSR;
+
+    CU_TRY(h, cudaStreamSynchronize(h->stream));
+    free_data(h);
+    std::vector<uint2> ent;
+    std::vector<float> xw;
+    if ((rc = bucket_tiles(h, indptr, indices, values, ent, xw))) return rc;
+    h->nnz = nnz;
+    h->refresh_grid = refresh_grid_for(h, n);
+
+    const size_t cnt = (size_t)std::max<int64_t>(nnz, 1);
+    if ((rc = dev_alloc(h, &h->d_indptr, (size_t)n + 1)) || (rc = dev_alloc(h, &h->d_idx, cnt)) ||
+        (rc = dev_alloc(h, &h->d_val, cnt)) || (rc = dev_alloc(h, &h->d_y, (size_t)n)) ||
+        (rc = dev_alloc(h, &h->d_A, (size_t)n * h->Kp)) || (rc = dev_alloc(h, &h->d_G, (size_t)n)) ||
+        (rc = dev_alloc(h, &h->d_tile_ptr, h->tile_ptr.size())) || (rc = dev_alloc(h, &h->d_ent, cnt)) ||
+        (rc = dev_alloc(h, &h->d_partials, 2 * ((size_t)h->refresh_grid + (size_t)h->norm_grid)))) {
+        free_data(h);
+        return rc;
+    }
+    if (h->wide && (rc = dev_alloc(h, &h->d_xw, cnt))) { free_data(h); return rc; }
+    cudaStream_t st = h->stream;
+    CU_TRY(h, cudaMemcpyAsync(h->d_indptr, indptr, sizeof(int64_t) * ((size_t)n + 1), cudaMemcpyHostToDevice, st));
+    if (nnz > 0) {
+        CU_TRY(h, cudaMemcpyAsync(h->d_idx, indices, sizeof(int32_t) * (size_t)nnz, cudaMemcpyHostToDevice, st));
+        CU_TRY(h, cudaMemcpyAsync(h->d_val, values, sizeof(float) * (size_t)nnz, cudaMemcpyHostToDevice, st));
+        CU_TRY(h, cudaMemcpyAsync(h->d_ent, ent.data(), sizeof(uint2) * (size_t)nnz, cudaMemcpyHostToDevice, st));
+        if (h->wide) CU_TRY(h, cudaMemcpyAsync(h->d_xw, xw.data(), sizeof(float) * (size_t)nnz, cudaMemcpyHostToDevice, st));
+    }
+    CU_TRY(h, cudaMemcpyAsync(h->d_y, y, sizeof(float) * (size_t)n, cudaMemcpyHostToDevice, st));
+    CU_TRY(h, cudaMemcpyAsync(h->d_tile_ptr, h->tile_ptr.data(), sizeof(int64_t) * h->tile_ptr.size(), cudaMemcpyHostToDevice, st));
+    CU_TRY(h, cudaStreamSynchronize(st));
+    h->loaded = true;
+    rc = run_refresh(h, false);
+    if (rc) return rc;
+    return std::isfinite(h->objective) ? DSFACTO_OK : DSFACTO_ERR_DIVERGED;
+}
+
+int dsfacto_epoch(dsfacto_t *h) {
+    if (!h) return DSFACTO_ERR_INVALID_ARG;
+    if (!h->loaded) return DSFACTO_ERR_NO_DATA;
+    cudaStream_t st = h->stream;
+    CU_TRY(h, cudaEventRecord(h->ev[0], st));
+    // w0 step with the frozen multipliers
+    h->w0 = (float)((double)h->w0 - (double)h->h * h->g_sum);
+    SgdArgs a{};
+    a.tile_ptr = h->d_tile_ptr; a.ent = h->d_ent; a.xw = h->d_xw; a.row_start = h->d_row_start;
+    a.col_start = h->d_col_start; a.A = h->d_A; a.G = h->d_G; a.w = h->d_w; a.V = h->d_V;
+    a.p = h->p; a.jbits = h->jbits; a.h = h->h; a.lambda_w = h->lambda_w; a.lambda_v = h->lambda_v;
+    for (int s = 0; s < h->p; ++s) {
+        a.s = s;
+        DSF_DISPATCH(h, launch_sgd, h, a);
+    }
+    h->launches += h->p;
+    CU_TRY(h, cudaEventRecord(h->ev[1], st));
+    int rc = run_refresh(h, true);
+    if (rc) return rc;
+    float t01 = 0, t12 = 0, t23 = 0;
+    cudaEventElapsedTime(&t01, h->ev[0], h->ev[1]);
+    cudaEventElapsedTime(&t12, h->ev[1], h->ev[2]);
+    cudaEventElapsedTime(&t23, h->ev[2], h->ev[3]);
+    h->ms[0] = t01 + t12 + t23; h->ms[1] = t01; h->ms[2] = t12; h->ms[3] = t23;
+    return std::isfinite(h->objective) ? DSFACTO_OK : DSFACTO_ERR_DIVERGED;
+}
+
+int dsfacto_objective(dsfacto_t *h, double *out) {
+    if (!h || !out) return DSFACTO_ERR_INVALID_ARG;
+    if (!h->loaded) return DSFACTO_ERR_NO_DATA;
+    *out = h->objective;
+    return DSFACTO_OK;
+}
+
+int dsfacto_get_stats(dsfacto_t *h, double *mean_loss, double *sum_G) {
+    if (!h) return DSFACTO_ERR_INVALID_ARG;
+    if (!h->loaded) return DSFACTO_ERR_NO_DATA;
+    if (mean_loss) *mean_loss = h->loss_sum / (double)h->n;
+    if (sum_G) *sum_G = h->g_sum;
+    return DSFACTO_OK;
+}
+
+int dsfacto_get_params(dsfacto_t *h, float *w0, float *w, float *V) {
+    if (!h) return DSFACTO_ERR_INVALID_ARG;
+    if (w0) *w0 = h->w0;
+    if (w) {
+        CU_TRY(h, cudaMemcpyAsync(w, h->d_w, sizeof(float) * (size_t)h->d, cudaMemcpyDeviceToHost, h->stream));
+        CU_TRY(h, cudaStreamSynchronize(h->stream));
+    }
+    if (V) return download_rows(h, V, h->d_V, h->d);
+    return DSFACTO_OK;
+}
+
+int dsfacto_set_params(dsfacto_t *h, const float *w0, const float *w, const float *V) {
+    if (!h) return DSFACTO_ERR_INVALID_ARG;
+    if (w0) { if (!std::isfinite(*w0)) return DSFACTO_ERR_INVALID_ARG; h->w0 = *w0; }
+    if (w) {
+        CU_TRY(h, cudaMemcpyAsync(h->d_w, w, sizeof(float) * (size_t)h->d, cudaMemcpyHostToDevice, h->stream));
+        CU_TRY(h, cudaStreamSynchronize(h->stream));
+    }
+    if (V) { int rc = upload_V(h, V); if (rc) return rc; }
+    if (h->loaded) {
+        int rc = run_refresh(h, false);
+        if (rc) return rc;
+        if (!std::isfinite(h->objective)) return DSFACTO_ERR_DIVERGED;
+    }
+    return DSFACTO_OK;
+}
+
+int dsfacto_get_aux(dsfacto_t *h, float *A, float *G) {
+    if (!h) return DSFACTO_ERR_INVALID_ARG;
+    if (!h->loaded) return DSFACTO_ERR_NO_DATA;
+    if (G) {
+        CU_TRY(h, cudaMemcpyAsync(G, h->d_G, sizeof(float) * (size_t)h->n, cudaMemcpyDeviceToHost, h->stream));
+        CU_TRY(h, cudaStreamSynchronize(h->stream));
+    }
+    if (A) return download_rows(h, A, h->d_A, h->n);
+    return DSFACTO_OK;
+}
+
+int dsfacto_get_tiles(dsfacto_t *h, int64_t *tile_ptr, int32_t *rows, int32_t *cols, float *vals) {
+    if (!h) return DSFACTO_ERR_INVALID_ARG;
+    if (!h->loaded) return DSFACTO_ERR_NO_DATA;
+    const int64_t nt = (int64_t)h->p * h->p;
+    if (tile_ptr) std::memcpy(tile_ptr, h->tile_ptr.data(), sizeof(int64_t) * ((size_t)nt + 1));
+    if (!rows && !cols && !vals) return DSFACTO_OK;
+    std::vector<uint2> ent;
+    std::vector<float> xw;
+    try {
+        ent.resize((size_t)std::max<int64_t>(h->nnz, 1));
+        if (h->wide) xw.resize((size_t)std::max<int64_t>(h->nnz, 1));
+    } catch (const std::bad_alloc &) { return DSFACTO_ERR_OOM; }
+    if (h->nnz > 0) {
+        CU_TRY(h, cudaMemcpyAsync(ent.data(), h->d_ent, sizeof(uint2) * (size_t)h->nnz, cudaMemcpyDeviceToHost, h->stream));
+        if (h->wide) CU_TRY(h, cudaMemcpyAsync(xw.data(), h->d_xw, sizeof(float) * (size_t)h->nnz, cudaMemcpyDeviceToHost, h->stream));
+        CU_TRY(h, cudaStreamSynchronize(h->stream));
+    }
+    unpack_tiles(h, ent.data(), xw.data(), rows, cols, vals);
+    return DSFACTO_OK;
+}
+
+int dsfacto_bucket_host(int64_t n, int32_t d, int32_t p, const int64_t *indptr, const int32_t *indices,
+                        const float *values, int64_t *tile_ptr, int32_t *rows, int32_t *cols, float *vals) {
+    if (n < 1 || n >= ((int64_t)1 << 31) || d < 1 || p < 1 || p > 4096 || !indptr || !tile_ptr) return DSFACTO_ERR_INVALID_ARG;
+    if (indptr[0] != 0 || indptr[n] < 0) return DSFACTO_ERR_INVALID_CSR;
+    if (indptr[n] > 0 && (!indices || !values)) return DSFACTO_ERR_INVALID_ARG;
+    int rc = validate_csr(n, d, indptr, indices, values);
+    if (rc) return rc;
+    dsfacto tmp;
+    tmp.n = n; tmp.d = d; tmp.p = p;
+    if ((rc = setup_partition(&tmp))) return rc;
+    std::vector<uint2> ent;
+    std::vector<float> xw;
+    if ((rc = bucket_tiles(&tmp, indptr, indices, values, ent, xw))) return rc;
+    std::memcpy(tile_ptr, tmp.tile_ptr.data(), sizeof(int64_t) * tmp.tile_ptr.size());
+    unpack_tiles(&tmp, ent.data(), xw.data(), rows, cols, vals);
+    return DSFACTO_OK;
+}
+
+int dsfacto_predict(dsfacto_t *h, int64_t m, const int64_t *indptr, const int32_t *indices, const float *values,
+                    float *scores_out) {
+    if (!h || !scores_out || m < 0) return DSFACTO_ERR_INVALID_ARG;
+    if (m == 0) return DSFACTO_OK;
+    RefreshArgs a{};
+    a.w = h->d_w; a.V = h->d_V; a.w0 = h->w0; a.loss = h->loss; a.n = m;
+    int64_t *d_ip = nullptr;
+    int32_t *d_ix = nullptr;
+    float *d_vl = nullptr, *d_f = nullptr;
+    int rc = DSFACTO_OK;
+    auto cleanup = [&]() { dev_free(d_ip); dev_free(d_ix); dev_free(d_vl); dev_free(d_f); };
+    if (!indptr) {
+        if (!h->loaded) return DSFACTO_ERR_NO_DATA;
+        if (m != h->n) return DSFACTO_ERR_INVALID_ARG;
+        a.indptr = h->d_indptr; a.idx = h->d_idx; a.val = h->d_val;
+    } else {
+        if (indptr[0] != 0 || indptr[m] < 0) return DSFACTO_ERR_INVALID_CSR;
+        const int64_t nnz = indptr[m];
+        if (nnz > 0 && (!indices || !values)) return DSFACTO_ERR_INVALID_ARG;
+        if ((rc = validate_csr(m, h->d, indptr, indices, values))) return rc;
+        const size_t cnt = (size_t)std::max<int64_t>(nnz, 1);
+        if ((rc = dev_alloc(h, &d_ip, (size_t)m + 1)) || (rc = dev_alloc(h, &d_ix, cnt)) || (rc = dev_alloc(h, &d_vl, cnt))) {
+            cleanup();
+            return rc;
+        }
+        cudaMemcpyAsync(d_ip, indptr, sizeof(int64_t) * ((size_t)m + 1), cudaMemcpyHostToDevice, h->stream);
+        if (nnz > 0) {
+            cudaMemcpyAsync(d_ix, indices, sizeof(int32_t) * (size_t)nnz, cudaMemcpyHostToDevice, h->stream);
+            cudaMemcpyAsync(d_vl, values, sizeof(float) * (size_t)nnz, cudaMemcpyHostToDevice, h->stream);
+        }
+        a.indptr = d_ip; a.idx = d_ix; a.val = d_vl;
+    }
+    if ((rc = dev_alloc(h, &d_f, (size_t)m))) { cleanup(); return rc; }
+    a.f_out = d_f;
+    DSF_DISPATCH(h, launch_refresh, h, a, false, refresh_grid_for(h, m));
+    h->launches += 1;
+    cudaError_t e = cudaMemcpyAsync(scores_out, d_f, sizeof(float) * (size_t)m, cudaMemcpyDeviceToHost, h->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
+    if (e == cudaSuccess) e = cudaGetLastError();
+    cleanup();
+    if (e != cudaSuccess) { h->err = cudaGetErrorString(e); return DSFACTO_ERR_CUDA; }
+    return DSFACTO_OK;
+}
+
+int dsfacto_last_epoch_ms(dsfacto_t *h, float ms[4]) {
+    if (!h || !ms) return DSFACTO_ERR_INVALID_ARG;
+    for (int i = 0; i < 4; ++i) ms[i] = h->ms[i];
+    return DSFACTO_OK;
+}
+
+int dsfacto_launch_count(dsfacto_t *h, int64_t *out) {
+    if (!h || !out) return DSFACTO_ERR_INVALID_ARG;
+    *out = h->launches;
+    return DSFACTO_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,229 @@
+"""ctypes binding of the CUDA C-ABI library (include/dsfacto.h).
+
+Argument marshalling only: every step of the path runs inside libdsfacto.so.  There is no CPU
+fallback: if the library is missing or cannot be built, importing symbols raises; if no CUDA
+device is usable, dsfacto_create returns DSFACTO_ERR_CUDA and `DSFacto(...)` raises."""
+from __future__ import annotations
+
+import ctypes
+from typing import Optional
+
+import numpy as np
+
+from . import build as _build
+
+SQUARED, LOGISTIC = 0, 1
+OK, ERR_INVALID_ARG, ERR_INVALID_CSR, ERR_NO_DATA, ERR_OOM, ERR_CUDA, ERR_DIVERGED = 0, -1, -2, -3, -4, -5, -6
+
+_c_i64, _c_i32, _c_f32, _c_u64, _vp = ctypes.c_int64, ctypes.c_int32, ctypes.c_float, ctypes.c_uint64, ctypes.c_void_p
+
+# name -> (restype, argtypes); one entry per declaration in include/dsfacto.h
+SIGNATURES = {
+    "dsfacto_create": (ctypes.c_int, [ctypes.POINTER(_vp), _c_i64, _c_i32, _c_i32, _c_i32, _c_i32, _c_f32, _c_f32,
+                                      _c_f32, _c_u64]),
+    "dsfacto_load_csr": (ctypes.c_int, [_vp, _vp, _vp, _vp, _vp]),
+    "dsfacto_epoch": (ctypes.c_int, [_vp]),
+    "dsfacto_predict": (ctypes.c_int, [_vp, _c_i64, _vp, _vp, _vp, _vp]),
+    "dsfacto_objective": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_double)]),
+    "dsfacto_get_params": (ctypes.c_int, [_vp, _vp, _vp, _vp]),
+    "dsfacto_set_params": (ctypes.c_int, [_vp, _vp, _vp, _vp]),
+    "dsfacto_destroy": (None, [_vp]),
+    "dsfacto_get_tiles": (ctypes.c_int, [_vp, _vp, _vp, _vp, _vp]),
+    "dsfacto_bucket_host": (ctypes.c_int, [_c_i64, _c_i32, _c_i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "dsfacto_get_aux": (ctypes.c_int, [_vp, _vp, _vp]),
+    "dsfacto_get_stats": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]),
+    "dsfacto_set_stream": (ctypes.c_int, [_vp, _vp]),
+    "dsfacto_last_epoch_ms": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_float)]),
+    "dsfacto_launch_count": (ctypes.c_int, [_vp, ctypes.POINTER(_c_i64)]),
+    "dsfacto_last_error": (ctypes.c_char_p, [_vp]),
+    "dsfacto_strerror": (ctypes.c_char_p, [ctypes.c_int]),
+}
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads (building first if the sources are newer) libdsfacto.so; raises if that fails."""
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(str(_build.build_cuda()))
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(L, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = L
+    return _lib
+
+
+class DSFactoError(RuntimeError):
+    def __init__(self, status: int, where: str, detail: str = ""):
+        self.status = status
+        msg = lib().dsfacto_strerror(status).decode()
+        super().__init__("%s: %s (%d)%s" % (where, msg, status, (": " + detail) if detail else ""))
+
+
+def _ptr(a: Optional[np.ndarray]):
+    return None if a is None else ctypes.c_void_p(a.ctypes.data)
+
+
+# ---- the C calls under their own names (thin wrappers: numpy arrays in, status out) ----
+def dsfacto_create(n, d, K, p, loss, lambda_w, lambda_v, eta, seed):
+    h = _vp()
+    rc = lib().dsfacto_create(ctypes.byref(h), n, d, K, p, loss, lambda_w, lambda_v, eta, seed)
+    return rc, h
+
+
+def dsfacto_load_csr(h, indptr, indices, values, y):
+    return lib().dsfacto_load_csr(h, _ptr(indptr), _ptr(indices), _ptr(values), _ptr(y))
+
+
+def dsfacto_epoch(h):
+    return lib().dsfacto_epoch(h)
+
+
+def dsfacto_predict(h, m, indptr, indices, values, out):
+    return lib().dsfacto_predict(h, m, _ptr(indptr), _ptr(indices), _ptr(values), _ptr(out))
+
+
+def dsfacto_objective(h):
+    v = ctypes.c_double()
+    rc = lib().dsfacto_objective(h, ctypes.byref(v))
+    return rc, v.value
+
+
+def dsfacto_get_params(h, w0, w, V):
+    return lib().dsfacto_get_params(h, _ptr(w0), _ptr(w), _ptr(V))
+
+
+def dsfacto_set_params(h, w0, w, V):
+    return lib().dsfacto_set_params(h, _ptr(w0), _ptr(w), _ptr(V))
+
+
+def dsfacto_destroy(h):
+    lib().dsfacto_destroy(h)
+
+
+def dsfacto_bucket_host(n, d, p, indptr, indices, values):
+    """Host tile bucketer alone -> (status, tile_ptr, rows, cols, vals); needs no GPU."""
+    nnz = int(indptr[-1])
+    tile_ptr = np.zeros(p * p + 1, np.int64)
+    rows = np.empty(max(nnz, 1), np.int32)[:nnz]
+    cols = np.empty(max(nnz, 1), np.int32)[:nnz]
+    vals = np.empty(max(nnz, 1), np.float32)[:nnz]
+    rc = lib().dsfacto_bucket_host(n, d, p, _ptr(indptr), _ptr(indices), _ptr(values), _ptr(tile_ptr), _ptr(rows),
+                                   _ptr(cols), _ptr(vals))
+    return rc, tile_ptr, rows, cols, vals
+
+
+class DSFacto:
+    """Convenience owner of one handle.  Every method is one C call plus array allocation."""
+
+    def __init__(self, n, d, K, p, loss, lambda_w, lambda_v, eta, seed):
+        self.n, self.d, self.K, self.p = int(n), int(d), int(K), int(p)
+        rc, self._h = dsfacto_create(self.n, self.d, self.K, self.p, int(loss), float(lambda_w), float(lambda_v),
+                                     float(eta), int(seed))
+        if rc != OK:
+            self._h = None
+            raise DSFactoError(rc, "dsfacto_create")
+        self.nnz = 0
+
+    def _check(self, rc, where):
+        if rc != OK:
+            raise DSFactoError(rc, where, lib().dsfacto_last_error(self._h).decode())
+
+    def close(self):
+        if getattr(self, "_h", None):
+            dsfacto_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        self.close()
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    def set_stream(self, cuda_stream_ptr: int):
+        self._check(lib().dsfacto_set_stream(self._h, ctypes.c_void_p(cuda_stream_ptr)), "dsfacto_set_stream")
+
+    def load_csr(self, indptr, indices, values, y):
+        indptr = np.ascontiguousarray(indptr, np.int64)
+        indices = np.ascontiguousarray(indices, np.int32)
+        values = np.ascontiguousarray(values, np.float32)
+        y = np.ascontiguousarray(y, np.float32)
+        if indptr.shape != (self.n + 1,) or y.shape != (self.n,):
+            raise ValueError("indptr must have n+1 entries and y n entries")
+        if indices.shape[0] < indptr[-1] or values.shape[0] < indptr[-1]:
+            raise ValueError("indices/values shorter than indptr[-1]")
+        self._check(dsfacto_load_csr(self._h, indptr, indices, values, y), "dsfacto_load_csr")
+        self.nnz = int(indptr[-1])
+
+    def epoch(self) -> float:
+        self._check(dsfacto_epoch(self._h), "dsfacto_epoch")
+        return self.objective()
+
+    def objective(self) -> float:
+        rc, v = dsfacto_objective(self._h)
+        self._check(rc, "dsfacto_objective")
+        return v
+
+    def stats(self):
+        ml, sg = ctypes.c_double(), ctypes.c_double()
+        self._check(lib().dsfacto_get_stats(self._h, ctypes.byref(ml), ctypes.byref(sg)), "dsfacto_get_stats")
+        return ml.value, sg.value
+
+    def get_params(self):
+        w0 = np.zeros(1, np.float32)
+        w = np.empty(self.d, np.float32)
+        V = np.empty((self.d, self.K), np.float32)
+        self._check(dsfacto_get_params(self._h, w0, w, V), "dsfacto_get_params")
+        return float(w0[0]), w, V
+
+    def set_params(self, w0=None, w=None, V=None):
+        w0a = None if w0 is None else np.asarray([w0], np.float32)
+        wa = None if w is None else np.ascontiguousarray(w, np.float32)
+        Va = None if V is None else np.ascontiguousarray(V, np.float32)
+        if wa is not None and wa.shape != (self.d,):
+            raise ValueError("w must have d entries")
+        if Va is not None and Va.shape != (self.d, self.K):
+            raise ValueError("V must be d x K")
+        self._check(dsfacto_set_params(self._h, w0a, wa, Va), "dsfacto_set_params")
+
+    def predict(self, indptr=None, indices=None, values=None):
+        if indptr is None:
+            out = np.empty(self.n, np.float32)
+            self._check(dsfacto_predict(self._h, self.n, None, None, None, out), "dsfacto_predict")
+            return out
+        indptr = np.ascontiguousarray(indptr, np.int64)
+        indices = np.ascontiguousarray(indices, np.int32)
+        values = np.ascontiguousarray(values, np.float32)
+        m = indptr.shape[0] - 1
+        out = np.empty(max(m, 1), np.float32)[:m]
+        self._check(dsfacto_predict(self._h, m, indptr, indices, values, out), "dsfacto_predict")
+        return out
+
+    def get_tiles(self):
+        tile_ptr = np.empty(self.p * self.p + 1, np.int64)
+        rows = np.empty(max(self.nnz, 1), np.int32)[: self.nnz]
+        cols = np.empty(max(self.nnz, 1), np.int32)[: self.nnz]
+        vals = np.empty(max(self.nnz, 1), np.float32)[: self.nnz]
+        self._check(lib().dsfacto_get_tiles(self._h, _ptr(tile_ptr), _ptr(rows), _ptr(cols), _ptr(vals)),
+                    "dsfacto_get_tiles")
+        return tile_ptr, rows, cols, vals
+
+    def get_aux(self):
+        A = np.empty((self.n, self.K), np.float32)
+        G = np.empty(self.n, np.float32)
+        self._check(lib().dsfacto_get_aux(self._h, _ptr(A), _ptr(G)), "dsfacto_get_aux")
+        return A, G
+
+    def last_epoch_ms(self):
+        ms = (ctypes.c_float * 4)()
+        self._check(lib().dsfacto_last_epoch_ms(self._h, ms), "dsfacto_last_epoch_ms")
+        return [float(x) for x in ms]
+
+    def launch_count(self) -> int:
+        v = _c_i64()
+        self._check(lib().dsfacto_launch_count(self._h, ctypes.byref(v)), "dsfacto_launch_count")
+        return int(v.value)
