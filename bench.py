@@ -1,0 +1,310 @@
+#!/usr/bin/env python
+"""Throughput of the DS-FACTO epoch on B200: nonzero-updates/s = nnz x epochs / seconds.
+
+A step is one dsfacto_epoch (w0 step, the p strata, the recompute pass, the objective) over the
+C4 synthetic workload (hashed categorical, n = 45M, d = 2^20, 39 entries per row, K = 16, p = 512).
+  value      inputs resident in HBM; CUDA events around exactly K epochs on the library's stream
+  e2e        dsfacto_load_csr from host buffers (host bucketing + host->device copies) + one epoch +
+             the objective read back, through the C ABI
+  roofline   dominant kernel (stratum SGD): algorithmic bytes / measured launch time vs the
+             measured HBM copy peak
+  cpu_baseline   the CPU oracle, as it stands, on a bounded row sample of the same workload
+
+--impl reference times the CPU oracle alone.  --gpus N (under torchrun) runs N independent
+replicas (the path is single-GPU; no collective on the data path)."""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+from pathlib import Path
+
+import numpy as np
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+METRIC = "nonzero-updates/sec"
+UNIT = "updates/s"
+ORACLE_SAMPLE_ROWS = 1_000_000
+
+
+def peaks():
+    f = ROOT / "MEASURED_PEAKS.json"
+    if f.exists():
+        try:
+            return float(json.loads(f.read_text())["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.proc = None
+        self.index = index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_leg(wl_name: str, rows: int, min_seconds: float, max_epochs: int):
+    """Times oracle epochs (as the oracle stands) on the first `rows` rows' worth of the workload."""
+    from oracle import dsfacto_oracle as O
+    from paper_2004_13940_b200 import workloads as W
+
+    wl = W.make(wl_name, n=rows)
+    o = O.Oracle(wl.n, wl.d, wl.K, wl.p, wl.loss, wl.lambda_w, wl.lambda_v, wl.eta, wl.init_seed)
+    o.load_csr(wl.indptr, wl.indices, wl.values, wl.y)
+    o.epoch()                                   # untimed: page in, OpenMP team start
+    t0 = time.perf_counter()
+    epochs = 0
+    while epochs < max_epochs and (epochs == 0 or time.perf_counter() - t0 < min_seconds):
+        o.epoch()
+        epochs += 1
+    dt = time.perf_counter() - t0
+    cores = int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
+    return {"value": wl.nnz * epochs / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "%s generator, first %d rows (nnz %d), p=%d, %d oracle epochs in %.1f s (fp64, OpenMP over the "
+                      "tiles of a round)" % (wl_name, wl.n, wl.nnz, wl.p, epochs, dt),
+            "seconds": dt, "epochs": epochs, "nnz": wl.nnz}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import dsfacto_oracle as O
+    from paper_2004_13940_b200 import workloads as W
+
+    wl = W.make(args.workload, n=args.oracle_rows)
+    o = O.Oracle(wl.n, wl.d, wl.K, wl.p, wl.loss, wl.lambda_w, wl.lambda_v, wl.eta, wl.init_seed)
+    o.load_csr(wl.indptr, wl.indices, wl.values, wl.y)
+    per_step = []
+    for step in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        o.epoch()
+        if step >= args.warmup:
+            per_step.append(time.perf_counter() - t0)
+    total = sum(per_step)
+    value = wl.nnz * len(per_step) / total
+    info = {"cores": int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))}
+    cfg = workload_config(args.workload, sample_rows=args.oracle_rows)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(per_step),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": cfg,
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": info["cores"], "kind": "oracle",
+                             "sample": "each step = one oracle epoch on the first %d rows of the %s generator"
+                                       % (args.oracle_rows, args.workload)},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(name, sample_rows=None):
+    from paper_2004_13940_b200 import workloads as W
+    c = W.CONFIGS[name]
+    cfg = {"workload": name, "n": c["n"], "d": c["d"], "K": c["K"], "p": c["p"],
+           "loss": "logistic" if c["loss"] else "squared", "eta": c["eta"], "lambda": 1e-3,
+           "l2": "inputs larger than L2 (no flush needed)"}
+    if sample_rows is not None:
+        cfg["sample_rows"] = sample_rows
+    return cfg
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2004_13940_b200 import dsfacto as D
+    from paper_2004_13940_b200 import workloads as W
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    D.lib()
+    # pinned host buffers for the CSR arrays: they are the e2e leg's source
+    def pinned_empty(count, dtype):
+        t = torch.empty(int(count), dtype={np.int64: torch.int64, np.int32: torch.int32,
+                                          np.float32: torch.float32}[np.dtype(dtype).type], pin_memory=args.pin)
+        return t.numpy()
+
+    t_gen = time.perf_counter()
+    wl = W.make(args.workload, n=args.rows, empty=pinned_empty)
+    t_gen = time.perf_counter() - t_gen
+    nnz = wl.nnz
+    stream = torch.cuda.current_stream()
+
+    def new_handle():
+        g = D.DSFacto(wl.n, wl.d, wl.K, wl.p, wl.loss, wl.lambda_w, wl.lambda_v, wl.eta, wl.init_seed)
+        g.set_stream(stream.cuda_stream)
+        return g
+
+    # ranks load one after another so that the host-side bucketing buffers never coexist
+    g = None
+    t_load = 0.0
+    for turn in range(world):
+        if turn == rank:
+            t0 = time.perf_counter()
+            g = new_handle()
+            g.load_csr(wl.indptr, wl.indices, wl.values, wl.y)
+            t_load = time.perf_counter() - t0
+        barrier()
+
+    for _ in range(args.warmup):
+        g.epoch()
+    sampler = ClockSampler(local)
+    launches0 = g.launch_count()
+    barrier(); torch.cuda.synchronize()
+    if rank == 0:
+        sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    phase = np.zeros(4)
+    ev0.record(stream)
+    for _ in range(args.steps):
+        g.epoch()
+        phase += np.asarray(g.last_epoch_ms())
+    ev1.record(stream)
+    torch.cuda.synchronize(); barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    ms = ev0.elapsed_time(ev1)
+    launches = g.launch_count() - launches0
+    objective = g.objective()
+    g.close()
+
+    # ---- e2e: host buffers -> load_csr -> epoch -> objective, through the C ABI ----
+    e2e_ms = 0.0
+    for turn in range(world):
+        if turn == rank:
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            for _ in range(args.e2e_steps):
+                h = new_handle()
+                h.load_csr(wl.indptr, wl.indices, wl.values, wl.y)
+                h.epoch()
+                _ = h.objective()
+                h.close()
+            torch.cuda.synchronize()
+            e2e_ms = 1e3 * (time.perf_counter() - t0)
+        barrier()
+
+    if world > 1:
+        t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, e2e_ms = float(t[0]), float(t[1])
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    phase /= args.steps
+    peak, peak_kind = peaks()
+    K, n, d, p = wl.K, wl.n, wl.d, wl.p
+    # stratum SGD, per epoch: every entry reads its 8-byte record, G_i and the K-wide row a_i (no reuse
+    # inside a round: the p tiles of a round own disjoint row blocks), plus w, V read+written once
+    sgd_bytes = nnz * (8 + 4 * K + 4) + 8 * d * (K + 1)
+    sgd_floor = 8 * nnz + 4 * n * (K + 1) + 8 * d * (K + 1)
+    ref_bytes = 8 * nnz + 8 * (n + 1) + 4 * d * (K + 2) + 4 * n * K + 8 * n
+    sgd_s, ref_s = phase[1] * 1e-3, phase[2] * 1e-3
+    roof = {"bound": "hbm", "kernel": "sgd_round_kernel", "launches_per_step": p,
+            "achieved": sgd_bytes / sgd_s / 1e9, "peak": peak, "unit": "GB/s", "frac": sgd_bytes / sgd_s / 1e9 / peak,
+            "peak_kind": "of " + peak_kind, "traffic": None,
+            "algorithmic_bytes_per_step": sgd_bytes, "avg_launch_us": 1e6 * sgd_s / p,
+            "model": "gather: nnz*(8+4K+4) + 8d(K+1)",
+            "stream_floor": {"bytes_per_step": sgd_floor, "achieved": sgd_floor / sgd_s / 1e9,
+                             "frac": sgd_floor / sgd_s / 1e9 / peak},
+            "refresh_kernel": {"algorithmic_bytes_per_step": ref_bytes, "ms": phase[2],
+                               "achieved": ref_bytes / ref_s / 1e9, "frac": ref_bytes / ref_s / 1e9 / peak}}
+    value = world * nnz * args.steps / (ms * 1e-3)
+    h2d = (wl.indptr.nbytes + wl.indices.nbytes + wl.values.nbytes + wl.y.nbytes + 8 * nnz + 8 * (p * p + 1))
+    e2e = {"value": world * nnz * args.e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+           "d2h_bytes_per_step": 32, "steps": args.e2e_steps, "ms_per_step": e2e_ms / args.e2e_steps,
+           "what": "dsfacto_create + dsfacto_load_csr (host bucketing, H2D) + dsfacto_epoch + dsfacto_objective"}
+    cfg = workload_config(args.workload)
+    cfg.update({"n": n, "nnz": nnz, "parallelism": "replicas x%d" % world if world > 1 else "single GPU",
+                "pinned_host": bool(args.pin)})
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": cfg, "clocks": clocks, "e2e": e2e,
+            "gpu_launches": int(launches), "roofline": roof,
+            "phase_ms": {"epoch": phase[0], "sgd_strata": phase[1], "refresh": phase[2], "norms": phase[3]},
+            "objective": objective, "setup_s": {"generate": t_gen, "create+load_csr": t_load}}
+    if world == 1 and not args.no_cpu_baseline:
+        cb = oracle_leg(args.workload, args.oracle_rows, args.oracle_seconds, 50)
+        line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="C4")
+    ap.add_argument("--rows", type=int, default=None, help="override the workload's row count (profiling)")
+    ap.add_argument("--e2e-steps", type=int, default=1)
+    ap.add_argument("--oracle-rows", type=int, default=ORACLE_SAMPLE_ROWS)
+    ap.add_argument("--oracle-seconds", type=float, default=10.0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-pin", dest="pin", action="store_false")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
