@@ -178,7 +178,7 @@ def run_ours(args):
         return t.numpy()
 
     t_gen = time.perf_counter()
-    wl = W.make(args.workload, n=args.rows, empty=pinned_empty)
+    wl = W.make(args.workload, n=args.rows, p=args.p, empty=pinned_empty)
     t_gen = time.perf_counter() - t_gen
     nnz = wl.nnz
     stream = torch.cuda.current_stream()
@@ -254,7 +254,7 @@ def run_ours(args):
     sgd_floor = 8 * nnz + 4 * n * (K + 1) + 8 * d * (K + 1)
     ref_bytes = 8 * nnz + 8 * (n + 1) + 4 * d * (K + 2) + 4 * n * K + 8 * n
     sgd_s, ref_s = phase[1] * 1e-3, phase[2] * 1e-3
-    roof = {"bound": "hbm", "kernel": "sgd_round_kernel", "launches_per_step": p,
+    roof = {"bound": "hbm", "kernel": "sgd_chunk_kernel", "launches_per_step": p,
             "achieved": sgd_bytes / sgd_s / 1e9, "peak": peak, "unit": "GB/s", "frac": sgd_bytes / sgd_s / 1e9 / peak,
             "peak_kind": "of " + peak_kind, "traffic": None,
             "algorithmic_bytes_per_step": sgd_bytes, "avg_launch_us": 1e6 * sgd_s / p,
@@ -265,11 +265,11 @@ def run_ours(args):
                                "achieved": ref_bytes / ref_s / 1e9, "frac": ref_bytes / ref_s / 1e9 / peak}}
     value = world * nnz * args.steps / (ms * 1e-3)
     h2d = (wl.indptr.nbytes + wl.indices.nbytes + wl.values.nbytes + wl.y.nbytes + 8 * nnz + 8 * (p * p + 1))
-    e2e = {"value": world * nnz * args.e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
-           "d2h_bytes_per_step": 32, "steps": args.e2e_steps, "ms_per_step": e2e_ms / args.e2e_steps,
+    e2e = {"value": world * nnz * args.e2e_steps / (e2e_ms * 1e-3) if args.e2e_steps > 0 else None, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+           "d2h_bytes_per_step": 32, "steps": args.e2e_steps, "ms_per_step": e2e_ms / max(args.e2e_steps, 1),
            "what": "dsfacto_create + dsfacto_load_csr (host bucketing, H2D) + dsfacto_epoch + dsfacto_objective"}
     cfg = workload_config(args.workload)
-    cfg.update({"n": n, "nnz": nnz, "parallelism": "replicas x%d" % world if world > 1 else "single GPU",
+    cfg.update({"n": n, "p": p, "nnz": nnz, "parallelism": "replicas x%d" % world if world > 1 else "single GPU",
                 "pinned_host": bool(args.pin)})
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
@@ -293,6 +293,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C4")
     ap.add_argument("--rows", type=int, default=None, help="override the workload's row count (profiling)")
+    ap.add_argument("--p", type=int, default=None, help="override the tile grid (profiling)")
     ap.add_argument("--e2e-steps", type=int, default=1)
     ap.add_argument("--oracle-rows", type=int, default=ORACLE_SAMPLE_ROWS)
     ap.add_argument("--oracle-seconds", type=float, default=10.0)

@@ -1,13 +1,15 @@
 // Host side of the DS-FACTO C ABI (include/dsfacto.h): handle, validation, seeded initialisation,
 // the tile bucketer, device memory, the epoch driver and the copy-out calls.
 #include "dsfacto.h"
-#include "dsfacto_kernels.cuh"
+#include "dsfacto_refresh.cuh"
+#include "dsfacto_sgd.cuh"
 
 #include <omp.h>
 
 #include <algorithm>
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <string>
@@ -16,11 +18,6 @@
 namespace {
 
 using namespace dsf;
-
-struct DevBuf {
-    void *p = nullptr;
-    size_t bytes = 0;
-};
 
 }  // namespace
 
@@ -50,6 +47,12 @@ struct dsfacto {
     int32_t *d_idx = nullptr, *d_col_start = nullptr;
     uint2 *d_ent = nullptr;
     double *d_partials = nullptr, *d_scal = nullptr;
+    // stratum SGD launch plan: launch L covers chunks [launch_ptr[L], launch_ptr[L+1]) of chunk_map
+    int sweep = 1;  // 1: a launch is a row block (p-1 .. 0); 0: a launch is an inner round (0 .. p-1)
+    std::vector<int64_t> launch_ptr;
+    int2 *d_chunk_map = nullptr;
+    float *d_records = nullptr, *d_Tb = nullptr, *d_Td = nullptr;
+    int *d_tile_count = nullptr;
     int refresh_grid = 0, norm_grid = 0;
 
     double loss_sum = 0, g_sum = 0, w2 = 0, v2 = 0, objective = 0;
@@ -147,7 +150,8 @@ void unpack_tiles(const dsfacto *h, const uint2 *ent, const float *xw, int32_t *
 void free_data(dsfacto *h) {
     dev_free(h->d_A); dev_free(h->d_G); dev_free(h->d_y); dev_free(h->d_val); dev_free(h->d_xw);
     dev_free(h->d_indptr); dev_free(h->d_tile_ptr); dev_free(h->d_idx); dev_free(h->d_ent);
-    dev_free(h->d_partials);
+    dev_free(h->d_partials); dev_free(h->d_chunk_map); dev_free(h->d_records); dev_free(h->d_tile_count);
+    h->launch_ptr.clear();
     h->loaded = false;
     h->nnz = 0;
 }
@@ -156,9 +160,9 @@ void free_data(dsfacto *h) {
 // kernel dispatch over the factor-row layout
 // ---------------------------------------------------------------------------------------------
 template <int LG, int NV>
-void launch_sgd(dsfacto *h, const SgdArgs &a) {
-    if (h->wide) sgd_round_kernel<LG, NV, true><<<h->p, kThreads, 0, h->stream>>>(a);
-    else sgd_round_kernel<LG, NV, false><<<h->p, kThreads, 0, h->stream>>>(a);
+void launch_sgd(dsfacto *h, const SgdChunkArgs &a, int grid) {
+    if (h->wide) sgd_chunk_kernel<LG, NV, true><<<grid, kThreads, 0, h->stream>>>(a);
+    else sgd_chunk_kernel<LG, NV, false><<<grid, kThreads, 0, h->stream>>>(a);
 }
 template <int LG, int NV>
 void launch_refresh(dsfacto *h, const RefreshArgs &a, bool train, int grid) {
@@ -187,6 +191,64 @@ int refresh_grid_for(const dsfacto *h, int64_t rows) {
     if (want > cap) want = cap;
     if (want < 1) want = 1;
     return (int)want;
+}
+
+// Launch plan of the stratum SGD phase: which tiles each launch covers and how they split into
+// chunks of kChunk entries.  Tiles of one launch have pairwise disjoint column blocks.
+int build_sgd_plan(dsfacto *h) {
+    const int64_t p = h->p;
+    std::vector<int2> map;
+    int64_t max_launch = 0;
+    try {
+        h->launch_ptr.assign((size_t)p + 1, 0);
+        map.reserve((size_t)(h->nnz / kChunk + p * p / 4 + 16));
+        for (int64_t L = 0; L < p; ++L) {
+            for (int64_t k = 0; k < p; ++k) {
+                int64_t r, s;
+                if (h->sweep == 1) { r = p - 1 - L; s = ((k - r) % p + p) % p; }   // column block c = k
+                else { s = L; r = k; }
+                const int64_t t = s * p + r;
+                const int64_t cnt = h->tile_ptr[t + 1] - h->tile_ptr[t];
+                const int64_t nch = (cnt + kChunk - 1) / kChunk;
+                for (int64_t ci = 0; ci < nch; ++ci) map.push_back(make_int2((int)t, (int)ci));
+            }
+            h->launch_ptr[L + 1] = (int64_t)map.size();
+            max_launch = std::max(max_launch, h->launch_ptr[L + 1] - h->launch_ptr[L]);
+        }
+    } catch (const std::bad_alloc &) { return DSFACTO_ERR_OOM; }
+    int rc;
+    if ((rc = dev_alloc(h, &h->d_chunk_map, map.size())) ||
+        (rc = dev_alloc(h, &h->d_records, (size_t)max_launch * chunk_record_floats(h->Kp))) ||
+        (rc = dev_alloc(h, &h->d_tile_count, (size_t)(p * p))))
+        return rc;
+    CU_TRY(h, cudaMemsetAsync(h->d_tile_count, 0, sizeof(int) * (size_t)(p * p), h->stream));
+    if (!map.empty())
+        CU_TRY(h, cudaMemcpyAsync(h->d_chunk_map, map.data(), sizeof(int2) * map.size(), cudaMemcpyHostToDevice, h->stream));
+    CU_TRY(h, cudaStreamSynchronize(h->stream));
+    return DSFACTO_OK;
+}
+
+// the p strata of one epoch (plus, after a row-block sweep, folding the tail composites in)
+void run_sgd_phase(dsfacto *h) {
+    SgdChunkArgs a{};
+    a.tile_ptr = h->d_tile_ptr; a.ent = h->d_ent; a.xw = h->d_xw; a.row_start = h->d_row_start;
+    a.col_start = h->d_col_start; a.A = h->d_A; a.G = h->d_G; a.w = h->d_w; a.V = h->d_V;
+    a.Tb = h->d_Tb; a.Td = h->d_Td; a.records = h->d_records; a.tile_count = h->d_tile_count;
+    a.p = h->p; a.jbits = h->jbits; a.sweep = h->sweep;
+    a.h = h->h; a.lambda_w = h->lambda_w; a.lambda_v = h->lambda_v;
+    for (int L = 0; L < h->p; ++L) {
+        const int64_t grid = h->launch_ptr[L + 1] - h->launch_ptr[L];
+        if (grid == 0) continue;
+        a.chunk_map = h->d_chunk_map + h->launch_ptr[L];
+        DSF_DISPATCH(h, launch_sgd, h, a, (int)grid);
+        h->launches += 1;
+    }
+    if (h->sweep == 1 && h->p > 1) {
+        const int grid = h->sm_count * 8;
+        sgd_finalize_v_kernel<<<grid, kThreads, 0, h->stream>>>(h->d_V, h->d_Tb, h->d_Td, h->d, h->Kp / 4);
+        sgd_finalize_w_kernel<<<grid, kThreads, 0, h->stream>>>(h->d_w, h->d_Td, h->d);
+        h->launches += 2;
+    }
 }
 
 // recompute pass + norms + objective; ends with a stream sync and the four sums on the host
@@ -458,6 +520,13 @@ int dsfacto_create(dsfacto_t **out, int64_t n, int32_t d, int32_t K, int32_t p, 
         cudaMemcpy(h->d_col_start, h->col_start.data(), sizeof(int32_t) * ((size_t)p + 1), cudaMemcpyHostToDevice) != cudaSuccess)
         return fail(DSFACTO_ERR_CUDA);
     h->norm_grid = h->sm_count * 8;
+    if (const char *env = std::getenv("DSFACTO_SWEEP")) h->sweep = (std::strcmp(env, "round") == 0) ? 0 : 1;
+    if (h->sweep == 1) {
+        if ((rc = dev_alloc(h, &h->d_Tb, (size_t)d * h->Kp)) || (rc = dev_alloc(h, &h->d_Td, (size_t)d * 4))) return fail(rc);
+        if (cudaMemset(h->d_Tb, 0, sizeof(float) * (size_t)d * h->Kp) != cudaSuccess ||
+            cudaMemset(h->d_Td, 0, sizeof(float) * (size_t)d * 4) != cudaSuccess)
+            return fail(DSFACTO_ERR_CUDA);
+    }
     *out = h;
     return DSFACTO_OK;
 }
@@ -466,7 +535,7 @@ void dsfacto_destroy(dsfacto_t *h) {
     if (!h) return;
     cudaStreamSynchronize(h->stream);
     free_data(h);
-    dev_free(h->d_w); dev_free(h->d_V); dev_free(h->d_row_start); dev_free(h->d_col_start); dev_free(h->d_scal);
+    dev_free(h->d_w); dev_free(h->d_V); dev_free(h->d_Tb); dev_free(h->d_Td); dev_free(h->d_row_start); dev_free(h->d_col_start); dev_free(h->d_scal);
     for (auto &e : h->ev)
         if (e) cudaEventDestroy(e);
     delete h;
@@ -522,6 +591,7 @@ int dsfacto_load_csr(dsfacto_t *h, const int64_t *indptr, const int32_t *indices
     CU_TRY(h, cudaMemcpyAsync(h->d_y, y, sizeof(float) * (size_t)n, cudaMemcpyHostToDevice, st));
     CU_TRY(h, cudaMemcpyAsync(h->d_tile_ptr, h->tile_ptr.data(), sizeof(int64_t) * h->tile_ptr.size(), cudaMemcpyHostToDevice, st));
     CU_TRY(h, cudaStreamSynchronize(st));
+    if ((rc = build_sgd_plan(h))) { free_data(h); return rc; }
     h->loaded = true;
     rc = run_refresh(h, false);
     if (rc) return rc;
@@ -535,15 +605,7 @@ int dsfacto_epoch(dsfacto_t *h) {
     CU_TRY(h, cudaEventRecord(h->ev[0], st));
     // w0 step with the frozen multipliers
     h->w0 = (float)((double)h->w0 - (double)h->h * h->g_sum);
-    SgdArgs a{};
-    a.tile_ptr = h->d_tile_ptr; a.ent = h->d_ent; a.xw = h->d_xw; a.row_start = h->d_row_start;
-    a.col_start = h->d_col_start; a.A = h->d_A; a.G = h->d_G; a.w = h->d_w; a.V = h->d_V;
-    a.p = h->p; a.jbits = h->jbits; a.h = h->h; a.lambda_w = h->lambda_w; a.lambda_v = h->lambda_v;
-    for (int s = 0; s < h->p; ++s) {
-        a.s = s;
-        DSF_DISPATCH(h, launch_sgd, h, a);
-    }
-    h->launches += h->p;
+    run_sgd_phase(h);
     CU_TRY(h, cudaEventRecord(h->ev[1], st));
     int rc = run_refresh(h, true);
     if (rc) return rc;

@@ -1,0 +1,140 @@
+// Recompute-pass kernels of the DS-FACTO epoch for sm_100a: auxiliaries, scores, multipliers, and the
+// fp64 sums behind the objective.
+#pragma once
+#include "dsfacto_common.cuh"
+
+namespace dsf {
+
+// ------------------------------------------------------------------------------------------
+// Recompute pass (eq. (compute_a_jk), eq. (fm_model2), multiplier G): one lane group per row.
+//   a_ik = sum_j v_jk x_ij ; lin_i = sum_j w_j x_ij ; q_i = sum_j sum_k (v_jk x_ij)^2
+//   f_i = w0 + lin_i + 1/2 (sum_k a_ik^2 - q_i)
+// TRAIN: writes A, G and per-CTA fp64 partial sums {sum l_i, sum G_i}; otherwise writes f only.
+// ------------------------------------------------------------------------------------------
+struct RefreshArgs {
+    int64_t n;
+    const int64_t *indptr;
+    const int32_t *idx;
+    const float *val;
+    const float *y;
+    const float *w;
+    const float *V;
+    float *A;
+    float *G;
+    float *f_out;
+    double *partials;  // 2 per CTA
+    float w0;
+    int loss;
+};
+
+template <int LG, int NV, bool TRAIN>
+__global__ void __launch_bounds__(kThreads) refresh_kernel(const RefreshArgs a) {
+    constexpr int G = kThreads / LG;
+    constexpr int KP4 = LG * NV;
+    const int g = threadIdx.x / LG;
+    const int l = threadIdx.x % LG;
+    const uint32_t gm = group_mask<LG>();
+    const float4 *V4 = reinterpret_cast<const float4 *>(a.V);
+    float4 *A4 = reinterpret_cast<float4 *>(a.A);
+    double loss_sum = 0.0, g_sum = 0.0;
+
+    for (int64_t row = (int64_t)blockIdx.x * G + g; row < a.n; row += (int64_t)gridDim.x * G) {
+        const int64_t beg = a.indptr[row], end = a.indptr[row + 1];
+        float4 acc[NV];
+#pragma unroll
+        for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+        float q = 0.f, lin = 0.f;
+        for (int64_t t0 = beg; t0 < end; t0 += LG) {
+            const int64_t mine = t0 + l;
+            int32_t jm = 0;
+            float xm = 0.f;
+            if (mine < end) { jm = __ldg(a.idx + mine); xm = __ldg(a.val + mine); lin = fmaf(__ldg(a.w + jm), xm, lin); }
+            const int cnt = (int)((end - t0) < (int64_t)LG ? (end - t0) : (int64_t)LG);
+            for (int u = 0; u < cnt; ++u) {
+                const int32_t j = __shfl_sync(gm, jm, u, LG);
+                const float x = __shfl_sync(gm, xm, u, LG);
+#pragma unroll
+                for (int v = 0; v < NV; ++v) {
+                    const float4 vv = __ldg(V4 + (size_t)j * KP4 + v * LG + l);
+                    const float px = vv.x * x, py = vv.y * x, pz = vv.z * x, pw = vv.w * x;
+                    acc[v].x += px; acc[v].y += py; acc[v].z += pz; acc[v].w += pw;
+                    q = fmaf(px, px, q); q = fmaf(py, py, q); q = fmaf(pz, pz, q); q = fmaf(pw, pw, q);
+                }
+            }
+        }
+        float sq = 0.f;
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            if (TRAIN) A4[(size_t)row * KP4 + v * LG + l] = acc[v];
+            sq = fmaf(acc[v].x, acc[v].x, sq); sq = fmaf(acc[v].y, acc[v].y, sq);
+            sq = fmaf(acc[v].z, acc[v].z, sq); sq = fmaf(acc[v].w, acc[v].w, sq);
+        }
+        float pair = sq - q;
+#pragma unroll
+        for (int o = LG / 2; o > 0; o >>= 1) {
+            pair += __shfl_xor_sync(gm, pair, o, LG);
+            lin += __shfl_xor_sync(gm, lin, o, LG);
+        }
+        if (l == 0) {
+            const float f = a.w0 + lin + 0.5f * pair;
+            if (TRAIN) {
+                const float yy = a.y[row];
+                float li, gi;
+                if (a.loss == 0) {
+                    gi = f - yy;
+                    li = 0.5f * gi * gi;
+                } else {
+                    const float m = yy * f;
+                    li = fmaxf(-m, 0.f) + log1pf(expf(-fabsf(m)));
+                    gi = -yy / (1.f + expf(m));
+                }
+                a.G[row] = gi;
+                loss_sum += (double)li;
+                g_sum += (double)gi;
+            } else {
+                a.f_out[row] = f;
+            }
+        }
+    }
+    if (TRAIN) {
+        block_sum2(loss_sum, g_sum);
+        if (threadIdx.x == 0) {
+            a.partials[2 * blockIdx.x] = loss_sum;
+            a.partials[2 * blockIdx.x + 1] = g_sum;
+        }
+    }
+}
+
+// per-CTA fp64 partial sums {sum w_j^2, sum v_jk^2}
+__global__ void __launch_bounds__(kThreads) sqnorm_kernel(const float *w, int64_t d, const float *V, int64_t dkp,
+                                                          double *partials) {
+    double sw = 0.0, sv = 0.0;
+    const int64_t stride = (int64_t)gridDim.x * kThreads;
+    for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < d; i += stride) {
+        const double x = (double)w[i];
+        sw += x * x;
+    }
+    const float4 *V4 = reinterpret_cast<const float4 *>(V);
+    for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < dkp / 4; i += stride) {
+        const float4 x = V4[i];
+        sv += (double)x.x * x.x + (double)x.y * x.y + (double)x.z * x.z + (double)x.w * x.w;
+    }
+    block_sum2(sw, sv);
+    if (threadIdx.x == 0) {
+        partials[2 * blockIdx.x] = sw;
+        partials[2 * blockIdx.x + 1] = sv;
+    }
+}
+
+// out[c] = sum over CTAs b (ascending, fixed tree) of partials[2*b + c], c = 0,1
+__global__ void __launch_bounds__(kThreads) reduce2_kernel(const double *partials, int nblocks, double *out) {
+    double s0 = 0.0, s1 = 0.0;
+    for (int b = threadIdx.x; b < nblocks; b += kThreads) {
+        s0 += partials[2 * b];
+        s1 += partials[2 * b + 1];
+    }
+    block_sum2(s0, s1);
+    if (threadIdx.x == 0) { out[0] = s0; out[1] = s1; }
+}
+
+}  // namespace dsf

@@ -67,8 +67,15 @@ def test_init_tiles_and_first_refresh(name):
     g.close()
 
 
+@pytest.fixture(params=["rowblock", "round"])
+def sweep(request, monkeypatch):
+    """Launch order of the strata: one launch per row block (default) or one per inner round."""
+    monkeypatch.setenv("DSFACTO_SWEEP", request.param)
+    return request.param
+
+
 @pytest.mark.parametrize("name,epochs", [("C1", 10), ("C2", 10), ("C3", 5), ("C4s", 2), ("C5s", 2)])
-def test_epochs_match_oracle(name, epochs):
+def test_epochs_match_oracle(name, epochs, sweep):
     wl = W.make(name)
     o, g = make_pair(wl)
     for e in range(epochs):
@@ -102,9 +109,9 @@ def test_sensitive_case_large_step():
 
 
 @pytest.mark.parametrize("K", [1, 3, 4, 5, 7, 12, 20, 33, 64, 100, 128, 129, 200, 256])
-def test_factor_widths(K):
-    wl = W.make("C1")
-    o, g = make_pair(wl, K=K, eta=1.0)
+def test_factor_widths(K, sweep):
+    wl = W.make("C2", n=6000)
+    o, g = make_pair(wl, K=K, eta=1.0, p=3)
     check_aux(o, g)
     before = (o.w0, o.w.copy(), o.V.copy())
     assert g.epoch() == pytest.approx(o.epoch(), rel=1e-4)
@@ -126,7 +133,7 @@ def test_tile_grids_including_empty_blocks(p):
 
 
 def _hot_column_problem(n, d, seed):
-    # column 0 is present in every row, column 1 in every second row: runs far longer than one slab
+    # column 0 is present in every row, column 1 in every second row: runs far longer than one chunk
     rng = np.random.default_rng(seed)
     rows = []
     for i in range(n):
@@ -144,7 +151,7 @@ def _hot_column_problem(n, d, seed):
 
 
 @pytest.mark.parametrize("K,p,loss", [(16, 1, 0), (16, 3, 1), (8, 2, 0), (128, 2, 0), (40, 1, 1)])
-def test_long_runs_cross_slab_and_group_boundaries(K, p, loss):
+def test_long_runs_cross_chunk_warp_and_group_boundaries(K, p, loss, sweep):
     n, d = 9000, 12
     indptr, indices, values, y = _hot_column_problem(n, d, 3)
     if loss:
