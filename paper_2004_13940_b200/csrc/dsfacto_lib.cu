@@ -51,7 +51,8 @@ struct dsfacto {
     int sweep = 1;  // 1: a launch is a row block (p-1 .. 0); 0: a launch is an inner round (0 .. p-1)
     std::vector<int64_t> launch_ptr;
     int2 *d_chunk_map = nullptr;
-    float *d_records = nullptr, *d_Tb = nullptr, *d_Td = nullptr;
+    float *d_records = nullptr, *d_Tb = nullptr, *d_Tw = nullptr;
+    float2 *d_S = nullptr, *d_TS = nullptr;  // scale pairs of the scaled column state (zero outside the SGD phase)
     int *d_tile_count = nullptr;
     int refresh_grid = 0, norm_grid = 0;
 
@@ -161,8 +162,15 @@ void free_data(dsfacto *h) {
 // ---------------------------------------------------------------------------------------------
 template <int LG, int NV>
 void launch_sgd(dsfacto *h, const SgdChunkArgs &a, int grid) {
-    if (h->wide) sgd_chunk_kernel<LG, NV, true><<<grid, kThreads, 0, h->stream>>>(a);
-    else sgd_chunk_kernel<LG, NV, false><<<grid, kThreads, 0, h->stream>>>(a);
+    constexpr int bytes = SgdSmem<LG, NV>::BYTES;
+    static bool opted_in = false;  // more than 48 KB of dynamic shared memory needs an opt-in per kernel
+    if (!opted_in) {
+        cudaFuncSetAttribute(sgd_chunk_kernel<LG, NV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        cudaFuncSetAttribute(sgd_chunk_kernel<LG, NV, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        opted_in = true;
+    }
+    if (h->wide) sgd_chunk_kernel<LG, NV, true><<<grid, kSgdThreads, bytes, h->stream>>>(a);
+    else sgd_chunk_kernel<LG, NV, false><<<grid, kSgdThreads, bytes, h->stream>>>(a);
 }
 template <int LG, int NV>
 void launch_refresh(dsfacto *h, const RefreshArgs &a, bool train, int grid) {
@@ -233,7 +241,7 @@ void run_sgd_phase(dsfacto *h) {
     SgdChunkArgs a{};
     a.tile_ptr = h->d_tile_ptr; a.ent = h->d_ent; a.xw = h->d_xw; a.row_start = h->d_row_start;
     a.col_start = h->d_col_start; a.A = h->d_A; a.G = h->d_G; a.w = h->d_w; a.V = h->d_V;
-    a.Tb = h->d_Tb; a.Td = h->d_Td; a.records = h->d_records; a.tile_count = h->d_tile_count;
+    a.S = h->d_S; a.Tb = h->d_Tb; a.Tw = h->d_Tw; a.TS = h->d_TS; a.records = h->d_records; a.tile_count = h->d_tile_count;
     a.p = h->p; a.jbits = h->jbits; a.sweep = h->sweep;
     a.h = h->h; a.lambda_w = h->lambda_w; a.lambda_v = h->lambda_v;
     for (int L = 0; L < h->p; ++L) {
@@ -243,10 +251,10 @@ void run_sgd_phase(dsfacto *h) {
         DSF_DISPATCH(h, launch_sgd, h, a, (int)grid);
         h->launches += 1;
     }
-    if (h->sweep == 1 && h->p > 1) {
+    {   // back from the scaled state to plain (w, V); folds the tail composites in after a row-block sweep
         const int grid = h->sm_count * 8;
-        sgd_finalize_v_kernel<<<grid, kThreads, 0, h->stream>>>(h->d_V, h->d_Tb, h->d_Td, h->d, h->Kp / 4);
-        sgd_finalize_w_kernel<<<grid, kThreads, 0, h->stream>>>(h->d_w, h->d_Td, h->d);
+        sgd_finalize_v_kernel<<<grid, kThreads, 0, h->stream>>>(h->d_V, h->d_Tb, h->d_S, h->d_TS, h->d, h->Kp / 4);
+        sgd_finalize_w_kernel<<<grid, kThreads, 0, h->stream>>>(h->d_w, h->d_Tw, h->d_S, h->d_TS, h->d);
         h->launches += 2;
     }
 }
@@ -521,10 +529,15 @@ int dsfacto_create(dsfacto_t **out, int64_t n, int32_t d, int32_t K, int32_t p, 
         return fail(DSFACTO_ERR_CUDA);
     h->norm_grid = h->sm_count * 8;
     if (const char *env = std::getenv("DSFACTO_SWEEP")) h->sweep = (std::strcmp(env, "round") == 0) ? 0 : 1;
+    if ((rc = dev_alloc(h, &h->d_S, (size_t)d))) return fail(rc);
+    if (cudaMemset(h->d_S, 0, sizeof(float2) * (size_t)d) != cudaSuccess) return fail(DSFACTO_ERR_CUDA);
     if (h->sweep == 1) {
-        if ((rc = dev_alloc(h, &h->d_Tb, (size_t)d * h->Kp)) || (rc = dev_alloc(h, &h->d_Td, (size_t)d * 4))) return fail(rc);
+        if ((rc = dev_alloc(h, &h->d_Tb, (size_t)d * h->Kp)) || (rc = dev_alloc(h, &h->d_Tw, (size_t)d)) ||
+            (rc = dev_alloc(h, &h->d_TS, (size_t)d)))
+            return fail(rc);
         if (cudaMemset(h->d_Tb, 0, sizeof(float) * (size_t)d * h->Kp) != cudaSuccess ||
-            cudaMemset(h->d_Td, 0, sizeof(float) * (size_t)d * 4) != cudaSuccess)
+            cudaMemset(h->d_Tw, 0, sizeof(float) * (size_t)d) != cudaSuccess ||
+            cudaMemset(h->d_TS, 0, sizeof(float2) * (size_t)d) != cudaSuccess)
             return fail(DSFACTO_ERR_CUDA);
     }
     *out = h;
@@ -535,7 +548,7 @@ void dsfacto_destroy(dsfacto_t *h) {
     if (!h) return;
     cudaStreamSynchronize(h->stream);
     free_data(h);
-    dev_free(h->d_w); dev_free(h->d_V); dev_free(h->d_Tb); dev_free(h->d_Td); dev_free(h->d_row_start); dev_free(h->d_col_start); dev_free(h->d_scal);
+    dev_free(h->d_w); dev_free(h->d_V); dev_free(h->d_Tb); dev_free(h->d_Tw); dev_free(h->d_S); dev_free(h->d_TS); dev_free(h->d_row_start); dev_free(h->d_col_start); dev_free(h->d_scal);
     for (auto &e : h->ev)
         if (e) cudaEventDestroy(e);
     delete h;

@@ -9,19 +9,54 @@
 // (0, 0): the per-entry shrink e is often below half an ulp of 1, and summing it into D keeps it at
 // full relative precision instead of losing it against v_j.  Consecutive pieces combine as
 //     (D2,B2) o (D1,B1) = (D1 + D2 + D1 D2,  B1 + D2 B1 + B2)
-// and a finished run is applied once: v_j += D v_j + B.
+// and a finished run is applied once: v_j <- (1 + D) v_j + B.
+//
+// During the SGD phase the column state is held in scaled form, v_j = (1 + sigma_j) u_j (and the
+// same for w_j), with sigma_j = 0 at the start of the phase.  Applying a run then needs only the
+// 8-byte scale pair of the column:  sigma' = sigma + D + sigma D,  u_j += B / (1 + sigma'),
+// so the K-wide part is an add that nobody waits for (red.global.add; every column receives at
+// most one per launch, so the result does not depend on timing).  sgd_finalize_* turns the state
+// back into plain (w, V) at the end of the phase.  The scaled form breaks down only if some
+// 1 + sigma reaches zero, i.e. a step so large that a run wipes its column; the parameters then
+// become non-finite and the epoch reports divergence.
 #pragma once
 #include "dsfacto_common.cuh"
 
 namespace dsf {
 
-constexpr int kChunk = 1024;       // entries per CTA
-constexpr int kWarpEntries = 128;  // entries per warp
+constexpr int kSgdThreads = 128;  // 4 warps per CTA
+constexpr int kSgdWarps = kSgdThreads / 32;
+constexpr int kWarpEntries = 512;                 // entries per warp
+constexpr int kChunk = kSgdWarps * kWarpEntries;  // entries per CTA
 
-// entries one lane group walks sequentially per pass
-__host__ __device__ constexpr int chunk_seq_len(int LG, int NV) { return LG == 1 ? 4 : (LG == 2 ? 8 : 16 / NV); }
+// entries of one warp pass: sized so that the gathered rows of A fill about 8 KB of shared memory
+__host__ __device__ constexpr int sgd_pass_len(int LG, int NV) {
+    return 512 / (LG * NV) > 256 ? 256 : (512 / (LG * NV) < 8 ? 8 : 512 / (LG * NV));
+}
 // floats per chunk record in global scratch: 3 header float4s + head offsets + tail offsets
 __host__ __device__ constexpr int chunk_record_floats(int Kp) { return 12 + 2 * Kp; }
+
+// shared-memory carve-up of one warp, in float4 units
+template <int LG, int NV>
+struct SgdSmem {
+    static constexpr int GW = 32 / LG;
+    static constexpr int KP4 = LG * NV;
+    static constexpr int PASS = sgd_pass_len(LG, NV);
+    static constexpr int S = PASS / GW;                  // entries a lane group walks per pass
+    static constexpr int ITEM_STRIDE = S + 1;            // +1: lane groups land in different banks
+    static constexpr int ROW_STRIDE = (S + (LG < 8 ? 1 : 0)) * KP4;
+    static constexpr int ITEMS = 0;                      // GW * ITEM_STRIDE   {e, b, row, j_local}
+    static constexpr int ROWS = ITEMS + GW * ITEM_STRIDE;  // GW * ROW_STRIDE  gathered rows a_i
+    static constexpr int SCALES = ROWS + GW * ROW_STRIDE;  // GW * ITEM_STRIDE float2: scale pair of the
+                                                         // column whose run starts at that entry
+    static constexpr int HEAD = SCALES + (GW * ITEM_STRIDE + 1) / 2;  // GW * (KP4+1)  head pieces
+    static constexpr int WARP = HEAD + GW * (KP4 + 1);   // float4s per warp
+    // per CTA, after the warps: per warp head/tail pieces, then the chunk head piece
+    static constexpr int WPIECE = kSgdWarps * WARP;      // kSgdWarps * 2 * (KP4+1)
+    static constexpr int CPIECE = WPIECE + kSgdWarps * 2 * (KP4 + 1);  // (KP4+1)
+    static constexpr int TOTAL = CPIECE + (KP4 + 1);
+    static constexpr int BYTES = TOTAL * 16 + 16 * kSgdWarps;  // + per-warp boundary flags
+};
 
 template <int NV>
 struct Comp {
@@ -85,25 +120,113 @@ __device__ __forceinline__ Comp<NV> comp_shfl(const Comp<NV> &c, int src) {
     return r;
 }
 
+// a composite as stored in shared or global memory: KP4 offset float4s, then {D, Dw, Bw, column}
+template <int LG, int NV>
+__device__ __forceinline__ void comp_store(float4 *dst, const Comp<NV> &c, uint32_t col, int l) {
+#pragma unroll
+    for (int v = 0; v < NV; ++v) dst[v * LG + l] = c.B[v];
+    if (l == 0) dst[LG * NV] = make_float4(c.D, c.Dw, c.Bw, __uint_as_float(col));
+}
+template <int LG, int NV>
+__device__ __forceinline__ uint32_t comp_load(const float4 *src, Comp<NV> &c, int l) {
+#pragma unroll
+    for (int v = 0; v < NV; ++v) c.B[v] = src[v * LG + l];
+    const float4 hd = src[LG * NV];
+    c.D = hd.x; c.Dw = hd.y; c.Bw = hd.z;
+    return __float_as_uint(hd.w);
+}
+
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src) {
+    const unsigned s = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async8(void *smem_dst, const void *gmem_src) {
+    const unsigned s = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;\n" ::"r"(s), "l"(gmem_src) : "memory");
+}
+// fire-and-forget adds into global memory
+__device__ __forceinline__ void red_add4(float4 *p, float x, float y, float z, float w) {
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(x), "f"(y), "f"(z), "f"(w) : "memory");
+}
+__device__ __forceinline__ void red_add1(float *p, float x) {
+    asm volatile("red.global.add.f32 [%0], %1;" ::"l"(p), "f"(x) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() {
+    asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;\n" ::: "memory");
+}
+
+// One step of a segmented scan over the lane groups of a warp (all 32 lanes must call it).
+// Each lane group contributes an element: `hasb` (it holds a run boundary), `head` (composite of
+// what precedes its first boundary) and `cur` (composite after its last boundary, or of the whole
+// element when it has none).  `carry`/`cflag` describe the run left open by earlier steps and are
+// updated to the run left open after this step.  For a group with a boundary, `closing` becomes
+// the composite of the run that ends at its first boundary and `outer` tells whether that run began
+// before the first step (nothing to its left held a boundary).
+template <int LG, int NV>
+__device__ __forceinline__ void scan_step(bool hasb, const Comp<NV> &head, const Comp<NV> &cur, Comp<NV> &carry,
+                                          bool &cflag, Comp<NV> &closing, bool &outer) {
+    constexpr int GW = 32 / LG;
+    const int lane = threadIdx.x & 31;
+    const int g = lane / LG, l = lane % LG;
+    Comp<NV> inc = cur;
+    bool finc = hasb;
+    if (GW > 1) {
+#pragma unroll
+        for (int delta = 1; delta < GW; delta <<= 1) {
+            const Comp<NV> o = comp_shfl_up<NV>(inc, delta * LG);
+            const bool of = __shfl_up_sync(0xFFFFFFFFu, (int)finc, delta * LG) != 0;
+            if (g >= delta) {
+                if (!finc) inc = compose<NV>(o, inc);
+                finc = finc || of;
+            }
+        }
+    }
+    Comp<NV> ex;  // what is open on this group's left, from earlier groups of this step
+    bool fex = false;
+    comp_identity(ex);
+    if (GW > 1) {
+        const Comp<NV> up = comp_shfl_up<NV>(inc, LG);
+        const bool fup = __shfl_up_sync(0xFFFFFFFFu, (int)finc, LG) != 0;
+        if (g > 0) { ex = up; fex = fup; }
+    }
+    outer = false;
+    if (hasb) {
+        closing = compose<NV>(fex ? ex : compose<NV>(carry, ex), head);
+        outer = !(fex || cflag);
+    }
+    const Comp<NV> lastc = comp_shfl<NV>(inc, (GW - 1) * LG + l);
+    const bool lastf = __shfl_sync(0xFFFFFFFFu, (int)finc, (GW - 1) * LG) != 0;
+    carry = lastf ? lastc : compose<NV>(carry, lastc);
+    cflag = cflag || lastf;
+}
+
 // ------------------------------------------------------------------------------------------
-// sgd_chunk_kernel: one CTA per chunk of kChunk consecutive entries of one tile.
+// sgd_chunk_kernel: one CTA (4 warps) per chunk of kChunk consecutive entries of one tile.
 //
 // A launch covers tiles with pairwise disjoint column blocks: the p tiles of one inner round
 // (sweep 0) or the p tiles of one row block (sweep 1).  A tile's entries are sorted by (column,
-// row).  Every warp owns kWarpEntries consecutive entries and walks them in passes; inside a pass
-// each lane group walks S consecutive entries sequentially.  A "boundary" sits before an entry
-// whose column differs from the entry before it (the tile start counts).  A run that lies inside
-// one lane group's piece is applied to the column state at once.  Runs that cross lane groups are
-// joined by a segmented scan over the groups of the warp (shuffles); runs that cross warps by the
-// first lane group of warp 0 (shared memory); runs that cross chunks by whichever chunk of the tile
-// finishes last (records in global scratch plus one counter per tile - no CTA waits for another).
+// row).  Every warp owns kWarpEntries consecutive entries and walks them in passes.  Per pass:
+//   1. one lane per entry turns the (prefetched) entry record and G_i into (e, b, row, column);
+//      a "boundary" sits before an entry whose column differs from the entry before it (the tile
+//      start counts), i.e. at every entry that starts a run;
+//   2. the rows a_i of the whole pass, and the scale pair of every column whose run starts in the
+//      pass, are gathered into shared memory with cp.async: one memory latency per pass;
+//   3. each lane group walks S consecutive entries sequentially.  The piece before its first
+//      boundary becomes its head; a run that starts and ends inside the group is applied on the
+//      spot from the prefetched scale pair (stores and adds nobody waits for);
+//   4. scan_step joins the pieces across the lane groups of the warp; the runs that end at the
+//      groups' first boundaries are applied together.
+// Runs that cross warps are joined by the same scan run by warp 0 over the warps' results (shared
+// memory); runs that cross chunks by the same scan run by whichever chunk of the tile finishes
+// last, over per-chunk records in global scratch (one counter per tile; no CTA waits for another).
 //
-// Column state: in a direct tile it is (w_j, v_j).  In a tail tile (sweep 1, r > c) it is a
-// per-column composite T_j, identity at the start of the epoch and applied to (w_j, v_j) by
-// sgd_finalize_* after the sweep.  The sweep visits row blocks p-1, .., 0, so for column block c
-// the tail tiles (r = p-1 .. c+1) and then the direct tiles (r = c .. 0) are each met in the
-// stratified order of the rounds, and "T_j after v_j" restores the order c, .., 0, p-1, .., c+1.
-// Meanwhile all entries of a row meet in one launch, so (a_i, G_i) come from L2 after first touch.
+// Column state: in a direct tile it is the scaled (w_j, v_j).  In a tail tile (sweep 1, r > c) it
+// is a per-column composite T_j in the same scaled form, identity at the start of the epoch and
+// applied to (w_j, v_j) by sgd_finalize_* after the sweep.  The sweep visits row blocks p-1, .., 0,
+// so for column block c the tail tiles (r = p-1 .. c+1) and then the direct tiles (r = c .. 0) are
+// each met in the stratified order of the rounds, and "T_j after v_j" restores the order
+// c, .., 0, p-1, .., c+1.  Meanwhile all entries of a row meet in one launch, so (a_i, G_i) come
+// from L2 after first touch.
 // ------------------------------------------------------------------------------------------
 struct SgdChunkArgs {
     const int64_t *tile_ptr;   // p*p+1, tile t = s*p + r
@@ -113,10 +236,12 @@ struct SgdChunkArgs {
     const int32_t *col_start;  // p+1
     const float *A;            // n * Kp
     const float *G;            // n
-    float *w;                  // d
-    float *V;                  // d * Kp
-    float *Tb;                 // d * Kp  offset part of T_j            (sweep 1)
-    float *Td;                 // d * 4   {D, Dw, Bw, -} of T_j         (sweep 1)
+    float *w;                  // d        u-part of w_j
+    float *V;                  // d * Kp   u-part of v_j
+    float2 *S;                 // d        {sigma of v_j, sigma of w_j}
+    float *Tw;                 // d        u-part of the w offset of T_j      (sweep 1)
+    float *Tb;                 // d * Kp   u-part of the v offset of T_j      (sweep 1)
+    float2 *TS;                // d        {D, Dw} of T_j                     (sweep 1)
     const int2 *chunk_map;     // per CTA of this launch: {tile t, chunk index inside the tile}
     float *records;            // chunk_record_floats(Kp) floats per CTA of this launch
     int *tile_count;           // p*p, all zero between launches
@@ -125,27 +250,29 @@ struct SgdChunkArgs {
 };
 
 template <int LG, int NV, bool WIDE>
-__global__ void __launch_bounds__(kThreads) sgd_chunk_kernel(const SgdChunkArgs a) {
-    constexpr int S = chunk_seq_len(LG, NV);
-    constexpr int GW = 32 / LG;   // lane groups per warp
-    constexpr int PASS = GW * S;  // entries per warp pass
+__global__ void __launch_bounds__(kSgdThreads, 4) sgd_chunk_kernel(const SgdChunkArgs a) {
+    typedef SgdSmem<LG, NV> L;
+    constexpr int GW = L::GW, KP4 = L::KP4, PASS = L::PASS, S = L::S;
     constexpr int PP = kWarpEntries / PASS;
-    constexpr int KP4 = LG * NV;
-    constexpr int NW = kThreads / 32;
-    constexpr int BATCH = S < 8 ? S : 8;  // rows of A fetched ahead of use
+    constexpr int EPL = (PASS + 31) / 32;  // entries staged per lane and pass
+    constexpr int NW = kSgdWarps;
     constexpr int REC4 = chunk_record_floats(4 * KP4) / 4;
-    static_assert(PP >= 1 && PASS * PP == kWarpEntries, "a warp's entries must be whole passes");
-    static_assert(NW * kWarpEntries == kChunk, "chunk = warps x entries per warp");
+    static_assert(PASS * PP == kWarpEntries && S * GW == PASS, "a warp's entries must be whole passes");
     typedef Comp<NV> C;
 
-    __shared__ float4 s_item[NW][PASS];  // {e, b, row (bits), j_local (bits)}
-    __shared__ float4 s_wB[NW][2][KP4];  // per warp: offsets of its head piece / open tail
-    __shared__ float4 s_wH[NW][2];       // per warp: {D, Dw, Bw, column (bits)} of head / tail
-    __shared__ int s_wflag[NW];          // warp saw a boundary
-    __shared__ int s_last;
-
+    extern __shared__ float4 smem4[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = lane / LG, l = lane % LG;
+    float4 *sw = smem4 + warp * L::WARP;
+    float4 *s_item = sw + L::ITEMS + g * L::ITEM_STRIDE;
+    float4 *s_rows = sw + L::ROWS + g * L::ROW_STRIDE;
+    float2 *s_scale_all = reinterpret_cast<float2 *>(sw + L::SCALES);
+    float2 *s_scale = s_scale_all + g * L::ITEM_STRIDE;
+    float4 *s_head = sw + L::HEAD + g * (KP4 + 1);
+    float4 *s_wpiece = smem4 + L::WPIECE;  // [warp][head/tail][KP4+1]
+    float4 *s_cpiece = smem4 + L::CPIECE;
+    int *s_wflag = reinterpret_cast<int *>(smem4 + L::TOTAL);
+
     const int2 cm = a.chunk_map[blockIdx.x];
     const int64_t t = cm.x;
     const int r = (int)(t % a.p), s = (int)(t / a.p);
@@ -161,46 +288,29 @@ __global__ void __launch_bounds__(kThreads) sgd_chunk_kernel(const SgdChunkArgs 
     const uint32_t jmask = a.jbits >= 32 ? 0xFFFFFFFFu : ((1u << a.jbits) - 1u);
     const float ew = a.h * a.lambda_w;
     const float4 *A4 = reinterpret_cast<const float4 *>(a.A);
-    float4 *V4 = reinterpret_cast<float4 *>(a.V);
-    float4 *Tb4 = reinterpret_cast<float4 *>(a.Tb);
-    float4 *Td4 = reinterpret_cast<float4 *>(a.Td);
+    // the column state this tile acts on (u-parts and scale pairs), shifted to the column block
+    float4 *U4 = reinterpret_cast<float4 *>(tail_mode ? a.Tb : a.V) + (size_t)col0 * KP4;
+    float *uw = (tail_mode ? a.Tw : a.w) + col0;
+    float2 *Sc = (tail_mode ? a.TS : a.S) + col0;
 
-    // applies a finished run to the state of local column jl (the LG lanes of one group)
-    auto apply = [&](uint32_t jl, const C &x) {
-        if (jl == kNoCol) return;
-        const size_t col = (size_t)(col0 + jl);
-        if (!tail_mode) {
+    // column state <- run o column state, given the column's scale pair (lanes of one group)
+    auto apply = [&](uint32_t jl, const C &x, float2 sc) {
+        const float sg = fmaf(sc.x, x.D, sc.x + x.D);
+        const float inv = 1.0f / (1.0f + sg);
 #pragma unroll
-            for (int v = 0; v < NV; ++v) {
-                float4 y = V4[col * KP4 + v * LG + l];
-                y.x += fmaf(x.D, y.x, x.B[v].x);
-                y.y += fmaf(x.D, y.y, x.B[v].y);
-                y.z += fmaf(x.D, y.z, x.B[v].z);
-                y.w += fmaf(x.D, y.w, x.B[v].w);
-                V4[col * KP4 + v * LG + l] = y;
-            }
-            if (l == 0) {
-                const float wj = a.w[col];
-                a.w[col] = wj + fmaf(x.Dw, wj, x.Bw);
-            }
-        } else {
-#pragma unroll
-            for (int v = 0; v < NV; ++v) {
-                float4 y = Tb4[col * KP4 + v * LG + l];
-                y.x = fmaf(x.D, y.x, y.x) + x.B[v].x;
-                y.y = fmaf(x.D, y.y, y.y) + x.B[v].y;
-                y.z = fmaf(x.D, y.z, y.z) + x.B[v].z;
-                y.w = fmaf(x.D, y.w, y.w) + x.B[v].w;
-                Tb4[col * KP4 + v * LG + l] = y;
-            }
-            if (l == 0) {
-                float4 y = Td4[col];
-                y.z = fmaf(x.Dw, y.z, y.z) + x.Bw;
-                y.x = fmaf(y.x, x.D, y.x + x.D);
-                y.y = fmaf(y.y, x.Dw, y.y + x.Dw);
-                Td4[col] = y;
-            }
+        for (int v = 0; v < NV; ++v)
+            red_add4(U4 + (size_t)jl * KP4 + v * LG + l, x.B[v].x * inv, x.B[v].y * inv, x.B[v].z * inv,
+                     x.B[v].w * inv);
+        if (l == 0) {
+            const float sgw = fmaf(sc.y, x.Dw, sc.y + x.Dw);
+            red_add1(uw + jl, x.Bw / (1.0f + sgw));
+            Sc[jl] = make_float2(sg, sgw);
         }
+    };
+    // the same with the scale pair fetched from global memory (an L2 hit after the first launch)
+    auto apply_fetch = [&](uint32_t jl, const C &x) {
+        if (jl == kNoCol) return;
+        apply(jl, x, Sc[jl]);
     };
 
     // ---------------- warp phase ----------------
@@ -209,241 +319,282 @@ __global__ void __launch_bounds__(kThreads) sgd_chunk_kernel(const SgdChunkArgs 
     bool wflag = false;  // a boundary has been seen in this warp
     uint32_t last_col = kNoCol;
 
+    // entry records are fetched two passes ahead and G one pass ahead, into registers
+    uint2 ent0[EPL], ent1[EPL];
+    float xw0[EPL], xw1[EPL], g0[EPL];
+    auto fetch_ent = [&](int pp, uint2 (&e)[EPL], float (&xv)[EPL]) {
+        const int64_t pb = wb + (int64_t)pp * PASS;
+#pragma unroll
+        for (int q = 0; q < EPL; ++q) {
+            const int64_t at = pb + lane + 32 * q;
+            if (lane + 32 * q < PASS && at < we) {
+                e[q] = a.ent[at];
+                if (WIDE) xv[q] = a.xw[at];
+            }
+        }
+    };
+    auto fetch_g = [&](int pp, const uint2 (&e)[EPL], float (&gv)[EPL]) {
+        const int64_t pb = wb + (int64_t)pp * PASS;
+#pragma unroll
+        for (int q = 0; q < EPL; ++q) {
+            const int64_t at = pb + lane + 32 * q;
+            if (lane + 32 * q < PASS && at < we) {
+                const uint32_t il = WIDE ? e[q].x : (e[q].x >> a.jbits);
+                gv[q] = __ldg(a.G + (row0 + il));
+            }
+        }
+    };
+    fetch_ent(0, ent0, xw0);
+    if (PP > 1) fetch_ent(1, ent1, xw1);
+    fetch_g(0, ent0, g0);
+
     for (int pp = 0; pp < PP; ++pp) {
         const int64_t pb = wb + (int64_t)pp * PASS;
         if (pb >= we) break;
         const int cnt = (int)((we - pb) < (int64_t)PASS ? (we - pb) : (int64_t)PASS);
-        // stage: one lane per entry gathers G_i and forms (e, b)
-        for (int q = lane; q < cnt; q += 32) {
-            const uint2 rec = a.ent[pb + q];
-            uint32_t il, jl;
-            float x;
-            if (WIDE) { il = rec.x; jl = rec.y; x = a.xw[pb + q]; }
-            else { il = rec.x >> a.jbits; jl = rec.x & jmask; x = __uint_as_float(rec.y); }
-            const uint32_t row = (uint32_t)(row0 + il);
-            const float gx = __ldg(a.G + row) * x;
-            s_item[warp][q] = make_float4(a.h * (a.lambda_v - gx * x), -a.h * gx, __uint_as_float(row),
-                                          __uint_as_float(jl));
-        }
         uint32_t before = kNoCol;  // column of the entry just before this pass, if it is in the tile
         if (pp > 0) before = last_col;
         else if (pb > tb) {
             const uint2 rec = a.ent[pb - 1];
             before = WIDE ? rec.y : (rec.x & jmask);
         }
+        // 1. items of this pass from the prefetched registers; scale pairs of the columns whose
+        //    runs start here
+        uint32_t carry_col = before;  // column of the entry before this lane's entry of round q
+#pragma unroll
+        for (int q = 0; q < EPL; ++q) {
+            const int at = lane + 32 * q;
+            uint32_t jl = kNoCol;
+            if (at < cnt) {
+                uint32_t il;
+                float x;
+                if (WIDE) { il = ent0[q].x; jl = ent0[q].y; x = xw0[q]; }
+                else { il = ent0[q].x >> a.jbits; jl = ent0[q].x & jmask; x = __uint_as_float(ent0[q].y); }
+                const uint32_t row = (uint32_t)(row0 + il);
+                const float gx = g0[q] * x;
+                sw[L::ITEMS + (at / S) * L::ITEM_STRIDE + (at % S)] =
+                    make_float4(a.h * (a.lambda_v - gx * x), -a.h * gx, __uint_as_float(row), __uint_as_float(jl));
+            }
+            uint32_t prevcol = __shfl_up_sync(0xFFFFFFFFu, jl, 1);
+            if (lane == 0) prevcol = carry_col;
+            carry_col = __shfl_sync(0xFFFFFFFFu, jl, 31);
+            if (at < cnt && jl != prevcol) cp_async8(s_scale_all + (at / S) * L::ITEM_STRIDE + (at % S), Sc + jl);
+        }
+        // rotate the prefetch registers and start the next fetches
+#pragma unroll
+        for (int q = 0; q < EPL; ++q) { ent0[q] = ent1[q]; xw0[q] = xw1[q]; }
+        if (pp + 1 < PP) fetch_g(pp + 1, ent0, g0);
+        if (pp + 2 < PP) fetch_ent(pp + 2, ent1, xw1);
         __syncwarp();
-        last_col = __float_as_uint(s_item[warp][cnt - 1].w);
+        // 2. gather the rows a_i of the pass
+        for (int idx = lane; idx < cnt * KP4; idx += 32) {
+            const int at = idx / KP4, part = idx % KP4;
+            const float4 it = sw[L::ITEMS + (at / S) * L::ITEM_STRIDE + (at % S)];
+            cp_async16(sw + L::ROWS + (at / S) * L::ROW_STRIDE + (at % S) * KP4 + part,
+                       A4 + (size_t)__float_as_uint(it.z) * KP4 + part);
+        }
+        {
+            const int at = cnt - 1;
+            last_col = __float_as_uint(sw[L::ITEMS + (at / S) * L::ITEM_STRIDE + (at % S)].w);
+        }
+        cp_async_wait_all();
+        __syncwarp();
 
+        // 3. sequential walk of each lane group
         const int lo = g * S;
-        const int hi = (lo + S < cnt) ? lo + S : cnt;
+        const int len = (lo >= cnt) ? 0 : ((cnt - lo < S) ? cnt - lo : S);
         bool hasb = false;
         uint32_t headcol = kNoCol;
-        C cur, head;
+        C cur;
         comp_identity(cur);
+        if (len > 0) {
+            uint32_t prevj = (lo == 0) ? before
+                                       : __float_as_uint(sw[L::ITEMS + (g - 1) * L::ITEM_STRIDE + (S - 1)].w);
+            int start = 0;  // entry of this piece at which the current run started
+#pragma unroll 4
+            for (int u = 0; u < len; ++u) {
+                const float4 it = s_item[u];
+                const uint32_t jl = __float_as_uint(it.w);
+                if (jl != prevj) {  // boundary before this entry
+                    if (!hasb) {
+                        comp_store<LG, NV>(s_head, cur, prevj, l);
+                        headcol = prevj;
+                        hasb = true;
+                    } else {
+                        apply(prevj, cur, s_scale[start]);
+                    }
+                    comp_identity(cur);
+                    prevj = jl;
+                    start = u;
+                }
+                const float e = it.x, b = it.y;
+                cur.D = fmaf(-e, cur.D, cur.D - e);
+                cur.Dw = fmaf(-ew, cur.Dw, cur.Dw - ew);
+                cur.Bw = fmaf(-ew, cur.Bw, cur.Bw + b);
+#pragma unroll
+                for (int v = 0; v < NV; ++v) {
+                    const float4 av = s_rows[u * KP4 + v * LG + l];
+                    cur.B[v].x = fmaf(b, av.x, fmaf(-e, cur.B[v].x, cur.B[v].x));
+                    cur.B[v].y = fmaf(b, av.y, fmaf(-e, cur.B[v].y, cur.B[v].y));
+                    cur.B[v].z = fmaf(b, av.z, fmaf(-e, cur.B[v].z, cur.B[v].z));
+                    cur.B[v].w = fmaf(b, av.w, fmaf(-e, cur.B[v].w, cur.B[v].w));
+                }
+            }
+        }
+        // 4. join the pieces across the lane groups
+        C head, closing;
         comp_identity(head);
-        if (lo < hi) {
-            uint32_t prevj = (lo == 0) ? before : __float_as_uint(s_item[warp][lo - 1].w);
-#pragma unroll
-            for (int u0 = 0; u0 < S; u0 += BATCH) {
-                float4 av[BATCH][NV];
-#pragma unroll
-                for (int u = 0; u < BATCH; ++u) {
-                    if (lo + u0 + u < hi) {
-                        const size_t row = __float_as_uint(s_item[warp][lo + u0 + u].z);
-#pragma unroll
-                        for (int v = 0; v < NV; ++v) av[u][v] = __ldg(A4 + row * KP4 + v * LG + l);
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < BATCH; ++u) {
-                    if (lo + u0 + u < hi) {
-                        const float4 it = s_item[warp][lo + u0 + u];
-                        const uint32_t jl = __float_as_uint(it.w);
-                        if (jl != prevj) {  // boundary before this entry
-                            if (!hasb) { head = cur; headcol = prevj; hasb = true; }
-                            else apply(prevj, cur);
-                            comp_identity(cur);
-                            prevj = jl;
-                        }
-                        const float e = it.x, b = it.y;
-                        cur.D = fmaf(-e, cur.D, cur.D - e);
-                        cur.Dw = fmaf(-ew, cur.Dw, cur.Dw - ew);
-                        cur.Bw = fmaf(-ew, cur.Bw, cur.Bw + b);
-#pragma unroll
-                        for (int v = 0; v < NV; ++v) {
-                            cur.B[v].x = fmaf(b, av[u][v].x, fmaf(-e, cur.B[v].x, cur.B[v].x));
-                            cur.B[v].y = fmaf(b, av[u][v].y, fmaf(-e, cur.B[v].y, cur.B[v].y));
-                            cur.B[v].z = fmaf(b, av[u][v].z, fmaf(-e, cur.B[v].z, cur.B[v].z));
-                            cur.B[v].w = fmaf(b, av[u][v].w, fmaf(-e, cur.B[v].w, cur.B[v].w));
-                        }
-                    }
-                }
-            }
+        __syncwarp();
+        if (hasb) comp_load<LG, NV>(s_head, head, l);
+        bool outer;
+        scan_step<LG, NV>(hasb, head, cur, wcarry, wflag, closing, outer);
+        if (hasb) {
+            if (outer) comp_store<LG, NV>(s_wpiece + (warp * 2 + 0) * (KP4 + 1), closing, headcol, l);
+            else apply_fetch(headcol, closing);
         }
-        // ---- segmented inclusive scan over the lane groups of the warp ----
-        // element of a group: (hasb, composite after its last boundary, or of its whole piece)
-        C inc = cur;
-        bool finc = hasb;
-        if (GW > 1) {
-#pragma unroll
-            for (int delta = 1; delta < GW; delta <<= 1) {
-                const C o = comp_shfl_up<NV>(inc, delta * LG);
-                const bool of = __shfl_up_sync(0xFFFFFFFFu, (int)finc, delta * LG) != 0;
-                if (g >= delta) {
-                    if (!finc) inc = compose<NV>(o, inc);
-                    finc = finc || of;
-                }
-            }
-        }
-        C ex;  // what is open on this group's left, from earlier groups of this pass
-        bool fex = false;
-        comp_identity(ex);
-        if (GW > 1) {
-            const C up = comp_shfl_up<NV>(inc, LG);
-            const bool fup = __shfl_up_sync(0xFFFFFFFFu, (int)finc, LG) != 0;
-            if (g > 0) { ex = up; fex = fup; }
-        }
-        if (hasb) {  // this group ends the run that was open on its left
-            C closing = fex ? ex : compose<NV>(wcarry, ex);
-            closing = compose<NV>(closing, head);
-            if (fex || wflag) {
-                apply(headcol, closing);
-            } else {  // the run began before this warp: hand it to the CTA phase
-#pragma unroll
-                for (int v = 0; v < NV; ++v) s_wB[warp][0][v * LG + l] = closing.B[v];
-                if (l == 0) s_wH[warp][0] = make_float4(closing.D, closing.Dw, closing.Bw, __uint_as_float(headcol));
-            }
-        }
-        // open run at the end of the pass = inclusive result of the last group
-        const C lastc = comp_shfl<NV>(inc, (GW - 1) * LG + l);
-        const bool lastf = __shfl_sync(0xFFFFFFFFu, (int)finc, (GW - 1) * LG) != 0;
-        wcarry = lastf ? lastc : compose<NV>(wcarry, lastc);
-        wflag = wflag || lastf;
         __syncwarp();
     }
     if (lane < LG) {
-#pragma unroll
-        for (int v = 0; v < NV; ++v) s_wB[warp][1][v * LG + l] = wcarry.B[v];
-        if (l == 0) {
-            s_wH[warp][1] = make_float4(wcarry.D, wcarry.Dw, wcarry.Bw, __uint_as_float(last_col));
-            s_wflag[warp] = wflag ? 1 : 0;
-        }
+        comp_store<LG, NV>(s_wpiece + (warp * 2 + 1) * (KP4 + 1), wcarry, last_col, l);
+        if (l == 0) s_wflag[warp] = wflag ? 1 : 0;
     }
     __syncthreads();
+    if (warp != 0) return;
 
-    // ---------------- CTA phase: first lane group of warp 0 joins the warps ----------------
+    // ---------------- chunk phase: warp 0 joins the warps ----------------
     const int nchunks = (int)((te - tb + kChunk - 1) / kChunk);
-    if (tid < LG) {
-        bool cta_flag = false;
-        uint32_t cta_headcol = kNoCol, cta_tailcol = kNoCol;
-        C cta_head, run;
-        comp_identity(cta_head);
-        comp_identity(run);
-        for (int w = 0; w < NW; ++w) {
-            C tl;
-            const float4 th = s_wH[w][1];
-            tl.D = th.x; tl.Dw = th.y; tl.Bw = th.z;
-#pragma unroll
-            for (int v = 0; v < NV; ++v) tl.B[v] = s_wB[w][1][v * LG + l];
-            if (!s_wflag[w]) {
-                run = compose<NV>(run, tl);
-            } else {
-                C hd;
-                const float4 hh = s_wH[w][0];
-                hd.D = hh.x; hd.Dw = hh.y; hd.Bw = hh.z;
-#pragma unroll
-                for (int v = 0; v < NV; ++v) hd.B[v] = s_wB[w][0][v * LG + l];
-                const C closing = compose<NV>(run, hd);
-                const uint32_t hc = __float_as_uint(hh.w);
-                if (!cta_flag) { cta_head = closing; cta_headcol = hc; cta_flag = true; }
-                else apply(hc, closing);
-                run = tl;
+    C ccarry;
+    comp_identity(ccarry);
+    bool cflag = false;
+    uint32_t ctailcol = kNoCol;
+    for (int w0 = 0; w0 < NW; w0 += GW) {
+        const int w = w0 + g;
+        bool hasb = false;
+        uint32_t headcol = kNoCol;
+        C head, cur, closing;
+        comp_identity(head);
+        comp_identity(cur);
+        if (w < NW) {
+            comp_load<LG, NV>(s_wpiece + (w * 2 + 1) * (KP4 + 1), cur, l);
+            if (s_wflag[w]) {
+                hasb = true;
+                headcol = comp_load<LG, NV>(s_wpiece + (w * 2 + 0) * (KP4 + 1), head, l);
             }
-            if (__float_as_uint(th.w) != kNoCol) cta_tailcol = __float_as_uint(th.w);
         }
-        if (nchunks == 1) {  // the tile starts and ends here: nothing stays open
-            if (cta_flag) apply(cta_headcol, cta_head);
-            apply(cta_tailcol, run);
-        } else {
-            float4 *rec4 = reinterpret_cast<float4 *>(a.records) + (size_t)blockIdx.x * REC4;
+        bool outer;
+        scan_step<LG, NV>(hasb, head, cur, ccarry, cflag, closing, outer);
+        if (hasb) {
+            if (outer) comp_store<LG, NV>(s_cpiece, closing, headcol, l);
+            else apply_fetch(headcol, closing);
+        }
+    }
+    for (int w = 0; w < NW; ++w) {
+        const uint32_t tc = __float_as_uint(s_wpiece[(w * 2 + 1) * (KP4 + 1) + KP4].w);
+        if (tc != kNoCol) ctailcol = tc;
+    }
+    __syncwarp();
+    if (nchunks == 1) {
+        // the tile starts and ends in this chunk: its head piece belongs to no column, and the end
+        // of the tile closes the run that is still open
+        if (g == 0) apply_fetch(ctailcol, ccarry);
+        return;
+    }
+    {
+        float4 *rec4 = reinterpret_cast<float4 *>(a.records) + (size_t)blockIdx.x * REC4;
+        if (lane < LG) {
             if (l == 0) {
-                rec4[0] = make_float4(cta_head.D, cta_head.Dw, cta_head.Bw, __uint_as_float(cta_headcol));
-                rec4[1] = make_float4(run.D, run.Dw, run.Bw, __uint_as_float(cta_tailcol));
-                rec4[2] = make_float4(__uint_as_float(cta_flag ? 1u : 0u), 0.f, 0.f, 0.f);
+                rec4[0] = cflag ? s_cpiece[KP4] : make_float4(0.f, 0.f, 0.f, __uint_as_float(kNoCol));
+                rec4[1] = make_float4(ccarry.D, ccarry.Dw, ccarry.Bw, __uint_as_float(ctailcol));
+                rec4[2] = make_float4(__uint_as_float(cflag ? 1u : 0u), 0.f, 0.f, 0.f);
             }
 #pragma unroll
             for (int v = 0; v < NV; ++v) {
-                rec4[3 + v * LG + l] = cta_head.B[v];
-                rec4[3 + KP4 + v * LG + l] = run.B[v];
+                rec4[3 + v * LG + l] = cflag ? s_cpiece[v * LG + l] : make_float4(0.f, 0.f, 0.f, 0.f);
+                rec4[3 + KP4 + v * LG + l] = ccarry.B[v];
             }
         }
     }
-    if (nchunks == 1) return;
 
     // ---------------- tile phase: the chunk that finishes last joins the chunks ----------------
     __threadfence();
-    __syncthreads();
-    if (tid == 0) s_last = (atomicAdd(a.tile_count + t, 1) == nchunks - 1) ? 1 : 0;
-    __syncthreads();
-    if (!s_last) return;
+    __syncwarp();
+    int last = 0;
+    if (lane == 0) last = (atomicAdd(a.tile_count + t, 1) == nchunks - 1) ? 1 : 0;
+    last = __shfl_sync(0xFFFFFFFFu, last, 0);
+    if (!last) return;
     __threadfence();
-    if (tid < LG) {
-        const float4 *base4 = reinterpret_cast<const float4 *>(a.records) + ((size_t)blockIdx.x - (size_t)cm.y) * REC4;
-        C run;
-        comp_identity(run);
-        uint32_t tailcol = kNoCol;
-        for (int k = 0; k < nchunks; ++k) {
+    const float4 *base4 = reinterpret_cast<const float4 *>(a.records) + ((size_t)blockIdx.x - (size_t)cm.y) * REC4;
+    C tcarry;
+    comp_identity(tcarry);
+    bool tflag = false;
+    for (int k0 = 0; k0 < nchunks; k0 += GW) {
+        const int k = k0 + g;
+        bool hasb = false;
+        uint32_t headcol = kNoCol;
+        C head, cur, closing;
+        comp_identity(head);
+        comp_identity(cur);
+        if (k < nchunks) {
             const float4 *rec4 = base4 + (size_t)k * REC4;
             const float4 hh = __ldcg(rec4 + 0);
             const float4 th = __ldcg(rec4 + 1);
-            const float4 fl = __ldcg(rec4 + 2);
-            C hd, tl;
-            hd.D = hh.x; hd.Dw = hh.y; hd.Bw = hh.z;
-            tl.D = th.x; tl.Dw = th.y; tl.Bw = th.z;
+            hasb = __float_as_uint(__ldcg(rec4 + 2).x) != 0u;
+            head.D = hh.x; head.Dw = hh.y; head.Bw = hh.z;
+            headcol = __float_as_uint(hh.w);
+            cur.D = th.x; cur.Dw = th.y; cur.Bw = th.z;
 #pragma unroll
             for (int v = 0; v < NV; ++v) {
-                hd.B[v] = __ldcg(rec4 + 3 + v * LG + l);
-                tl.B[v] = __ldcg(rec4 + 3 + KP4 + v * LG + l);
+                head.B[v] = __ldcg(rec4 + 3 + v * LG + l);
+                cur.B[v] = __ldcg(rec4 + 3 + KP4 + v * LG + l);
             }
-            if (__float_as_uint(fl.x) == 0u) {
-                run = compose<NV>(run, tl);
-            } else {
-                apply(__float_as_uint(hh.w), compose<NV>(run, hd));
-                run = tl;
-            }
-            tailcol = __float_as_uint(th.w);
         }
-        apply(tailcol, run);  // the end of the tile closes the last run
-        if (l == 0) a.tile_count[t] = 0;
+        bool outer;
+        scan_step<LG, NV>(hasb, head, cur, tcarry, tflag, closing, outer);
+        // the first boundary of a tile is its start, whose head column is kNoCol: nothing to apply
+        if (hasb) apply_fetch(headcol, closing);
     }
+    const uint32_t ttailcol = __float_as_uint(__ldcg(base4 + (size_t)(nchunks - 1) * REC4 + 1).w);
+    if (g == 0) apply_fetch(ttailcol, tcarry);  // the end of the tile closes the last run
+    if (lane == 0) a.tile_count[t] = 0;
 }
 
-// After a row-block sweep: (w_j, v_j) <- T_j (w_j, v_j), then T_j <- identity.
-__global__ void __launch_bounds__(kThreads) sgd_finalize_v_kernel(float *V, float *Tb, const float *Td, int64_t d,
-                                                                  int kp4) {
+// End of the SGD phase: back from the scaled state to plain parameters,
+//     v_j <- (1 + D_T) ((1 + sigma_j) u_j + ub_j),   w_j likewise,
+// where T_j = (D_T, ub_j) is the tail composite (identity unless the launch order was the row-block
+// sweep), and reset of the scale pairs and of T_j.  Two kernels because the first reads the scale
+// pairs that the second clears.
+__global__ void __launch_bounds__(kThreads) sgd_finalize_v_kernel(float *V, float *Tb, const float2 *S,
+                                                                  const float2 *TS, int64_t d, int kp4) {
     const int64_t total = d * kp4;
     float4 *V4 = reinterpret_cast<float4 *>(V);
     float4 *Tb4 = reinterpret_cast<float4 *>(Tb);
-    const float4 *Td4 = reinterpret_cast<const float4 *>(Td);
     for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < total; i += (int64_t)gridDim.x * kThreads) {
-        const float D = Td4[i / kp4].x;
+        const int64_t j = i / kp4;
+        const float sg = S[j].x;
         float4 y = V4[i];
-        const float4 b = Tb4[i];
-        y.x += fmaf(D, y.x, b.x);
-        y.y += fmaf(D, y.y, b.y);
-        y.z += fmaf(D, y.z, b.z);
-        y.w += fmaf(D, y.w, b.w);
+        y.x = fmaf(sg, y.x, y.x); y.y = fmaf(sg, y.y, y.y); y.z = fmaf(sg, y.z, y.z); y.w = fmaf(sg, y.w, y.w);
+        if (Tb != nullptr) {
+            const float dt = TS[j].x;
+            const float4 b = Tb4[i];
+            y.x += b.x; y.y += b.y; y.z += b.z; y.w += b.w;
+            y.x = fmaf(dt, y.x, y.x); y.y = fmaf(dt, y.y, y.y); y.z = fmaf(dt, y.z, y.z); y.w = fmaf(dt, y.w, y.w);
+            Tb4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
         V4[i] = y;
-        Tb4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
 }
-__global__ void __launch_bounds__(kThreads) sgd_finalize_w_kernel(float *w, float *Td, int64_t d) {
-    float4 *Td4 = reinterpret_cast<float4 *>(Td);
+__global__ void __launch_bounds__(kThreads) sgd_finalize_w_kernel(float *w, float *Tw, float2 *S, float2 *TS, int64_t d) {
     for (int64_t j = (int64_t)blockIdx.x * kThreads + threadIdx.x; j < d; j += (int64_t)gridDim.x * kThreads) {
-        const float4 tj = Td4[j];
-        const float wj = w[j];
-        w[j] = wj + fmaf(tj.y, wj, tj.z);
-        Td4[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+        float wj = w[j];
+        wj = fmaf(S[j].y, wj, wj);
+        S[j] = make_float2(0.f, 0.f);
+        if (Tw != nullptr) {
+            wj += Tw[j];
+            wj = fmaf(TS[j].y, wj, wj);
+            Tw[j] = 0.f;
+            TS[j] = make_float2(0.f, 0.f);
+        }
+        w[j] = wj;
     }
 }
 
