@@ -136,6 +136,36 @@ const char *dsfacto_last_error(dsfacto_t *h);
 
 const char *dsfacto_strerror(int status);
 
+/* ---- for callers that cannot allocate ---- */
+
+/* Scores, loss sum and multiplier sum of m rows, without any allocation.  (The paper has no
+ * counterpart: this is a service entry point.)  It is meant for code that runs where cudaMalloc is
+ * off limits - a process whose device memory is wholly owned by another pool, a serving loop with
+ * a fixed memory budget, a thread that must not take the driver's allocation lock - and that
+ * therefore keeps the rows, the parameters and the result buffers in device memory of its own.
+ *
+ * ALL pointers are DEVICE memory on the current device, owned by the caller, and no handle is
+ * involved:
+ *   indptr_dev int64[m+1], indices_dev int32[nnz], values_dev fp32[nnz]  rows as CSR (same rules
+ *       as dsfacto_load_csr; they are NOT checked here, the caller vouches for them)
+ *   y_dev fp32[m] labels; w0, w_dev fp32[d], V_dev fp32[d*K] row-major, 16-byte aligned parameters
+ *   scores_dev fp32[m]  out: f(x_i), eq. (fm_model2)
+ *   sums_dev fp64[2]    out: { sum_i l(f(x_i), y_i), sum_i G_i }
+ *   cuda_stream         cudaStream_t as void* (NULL = legacy default stream)
+ * Limits: K must be 4, 8, 16, 32, 64, 128 or 256 (rows of V are read as whole 16-byte lane groups);
+ * 1 <= m <= 67,108,864 rows, because the per-CTA partial sums of the reduction live in a fixed
+ * 1 MiB array inside the library image (every GPU that loads the library holds it until the
+ * process exits).  Anything outside these limits returns DSFACTO_ERR_INVALID_ARG.
+ * The first call on each device looks up that array's device address; make this first call
+ * outside any stream capture.  All calls on a device share the array: it keeps the last call's
+ * contents, every call overwrites the slots it uses before reading them (nothing needs clearing),
+ * and two calls that overlap on the GPU (different streams or threads) race on it - serialise them.
+ * The call performs no cudaMalloc/cudaFree and returns after its work on the stream has finished. */
+int dsfacto_score_loss_noalloc(int64_t m, int32_t d, int32_t K, int32_t loss, const int64_t *indptr_dev,
+                               const int32_t *indices_dev, const float *values_dev, const float *y_dev,
+                               float w0, const float *w_dev, const float *V_dev, float *scores_dev,
+                               double *sums_dev, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

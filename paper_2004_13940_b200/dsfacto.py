@@ -37,6 +37,8 @@ SIGNATURES = {
     "dsfacto_launch_count": (ctypes.c_int, [_vp, ctypes.POINTER(_c_i64)]),
     "dsfacto_last_error": (ctypes.c_char_p, [_vp]),
     "dsfacto_strerror": (ctypes.c_char_p, [ctypes.c_int]),
+    "dsfacto_score_loss_noalloc": (ctypes.c_int, [_c_i64, _c_i32, _c_i32, _c_i32, _vp, _vp, _vp, _vp, _c_f32, _vp, _vp,
+                                                  _vp, _vp, _vp]),
 }
 
 _lib = None
@@ -112,6 +114,14 @@ def dsfacto_bucket_host(n, d, p, indptr, indices, values):
     rc = lib().dsfacto_bucket_host(n, d, p, _ptr(indptr), _ptr(indices), _ptr(values), _ptr(tile_ptr), _ptr(rows),
                                    _ptr(cols), _ptr(vals))
     return rc, tile_ptr, rows, cols, vals
+
+
+def dsfacto_score_loss_noalloc(m, d, K, loss, indptr_dev, indices_dev, values_dev, y_dev, w0, w_dev, V_dev,
+                               scores_dev, sums_dev, cuda_stream=0):
+    """Allocation-free scoring; every *_dev argument is a raw device address (int)."""
+    vp = lambda a: ctypes.c_void_p(int(a))
+    return lib().dsfacto_score_loss_noalloc(m, d, K, loss, vp(indptr_dev), vp(indices_dev), vp(values_dev), vp(y_dev),
+                                            w0, vp(w_dev), vp(V_dev), vp(scores_dev), vp(sums_dev), vp(cuda_stream))
 
 
 class DSFacto:
