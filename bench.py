@@ -31,6 +31,9 @@ sys.path.insert(0, str(ROOT))
 METRIC = "nonzero-updates/sec"
 UNIT = "updates/s"
 ORACLE_SAMPLE_ROWS = 1_000_000
+# dram__bytes_read.sum + dram__bytes_write.sum of sgd_chunk_kernel per stored entry, from the ncu capture
+# summarised in profiles/ (None once the kernel has changed since the counters were taken)
+SGD_DRAM_BYTES_PER_ENTRY = None
 
 
 def peaks():
@@ -248,19 +251,24 @@ def run_ours(args):
     phase /= args.steps
     peak, peak_kind = peaks()
     K, n, d, p = wl.K, wl.n, wl.d, wl.p
-    # stratum SGD, per epoch: every entry reads its 8-byte record, G_i and the K-wide row a_i (no reuse
-    # inside a round: the p tiles of a round own disjoint row blocks), plus w, V read+written once
-    sgd_bytes = nnz * (8 + 4 * K + 4) + 8 * d * (K + 1)
+    # Stratum SGD, algorithmic bytes per epoch.  Row-block sweep (default): every array once - the 8-byte
+    # entry records, A and G once (all entries of a row meet in one launch), w and V read + written.
+    # Round sweep: the p tiles of a round own disjoint row blocks, so every entry re-reads G_i and a_i.
+    sweep = os.environ.get("DSFACTO_SWEEP", "rowblock")
+    sgd_gather = nnz * (8 + 4 * K + 4) + 8 * d * (K + 1)
     sgd_floor = 8 * nnz + 4 * n * (K + 1) + 8 * d * (K + 1)
+    sgd_bytes = sgd_gather if sweep == "round" else sgd_floor
     ref_bytes = 8 * nnz + 8 * (n + 1) + 4 * d * (K + 2) + 4 * n * K + 8 * n
     sgd_s, ref_s = phase[1] * 1e-3, phase[2] * 1e-3
-    roof = {"bound": "hbm", "kernel": "sgd_chunk_kernel", "launches_per_step": p,
+    traffic = None if SGD_DRAM_BYTES_PER_ENTRY is None else SGD_DRAM_BYTES_PER_ENTRY * nnz / p
+    roof = {"bound": "hbm", "kernel": "sgd_chunk_kernel", "launches_per_step": p, "sweep": sweep,
             "achieved": sgd_bytes / sgd_s / 1e9, "peak": peak, "unit": "GB/s", "frac": sgd_bytes / sgd_s / 1e9 / peak,
-            "peak_kind": "of " + peak_kind, "traffic": None,
-            "algorithmic_bytes_per_step": sgd_bytes, "avg_launch_us": 1e6 * sgd_s / p,
-            "model": "gather: nnz*(8+4K+4) + 8d(K+1)",
-            "stream_floor": {"bytes_per_step": sgd_floor, "achieved": sgd_floor / sgd_s / 1e9,
-                             "frac": sgd_floor / sgd_s / 1e9 / peak},
+            "peak_kind": "of " + peak_kind, "traffic": traffic,
+            "algorithmic_bytes_per_launch": sgd_bytes / p, "avg_launch_us": 1e6 * sgd_s / p,
+            "model": ("gather: nnz*(8+4K+4) + 8d(K+1)" if sweep == "round" else "stream floor: 8nnz + 4n(K+1) + 8d(K+1)")
+                     + ", per launch = 1/p of it",
+            "gather_model": {"bytes_per_step": sgd_gather, "achieved": sgd_gather / sgd_s / 1e9,
+                             "frac": sgd_gather / sgd_s / 1e9 / peak},
             "refresh_kernel": {"algorithmic_bytes_per_step": ref_bytes, "ms": phase[2],
                                "achieved": ref_bytes / ref_s / 1e9, "frac": ref_bytes / ref_s / 1e9 / peak}}
     value = world * nnz * args.steps / (ms * 1e-3)
