@@ -1,0 +1,96 @@
+"""Parity at the size bench.py times: C4 in full (45 M rows, 1.755 G stored entries, p = 512, K = 16),
+same launch configuration as the bench.
+
+The oracle cannot run a whole epoch at this size in seconds, so the comparison is on outputs it can
+compute one by one, each from the data and the seeded initial parameters alone (nothing the CUDA
+path produced is fed to it):
+  * the first recompute pass: every G_i, every a_i, mean loss, sum of G and the objective, from the
+    oracle's refresh routine over the full CSR;
+  * after one epoch: w0, and (w_j, v_j) of sampled columns - the hottest column (about 9 M entries,
+    present in every tile of its column block), mid-frequency and rare ones, the first and the last
+    id - from the oracle's one-column epoch, which visits that column's rows in the stratified
+    order (pinned against the full oracle epoch on small cases in tests/test_oracle_sgd.py).
+Tolerances are those of tests/test_gpu_parity.py."""
+import ctypes
+
+import numpy as np
+import pytest
+
+from oracle import dsfacto_oracle as O
+from paper_2004_13940_b200 import dsfacto as D
+from paper_2004_13940_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+def _enough_memory():
+    try:
+        import psutil
+        return psutil.virtual_memory().available > 110 * 2 ** 30
+    except Exception:
+        return False
+
+
+@pytest.mark.skipif(not _enough_memory(), reason="needs about 110 GB of host memory")
+def test_c4_full_size_first_refresh_and_sampled_columns():
+    wl = W.make("C4")
+    n, d, K, p = wl.n, wl.d, wl.K, wl.p
+    eta_s = wl.eta / n
+
+    # ---- oracle side, epoch 0: refresh over the full CSR from the seeded initial parameters ----
+    w0, w, V = O.init_params(d, K, wl.init_seed)
+    A = np.empty((n, K), np.float64)
+    lin, q, f, lossv, G = (np.empty(n, np.float64) for _ in range(5))
+    out3 = np.zeros(3, np.float64)
+    P = lambda a: ctypes.c_void_p(a.ctypes.data)
+    O.lib().oracle_refresh(ctypes.c_int64(n), ctypes.c_int32(d), ctypes.c_int32(K), ctypes.c_int32(wl.loss),
+                           ctypes.c_double(wl.lambda_w), ctypes.c_double(wl.lambda_v), P(wl.indptr), P(wl.indices),
+                           P(wl.values), P(wl.y), ctypes.c_double(w0), P(w), P(V), P(A), P(lin), P(q), P(f),
+                           P(lossv), P(G), P(out3))
+    del lin, q, f, lossv
+
+    g = D.DSFacto(n, d, K, p, wl.loss, wl.lambda_w, wl.lambda_v, wl.eta, wl.init_seed)
+    g.load_csr(wl.indptr, wl.indices, wl.values, wl.y)
+    mean_loss, sum_g = g.stats()
+    assert mean_loss == pytest.approx(out3[1], rel=1e-5)
+    assert sum_g == pytest.approx(out3[0], rel=1e-4, abs=1e-3 + 1e-6 * np.abs(G).sum())
+    assert g.objective() == pytest.approx(out3[2], rel=1e-5)
+    A_gpu, G_gpu = g.get_aux()
+    assert np.abs(G_gpu - G).max() <= 2e-5 * (1 + np.abs(G).max())
+    tolA = 2e-5 * (1 + np.abs(A).max())
+    for lo in range(0, n, 5_000_000):                       # blockwise to bound temporaries
+        assert np.abs(A_gpu[lo:lo + 5_000_000] - A[lo:lo + 5_000_000]).max() <= tolA
+    del A, A_gpu, G_gpu
+    # tile sizes: every stored entry in exactly one tile, and the Latin-square row/column sums
+    tile_ptr = np.empty(p * p + 1, np.int64)
+    assert D.lib().dsfacto_get_tiles(g._h, P(tile_ptr), None, None, None) == D.OK
+    assert tile_ptr[0] == 0 and tile_ptr[-1] == wl.nnz and np.all(np.diff(tile_ptr) >= 0)
+    sizes = np.diff(tile_ptr).reshape(p, p)                 # [round s, row block r]
+    rows_per_block = np.diff((np.arange(p + 1) * n + p - 1) // p)
+    assert np.array_equal(sizes.sum(0), rows_per_block * 39)
+
+    # ---- one epoch ----
+    obj0 = g.objective()
+    obj1 = g.epoch()
+    assert np.isfinite(obj1) and obj1 < obj0
+    w0_gpu, w_gpu, V_gpu = g.get_params()
+    g.close()
+    assert w0_gpu == pytest.approx(w0 - eta_s * out3[0], rel=1e-5, abs=1e-7)
+
+    counts = np.bincount(wl.indices[: 39 * 2_000_000], minlength=d)   # popularity from the first 2 M rows
+    order = np.argsort(-counts)
+    present = order[counts[order] > 0]
+    sample = [int(present[0]), int(present[40]), int(present[2000]), int(present[len(present) // 2]),
+              int(present[-1]), 0, d - 23]
+    dw_max = dv_max = 0.0
+    for j in sample:
+        wj, vj, cnt = O.column_epoch(n, d, K, p, wl.loss, eta_s, wl.lambda_w, wl.lambda_v, wl.indptr, wl.indices,
+                                     wl.values, wl.y, w0, w, V, j)
+        assert abs(w_gpu[j] - wj) <= 1e-4 * (1 + abs(wj)), (j, cnt)
+        assert np.all(np.abs(V_gpu[j] - vj) <= 1e-4 * (1 + np.abs(vj))), (j, cnt)
+        # the change itself, which is what one epoch computes
+        dw, dv = wj - w[j], vj - V[j]
+        assert abs((w_gpu[j] - w[j]) - dw) <= 2e-3 * abs(dw) + 2e-7, (j, cnt)
+        assert np.abs((V_gpu[j].astype(np.float64) - V[j]) - dv).max() <= 2e-3 * np.abs(dv).max() + 2e-7, (j, cnt)
+        dw_max, dv_max = max(dw_max, abs(dw)), max(dv_max, np.abs(dv).max())
+    assert dw_max > 1e-4 and dv_max > 1e-5                  # the sampled columns did move
