@@ -49,8 +49,7 @@ struct SgdSmem {
     static constexpr int ROWS = ITEMS + GW * ITEM_STRIDE;  // GW * ROW_STRIDE  gathered rows a_i
     static constexpr int SCALES = ROWS + GW * ROW_STRIDE;  // GW * ITEM_STRIDE float2: scale pair of the
                                                          // column whose run starts at that entry
-    static constexpr int HEAD = SCALES + (GW * ITEM_STRIDE + 1) / 2;  // GW * (KP4+1)  head pieces
-    static constexpr int WARP = HEAD + GW * (KP4 + 1);   // float4s per warp
+    static constexpr int WARP = SCALES + (GW * ITEM_STRIDE + 1) / 2;  // float4s per warp
     // per CTA, after the warps: per warp head/tail pieces, then the chunk head piece
     static constexpr int WPIECE = kSgdWarps * WARP;      // kSgdWarps * 2 * (KP4+1)
     static constexpr int CPIECE = WPIECE + kSgdWarps * 2 * (KP4 + 1);  // (KP4+1)
@@ -268,7 +267,6 @@ __global__ void __launch_bounds__(kSgdThreads, 4) sgd_chunk_kernel(const SgdChun
     float4 *s_rows = sw + L::ROWS + g * L::ROW_STRIDE;
     float2 *s_scale_all = reinterpret_cast<float2 *>(sw + L::SCALES);
     float2 *s_scale = s_scale_all + g * L::ITEM_STRIDE;
-    float4 *s_head = sw + L::HEAD + g * (KP4 + 1);
     float4 *s_wpiece = smem4 + L::WPIECE;  // [warp][head/tail][KP4+1]
     float4 *s_cpiece = smem4 + L::CPIECE;
     int *s_wflag = reinterpret_cast<int *>(smem4 + L::TOTAL);
@@ -287,7 +285,12 @@ __global__ void __launch_bounds__(kSgdThreads, 4) sgd_chunk_kernel(const SgdChun
     const int64_t col0 = a.col_start[c];
     const uint32_t jmask = a.jbits >= 32 ? 0xFFFFFFFFu : ((1u << a.jbits) - 1u);
     const float ew = a.h * a.lambda_w;
-    const float4 *A4 = reinterpret_cast<const float4 *>(a.A);
+    // everything a warp touches is addressed with 32-bit offsets from pointers set up once
+    const float4 *A4 = reinterpret_cast<const float4 *>(a.A) + (size_t)row0 * KP4;  // rows of this row block
+    const float *Gr = a.G + row0;
+    const uint2 *entw = a.ent + wb;                      // this warp's entries
+    const float *xww = WIDE ? a.xw + wb : nullptr;
+    const int wlen = we > wb ? (int)(we - wb) : 0;
     // the column state this tile acts on (u-parts and scale pairs), shifted to the column block
     float4 *U4 = reinterpret_cast<float4 *>(tail_mode ? a.Tb : a.V) + (size_t)col0 * KP4;
     float *uw = (tail_mode ? a.Tw : a.w) + col0;
@@ -296,14 +299,14 @@ __global__ void __launch_bounds__(kSgdThreads, 4) sgd_chunk_kernel(const SgdChun
     // column state <- run o column state, given the column's scale pair (lanes of one group)
     auto apply = [&](uint32_t jl, const C &x, float2 sc) {
         const float sg = fmaf(sc.x, x.D, sc.x + x.D);
-        const float inv = 1.0f / (1.0f + sg);
+        const float inv = __frcp_rn(1.0f + sg);
 #pragma unroll
         for (int v = 0; v < NV; ++v)
             red_add4(U4 + (size_t)jl * KP4 + v * LG + l, x.B[v].x * inv, x.B[v].y * inv, x.B[v].z * inv,
                      x.B[v].w * inv);
         if (l == 0) {
             const float sgw = fmaf(sc.y, x.Dw, sc.y + x.Dw);
-            red_add1(uw + jl, x.Bw / (1.0f + sgw));
+            red_add1(uw + jl, x.Bw * __frcp_rn(1.0f + sgw));
             Sc[jl] = make_float2(sg, sgw);
         }
     };
@@ -323,25 +326,20 @@ __global__ void __launch_bounds__(kSgdThreads, 4) sgd_chunk_kernel(const SgdChun
     uint2 ent0[EPL], ent1[EPL];
     float xw0[EPL], xw1[EPL], g0[EPL];
     auto fetch_ent = [&](int pp, uint2 (&e)[EPL], float (&xv)[EPL]) {
-        const int64_t pb = wb + (int64_t)pp * PASS;
 #pragma unroll
         for (int q = 0; q < EPL; ++q) {
-            const int64_t at = pb + lane + 32 * q;
-            if (lane + 32 * q < PASS && at < we) {
-                e[q] = a.ent[at];
-                if (WIDE) xv[q] = a.xw[at];
+            const int at = pp * PASS + lane + 32 * q;
+            if ((PASS >= 32 || lane < PASS) && at < wlen) {
+                e[q] = entw[at];
+                if (WIDE) xv[q] = xww[at];
             }
         }
     };
     auto fetch_g = [&](int pp, const uint2 (&e)[EPL], float (&gv)[EPL]) {
-        const int64_t pb = wb + (int64_t)pp * PASS;
 #pragma unroll
         for (int q = 0; q < EPL; ++q) {
-            const int64_t at = pb + lane + 32 * q;
-            if (lane + 32 * q < PASS && at < we) {
-                const uint32_t il = WIDE ? e[q].x : (e[q].x >> a.jbits);
-                gv[q] = __ldg(a.G + (row0 + il));
-            }
+            const int at = pp * PASS + lane + 32 * q;
+            if ((PASS >= 32 || lane < PASS) && at < wlen) gv[q] = __ldg(Gr + (WIDE ? e[q].x : (e[q].x >> a.jbits)));
         }
     };
     fetch_ent(0, ent0, xw0);
@@ -349,49 +347,63 @@ __global__ void __launch_bounds__(kSgdThreads, 4) sgd_chunk_kernel(const SgdChun
     fetch_g(0, ent0, g0);
 
     for (int pp = 0; pp < PP; ++pp) {
-        const int64_t pb = wb + (int64_t)pp * PASS;
-        if (pb >= we) break;
-        const int cnt = (int)((we - pb) < (int64_t)PASS ? (we - pb) : (int64_t)PASS);
+        if (pp * PASS >= wlen) break;
+        const int cnt = (wlen - pp * PASS) < PASS ? (wlen - pp * PASS) : PASS;
         uint32_t before = kNoCol;  // column of the entry just before this pass, if it is in the tile
         if (pp > 0) before = last_col;
-        else if (pb > tb) {
-            const uint2 rec = a.ent[pb - 1];
+        else if (wb > tb) {
+            const uint2 rec = entw[-1];
             before = WIDE ? rec.y : (rec.x & jmask);
         }
-        // 1. items of this pass from the prefetched registers; scale pairs of the columns whose
-        //    runs start here
-        uint32_t carry_col = before;  // column of the entry before this lane's entry of round q
+        // column of the entry just after this pass when it is known to this warp (its own next
+        // pass); otherwise the last run of the pass is left open and closed by a later phase
+        uint32_t after = kNoCol;
+        const bool after_known = (pp + 1 < PP) && ((pp + 1) * PASS < wlen);
+        // 1. items of this pass from the prefetched registers
+        uint32_t jq[EPL];
 #pragma unroll
         for (int q = 0; q < EPL; ++q) {
             const int at = lane + 32 * q;
-            uint32_t jl = kNoCol;
+            jq[q] = kNoCol;
             if (at < cnt) {
                 uint32_t il;
                 float x;
-                if (WIDE) { il = ent0[q].x; jl = ent0[q].y; x = xw0[q]; }
-                else { il = ent0[q].x >> a.jbits; jl = ent0[q].x & jmask; x = __uint_as_float(ent0[q].y); }
-                const uint32_t row = (uint32_t)(row0 + il);
+                if (WIDE) { il = ent0[q].x; jq[q] = ent0[q].y; x = xw0[q]; }
+                else { il = ent0[q].x >> a.jbits; jq[q] = ent0[q].x & jmask; x = __uint_as_float(ent0[q].y); }
                 const float gx = g0[q] * x;
                 sw[L::ITEMS + (at / S) * L::ITEM_STRIDE + (at % S)] =
-                    make_float4(a.h * (a.lambda_v - gx * x), -a.h * gx, __uint_as_float(row), __uint_as_float(jl));
+                    make_float4(a.h * (a.lambda_v - gx * x), -a.h * gx, __uint_as_float(il), __uint_as_float(jq[q]));
             }
-            uint32_t prevcol = __shfl_up_sync(0xFFFFFFFFu, jl, 1);
-            if (lane == 0) prevcol = carry_col;
-            carry_col = __shfl_sync(0xFFFFFFFFu, jl, 31);
-            if (at < cnt && jl != prevcol) cp_async8(s_scale_all + (at / S) * L::ITEM_STRIDE + (at % S), Sc + jl);
         }
         // rotate the prefetch registers and start the next fetches
 #pragma unroll
         for (int q = 0; q < EPL; ++q) { ent0[q] = ent1[q]; xw0[q] = xw1[q]; }
+        if (after_known) after = __shfl_sync(0xFFFFFFFFu, WIDE ? ent0[0].y : (ent0[0].x & jmask), 0);
         if (pp + 1 < PP) fetch_g(pp + 1, ent0, g0);
         if (pp + 2 < PP) fetch_ent(pp + 2, ent1, xw1);
+        //    scale pairs of the columns whose runs end in this pass (an entry ends a run when the
+        //    next entry has another column)
+#pragma unroll
+        for (int q = 0; q < EPL; ++q) {
+            const int at = lane + 32 * q;
+            uint32_t nextcol = __shfl_down_sync(0xFFFFFFFFu, jq[q], 1);
+            const uint32_t wrap = __shfl_sync(0xFFFFFFFFu, q + 1 < EPL ? jq[q + 1 < EPL ? q + 1 : q] : kNoCol, 0);
+            if (lane == 31) nextcol = wrap;
+            bool ends;
+            if (at + 1 < cnt) ends = nextcol != jq[q];
+            else ends = after_known && after != jq[q];
+            if (at < cnt && ends) cp_async8(s_scale_all + (at / S) * L::ITEM_STRIDE + (at % S), Sc + jq[q]);
+        }
         __syncwarp();
         // 2. gather the rows a_i of the pass
-        for (int idx = lane; idx < cnt * KP4; idx += 32) {
+#pragma unroll
+        for (int it = 0; it < PASS * KP4 / 32; ++it) {
+            const int idx = lane + 32 * it;
             const int at = idx / KP4, part = idx % KP4;
-            const float4 it = sw[L::ITEMS + (at / S) * L::ITEM_STRIDE + (at % S)];
-            cp_async16(sw + L::ROWS + (at / S) * L::ROW_STRIDE + (at % S) * KP4 + part,
-                       A4 + (size_t)__float_as_uint(it.z) * KP4 + part);
+            if (at < cnt) {
+                const uint32_t il = __float_as_uint(sw[L::ITEMS + (at / S) * L::ITEM_STRIDE + (at % S)].z);
+                cp_async16(sw + L::ROWS + (at / S) * L::ROW_STRIDE + (at % S) * KP4 + part, A4 + (size_t)il * KP4 + part);
+            }
         }
         {
             const int at = cnt - 1;
@@ -400,44 +412,50 @@ __global__ void __launch_bounds__(kSgdThreads, 4) sgd_chunk_kernel(const SgdChun
         cp_async_wait_all();
         __syncwarp();
 
-        // 3. sequential walk of each lane group
+        // 3. sequential walk of each lane group.  A run that ends before entry u is parked in the
+        //    slots of entry u-1, which have been consumed: offsets over its row, {D, Dw, Bw} over
+        //    its item.  The first such run of the group is its head piece; the others started inside
+        //    the group and are marked in `emask` for step 5.
         const int lo = g * S;
         const int len = (lo >= cnt) ? 0 : ((cnt - lo < S) ? cnt - lo : S);
         bool hasb = false;
-        uint32_t headcol = kNoCol;
+        int head_pos = -1;
+        uint32_t headcol = kNoCol, emask = 0;
         C cur;
         comp_identity(cur);
         if (len > 0) {
             uint32_t prevj = (lo == 0) ? before
                                        : __float_as_uint(sw[L::ITEMS + (g - 1) * L::ITEM_STRIDE + (S - 1)].w);
-            int start = 0;  // entry of this piece at which the current run started
-#pragma unroll 4
-            for (int u = 0; u < len; ++u) {
-                const float4 it = s_item[u];
-                const uint32_t jl = __float_as_uint(it.w);
-                if (jl != prevj) {  // boundary before this entry
-                    if (!hasb) {
-                        comp_store<LG, NV>(s_head, cur, prevj, l);
-                        headcol = prevj;
-                        hasb = true;
-                    } else {
-                        apply(prevj, cur, s_scale[start]);
-                    }
-                    comp_identity(cur);
-                    prevj = jl;
-                    start = u;
-                }
-                const float e = it.x, b = it.y;
-                cur.D = fmaf(-e, cur.D, cur.D - e);
-                cur.Dw = fmaf(-ew, cur.Dw, cur.Dw - ew);
-                cur.Bw = fmaf(-ew, cur.Bw, cur.Bw + b);
 #pragma unroll
-                for (int v = 0; v < NV; ++v) {
-                    const float4 av = s_rows[u * KP4 + v * LG + l];
-                    cur.B[v].x = fmaf(b, av.x, fmaf(-e, cur.B[v].x, cur.B[v].x));
-                    cur.B[v].y = fmaf(b, av.y, fmaf(-e, cur.B[v].y, cur.B[v].y));
-                    cur.B[v].z = fmaf(b, av.z, fmaf(-e, cur.B[v].z, cur.B[v].z));
-                    cur.B[v].w = fmaf(b, av.w, fmaf(-e, cur.B[v].w, cur.B[v].w));
+            for (int u = 0; u < S; ++u) {
+                if (u < len) {
+                    const float4 it = s_item[u];
+                    float4 av[NV];
+#pragma unroll
+                    for (int v = 0; v < NV; ++v) av[v] = s_rows[u * KP4 + v * LG + l];
+                    const uint32_t jl = __float_as_uint(it.w);
+                    if (jl != prevj) {  // boundary before this entry
+                        if (u > 0) {
+#pragma unroll
+                            for (int v = 0; v < NV; ++v) s_rows[(u - 1) * KP4 + v * LG + l] = cur.B[v];
+                            if (l == 0) s_item[u - 1] = make_float4(cur.D, cur.Dw, cur.Bw, __uint_as_float(prevj));
+                        }
+                        if (!hasb) { hasb = true; headcol = prevj; head_pos = u - 1; }
+                        else emask |= 1u << (u - 1);
+                        comp_identity(cur);
+                        prevj = jl;
+                    }
+                    const float e = it.x, b = it.y;
+                    cur.D = fmaf(-e, cur.D, cur.D - e);
+                    cur.Dw = fmaf(-ew, cur.Dw, cur.Dw - ew);
+                    cur.Bw = fmaf(-ew, cur.Bw, cur.Bw + b);
+#pragma unroll
+                    for (int v = 0; v < NV; ++v) {
+                        cur.B[v].x = fmaf(b, av[v].x, fmaf(-e, cur.B[v].x, cur.B[v].x));
+                        cur.B[v].y = fmaf(b, av[v].y, fmaf(-e, cur.B[v].y, cur.B[v].y));
+                        cur.B[v].z = fmaf(b, av[v].z, fmaf(-e, cur.B[v].z, cur.B[v].z));
+                        cur.B[v].w = fmaf(b, av[v].w, fmaf(-e, cur.B[v].w, cur.B[v].w));
+                    }
                 }
             }
         }
@@ -445,12 +463,37 @@ __global__ void __launch_bounds__(kSgdThreads, 4) sgd_chunk_kernel(const SgdChun
         C head, closing;
         comp_identity(head);
         __syncwarp();
-        if (hasb) comp_load<LG, NV>(s_head, head, l);
+        if (hasb && head_pos >= 0) {
+#pragma unroll
+            for (int v = 0; v < NV; ++v) head.B[v] = s_rows[head_pos * KP4 + v * LG + l];
+            const float4 hd = s_item[head_pos];
+            head.D = hd.x; head.Dw = hd.y; head.Bw = hd.z;
+        }
         bool outer;
         scan_step<LG, NV>(hasb, head, cur, wcarry, wflag, closing, outer);
         if (hasb) {
-            if (outer) comp_store<LG, NV>(s_wpiece + (warp * 2 + 0) * (KP4 + 1), closing, headcol, l);
-            else apply_fetch(headcol, closing);
+            if (outer) {
+                comp_store<LG, NV>(s_wpiece + (warp * 2 + 0) * (KP4 + 1), closing, headcol, l);
+            } else if (headcol != kNoCol) {
+                // the run ended at entry lo + head_pos of this pass if that is >= 0 (its scale pair
+                // was prefetched there), else in an earlier pass
+                const int pos = lo + head_pos;
+                if (pos >= 0) apply(headcol, closing, s_scale_all[(pos / S) * L::ITEM_STRIDE + (pos % S)]);
+                else apply_fetch(headcol, closing);
+            }
+        }
+        // 5. apply the runs parked in step 3, all lane groups side by side
+        while (__any_sync(0xFFFFFFFFu, emask != 0)) {
+            if (emask != 0) {
+                const int pos = __ffs(emask) - 1;
+                emask &= emask - 1;
+                C x;
+#pragma unroll
+                for (int v = 0; v < NV; ++v) x.B[v] = s_rows[pos * KP4 + v * LG + l];
+                const float4 hd = s_item[pos];
+                x.D = hd.x; x.Dw = hd.y; x.Bw = hd.z;
+                apply(__float_as_uint(hd.w), x, s_scale[pos]);
+            }
         }
         __syncwarp();
     }
