@@ -50,15 +50,33 @@ __global__ void __launch_bounds__(kThreads) refresh_kernel(const RefreshArgs a) 
             float xm = 0.f;
             if (mine < end) { jm = __ldg(a.idx + mine); xm = __ldg(a.val + mine); lin = fmaf(__ldg(a.w + jm), xm, lin); }
             const int cnt = (int)((end - t0) < (int64_t)LG ? (end - t0) : (int64_t)LG);
-            for (int u = 0; u < cnt; ++u) {
-                const int32_t j = __shfl_sync(gm, jm, u, LG);
-                const float x = __shfl_sync(gm, xm, u, LG);
+            // the rows of up to UB entries are requested before any of them is used
+            constexpr int UB = LG < 8 ? LG : 8 / NV;
 #pragma unroll
-                for (int v = 0; v < NV; ++v) {
-                    const float4 vv = __ldg(V4 + (size_t)j * KP4 + v * LG + l);
-                    const float px = vv.x * x, py = vv.y * x, pz = vv.z * x, pw = vv.w * x;
-                    acc[v].x += px; acc[v].y += py; acc[v].z += pz; acc[v].w += pw;
-                    q = fmaf(px, px, q); q = fmaf(py, py, q); q = fmaf(pz, pz, q); q = fmaf(pw, pw, q);
+            for (int u0 = 0; u0 < LG; u0 += UB) {
+                if (u0 >= cnt) break;
+                float4 vv[UB][NV];
+                float xs[UB];
+#pragma unroll
+                for (int u = 0; u < UB; ++u) {
+                    const int32_t j = __shfl_sync(gm, jm, u0 + u, LG);
+                    xs[u] = __shfl_sync(gm, xm, u0 + u, LG);
+                    if (u0 + u < cnt) {
+#pragma unroll
+                        for (int v = 0; v < NV; ++v) vv[u][v] = __ldg(V4 + (size_t)j * KP4 + v * LG + l);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < UB; ++u) {
+                    if (u0 + u < cnt) {
+                        const float x = xs[u];
+#pragma unroll
+                        for (int v = 0; v < NV; ++v) {
+                            const float px = vv[u][v].x * x, py = vv[u][v].y * x, pz = vv[u][v].z * x, pw = vv[u][v].w * x;
+                            acc[v].x += px; acc[v].y += py; acc[v].z += pz; acc[v].w += pw;
+                            q = fmaf(px, px, q); q = fmaf(py, py, q); q = fmaf(pz, pz, q); q = fmaf(pw, pw, q);
+                        }
+                    }
                 }
             }
         }
