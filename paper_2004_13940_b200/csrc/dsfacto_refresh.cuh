@@ -44,11 +44,17 @@ __global__ void __launch_bounds__(kThreads) refresh_kernel(const RefreshArgs a) 
 #pragma unroll
         for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
         float q = 0.f, lin = 0.f;
+        // this lane's entry of the next batch is fetched while the current batch is processed
+        int32_t jn = 0;
+        float xn = 0.f;
+        if (beg + l < end) { jn = __ldg(a.idx + beg + l); xn = __ldg(a.val + beg + l); }
         for (int64_t t0 = beg; t0 < end; t0 += LG) {
-            const int64_t mine = t0 + l;
-            int32_t jm = 0;
-            float xm = 0.f;
-            if (mine < end) { jm = __ldg(a.idx + mine); xm = __ldg(a.val + mine); lin = fmaf(__ldg(a.w + jm), xm, lin); }
+            const int32_t jm = jn;
+            const float xm = xn;
+            const int64_t ahead = t0 + LG + l;
+            jn = 0; xn = 0.f;
+            if (ahead < end) { jn = __ldg(a.idx + ahead); xn = __ldg(a.val + ahead); }
+            if (t0 + l < end) lin = fmaf(__ldg(a.w + jm), xm, lin);
             const int cnt = (int)((end - t0) < (int64_t)LG ? (end - t0) : (int64_t)LG);
             // the rows of up to UB entries are requested before any of them is used
             constexpr int UB = LG < 8 ? LG : 8 / NV;
