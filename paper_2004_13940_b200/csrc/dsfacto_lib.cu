@@ -50,9 +50,11 @@ struct dsfacto {
     // stratum SGD launch plan: launch L covers chunks [launch_ptr[L], launch_ptr[L+1]) of chunk_map
     int sweep = 1;  // 1: a launch is a row block (p-1 .. 0); 0: a launch is an inner round (0 .. p-1)
     std::vector<int64_t> launch_ptr;
-    int2 *d_chunk_map = nullptr;
+    int4 *d_chunk_map = nullptr;
+    int *d_sync = nullptr;     // ticket, error flag, per-column-block progress of the fused SGD launch
+    int64_t total_chunks = 0;
     float *d_records = nullptr, *d_Tb = nullptr, *d_Tw = nullptr;
-    float2 *d_S = nullptr, *d_TS = nullptr;  // scale pairs of the scaled column state (zero outside the SGD phase)
+    float4 *d_S = nullptr, *d_TS = nullptr;  // scale pairs of the scaled column state (zero outside the SGD phase)
     int *d_tile_count = nullptr;
     int refresh_grid = 0, norm_grid = 0;
 
@@ -151,7 +153,7 @@ void unpack_tiles(const dsfacto *h, const uint2 *ent, const float *xw, int32_t *
 void free_data(dsfacto *h) {
     dev_free(h->d_A); dev_free(h->d_G); dev_free(h->d_y); dev_free(h->d_val); dev_free(h->d_xw);
     dev_free(h->d_indptr); dev_free(h->d_tile_ptr); dev_free(h->d_idx); dev_free(h->d_ent);
-    dev_free(h->d_partials); dev_free(h->d_chunk_map); dev_free(h->d_records); dev_free(h->d_tile_count);
+    dev_free(h->d_partials); dev_free(h->d_chunk_map); dev_free(h->d_records); dev_free(h->d_tile_count); dev_free(h->d_sync);
     h->launch_ptr.clear();
     h->loaded = false;
     h->nnz = 0;
@@ -205,10 +207,11 @@ int refresh_grid_for(const dsfacto *h, int64_t rows) {
 // chunks of kChunk entries.  Tiles of one launch have pairwise disjoint column blocks.
 int build_sgd_plan(dsfacto *h) {
     const int64_t p = h->p;
-    std::vector<int2> map;
-    int64_t max_launch = 0;
+    std::vector<int4> map;
+    std::vector<int> seen;  // non-empty tiles met so far per column block
     try {
         h->launch_ptr.assign((size_t)p + 1, 0);
+        seen.assign((size_t)p, 0);
         map.reserve((size_t)(h->nnz / kChunk + p * p / 4 + 16));
         for (int64_t L = 0; L < p; ++L) {
             for (int64_t k = 0; k < p; ++k) {
@@ -216,27 +219,30 @@ int build_sgd_plan(dsfacto *h) {
                 if (h->sweep == 1) { r = p - 1 - L; s = ((k - r) % p + p) % p; }   // column block c = k
                 else { s = L; r = k; }
                 const int64_t t = s * p + r;
+                const int64_t c = (r + s) % p;
                 const int64_t cnt = h->tile_ptr[t + 1] - h->tile_ptr[t];
                 const int64_t nch = (cnt + kChunk - 1) / kChunk;
-                for (int64_t ci = 0; ci < nch; ++ci) map.push_back(make_int2((int)t, (int)ci));
+                for (int64_t ci = 0; ci < nch; ++ci) map.push_back(make_int4((int)t, (int)ci, seen[c], 0));
+                if (nch > 0) seen[c] += 1;
             }
             h->launch_ptr[L + 1] = (int64_t)map.size();
-            max_launch = std::max(max_launch, h->launch_ptr[L + 1] - h->launch_ptr[L]);
         }
     } catch (const std::bad_alloc &) { return DSFACTO_ERR_OOM; }
+    if (map.size() >= ((size_t)1 << 31)) return DSFACTO_ERR_INVALID_ARG;
+    h->total_chunks = (int64_t)map.size();
     int rc;
     if ((rc = dev_alloc(h, &h->d_chunk_map, map.size())) ||
-        (rc = dev_alloc(h, &h->d_records, (size_t)max_launch * chunk_record_floats(h->Kp))) ||
-        (rc = dev_alloc(h, &h->d_tile_count, (size_t)(p * p))))
+        (rc = dev_alloc(h, &h->d_records, map.size() * chunk_record_floats(h->Kp))) ||
+        (rc = dev_alloc(h, &h->d_tile_count, (size_t)(p * p))) || (rc = dev_alloc(h, &h->d_sync, (size_t)p + 2)))
         return rc;
     CU_TRY(h, cudaMemsetAsync(h->d_tile_count, 0, sizeof(int) * (size_t)(p * p), h->stream));
     if (!map.empty())
-        CU_TRY(h, cudaMemcpyAsync(h->d_chunk_map, map.data(), sizeof(int2) * map.size(), cudaMemcpyHostToDevice, h->stream));
+        CU_TRY(h, cudaMemcpyAsync(h->d_chunk_map, map.data(), sizeof(int4) * map.size(), cudaMemcpyHostToDevice, h->stream));
     CU_TRY(h, cudaStreamSynchronize(h->stream));
     return DSFACTO_OK;
 }
 
-// the p strata of one epoch (plus, after a row-block sweep, folding the tail composites in)
+// the p strata of one epoch, then the return from the scaled state to plain parameters
 void run_sgd_phase(dsfacto *h) {
     SgdChunkArgs a{};
     a.tile_ptr = h->d_tile_ptr; a.ent = h->d_ent; a.xw = h->d_xw; a.row_start = h->d_row_start;
@@ -244,11 +250,13 @@ void run_sgd_phase(dsfacto *h) {
     a.S = h->d_S; a.Tb = h->d_Tb; a.Tw = h->d_Tw; a.TS = h->d_TS; a.records = h->d_records; a.tile_count = h->d_tile_count;
     a.p = h->p; a.jbits = h->jbits; a.sweep = h->sweep;
     a.h = h->h; a.lambda_w = h->lambda_w; a.lambda_v = h->lambda_v;
-    for (int L = 0; L < h->p; ++L) {
-        const int64_t grid = h->launch_ptr[L + 1] - h->launch_ptr[L];
-        if (grid == 0) continue;
-        a.chunk_map = h->d_chunk_map + h->launch_ptr[L];
-        DSF_DISPATCH(h, launch_sgd, h, a, (int)grid);
+    // One launch for the whole sweep: chunks are taken in sweep order (row block by row block, or round
+    // by round) and a tile waits only for the earlier tiles of its own column block.
+    cudaMemsetAsync(h->d_sync, 0, sizeof(int) * ((size_t)h->p + 2), h->stream);
+    a.chunk_map = h->d_chunk_map;
+    a.sync = h->d_sync;
+    if (h->total_chunks > 0) {
+        DSF_DISPATCH(h, launch_sgd, h, a, (int)h->total_chunks);
         h->launches += 1;
     }
     {   // back from the scaled state to plain (w, V); folds the tail composites in after a row-block sweep
@@ -530,14 +538,14 @@ int dsfacto_create(dsfacto_t **out, int64_t n, int32_t d, int32_t K, int32_t p, 
     h->norm_grid = h->sm_count * 8;
     if (const char *env = std::getenv("DSFACTO_SWEEP")) h->sweep = (std::strcmp(env, "round") == 0) ? 0 : 1;
     if ((rc = dev_alloc(h, &h->d_S, (size_t)d))) return fail(rc);
-    if (cudaMemset(h->d_S, 0, sizeof(float2) * (size_t)d) != cudaSuccess) return fail(DSFACTO_ERR_CUDA);
+    if (cudaMemset(h->d_S, 0, sizeof(float4) * (size_t)d) != cudaSuccess) return fail(DSFACTO_ERR_CUDA);
     if (h->sweep == 1) {
         if ((rc = dev_alloc(h, &h->d_Tb, (size_t)d * h->Kp)) || (rc = dev_alloc(h, &h->d_Tw, (size_t)d)) ||
             (rc = dev_alloc(h, &h->d_TS, (size_t)d)))
             return fail(rc);
         if (cudaMemset(h->d_Tb, 0, sizeof(float) * (size_t)d * h->Kp) != cudaSuccess ||
             cudaMemset(h->d_Tw, 0, sizeof(float) * (size_t)d) != cudaSuccess ||
-            cudaMemset(h->d_TS, 0, sizeof(float2) * (size_t)d) != cudaSuccess)
+            cudaMemset(h->d_TS, 0, sizeof(float4) * (size_t)d) != cudaSuccess)
             return fail(DSFACTO_ERR_CUDA);
     }
     *out = h;
@@ -622,6 +630,9 @@ int dsfacto_epoch(dsfacto_t *h) {
     CU_TRY(h, cudaEventRecord(h->ev[1], st));
     int rc = run_refresh(h, true);
     if (rc) return rc;
+    int sgd_error = 0;  // set by the SGD kernel if a dependency wait ran out (never seen; the state is then unusable)
+    CU_TRY(h, cudaMemcpy(&sgd_error, h->d_sync + 1, sizeof(int), cudaMemcpyDeviceToHost));
+    if (sgd_error) { h->err = "stratum SGD: a wait for an earlier tile of the same column block timed out"; return DSFACTO_ERR_CUDA; }
     float t01 = 0, t12 = 0, t23 = 0;
     cudaEventElapsedTime(&t01, h->ev[0], h->ev[1]);
     cudaEventElapsedTime(&t12, h->ev[1], h->ev[2]);

@@ -28,6 +28,7 @@ constexpr int kSgdThreads = 128;  // 4 warps per CTA
 constexpr int kSgdWarps = kSgdThreads / 32;
 constexpr int kWarpEntries = 512;                 // entries per warp
 constexpr int kChunk = kSgdWarps * kWarpEntries;  // entries per CTA
+constexpr int kSgdSpinLimit = 1 << 22;            // polls (about 100 ns each) before a dependency wait gives up
 
 // entries of one warp pass: sized so that the gathered rows of A fill about 8 KB of shared memory
 __host__ __device__ constexpr int sgd_pass_len(int LG, int NV) {
@@ -47,9 +48,9 @@ struct SgdSmem {
     static constexpr int ROW_STRIDE = (S + (LG < 8 ? 1 : 0)) * KP4;
     static constexpr int ITEMS = 0;                      // GW * ITEM_STRIDE   {e, b, row, j_local}
     static constexpr int ROWS = ITEMS + GW * ITEM_STRIDE;  // GW * ROW_STRIDE  gathered rows a_i
-    static constexpr int SCALES = ROWS + GW * ROW_STRIDE;  // GW * ITEM_STRIDE float2: scale pair of the
+    static constexpr int SCALES = ROWS + GW * ROW_STRIDE;  // GW * ITEM_STRIDE float4: scale pair of the
                                                          // column whose run starts at that entry
-    static constexpr int WARP = SCALES + (GW * ITEM_STRIDE + 1) / 2;  // float4s per warp
+    static constexpr int WARP = SCALES + GW * ITEM_STRIDE;  // float4s per warp
     // per CTA, after the warps: per warp head/tail pieces, then the chunk head piece
     static constexpr int WPIECE = kSgdWarps * WARP;      // kSgdWarps * 2 * (KP4+1)
     static constexpr int CPIECE = WPIECE + kSgdWarps * 2 * (KP4 + 1);  // (KP4+1)
@@ -138,10 +139,6 @@ __device__ __forceinline__ uint32_t comp_load(const float4 *src, Comp<NV> &c, in
 __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src) {
     const unsigned s = (unsigned)__cvta_generic_to_shared(smem_dst);
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem_src) : "memory");
-}
-__device__ __forceinline__ void cp_async8(void *smem_dst, const void *gmem_src) {
-    const unsigned s = (unsigned)__cvta_generic_to_shared(smem_dst);
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;\n" ::"r"(s), "l"(gmem_src) : "memory");
 }
 // fire-and-forget adds into global memory
 __device__ __forceinline__ void red_add4(float4 *p, float x, float y, float z, float w) {
@@ -237,13 +234,16 @@ struct SgdChunkArgs {
     const float *G;            // n
     float *w;                  // d        u-part of w_j
     float *V;                  // d * Kp   u-part of v_j
-    float2 *S;                 // d        {sigma of v_j, sigma of w_j}
+    float4 *S;                 // d        {sigma of v_j, sigma of w_j, -, -}
     float *Tw;                 // d        u-part of the w offset of T_j      (sweep 1)
     float *Tb;                 // d * Kp   u-part of the v offset of T_j      (sweep 1)
-    float2 *TS;                // d        {D, Dw} of T_j                     (sweep 1)
-    const int2 *chunk_map;     // per CTA of this launch: {tile t, chunk index inside the tile}
-    float *records;            // chunk_record_floats(Kp) floats per CTA of this launch
+    float4 *TS;                // d        {D, Dw, -, -} of T_j               (sweep 1)
+    const int4 *chunk_map;     // per chunk, in sweep order: {tile t, chunk index inside the tile, number
+                               // of earlier non-empty tiles of the same column block, -}
+    float *records;            // chunk_record_floats(Kp) floats per chunk
     int *tile_count;           // p*p, all zero between launches
+    int *sync;                 // [0] ticket counter, [1] error flag, [2 + c] finished tiles of column block c;
+                               // all zero at launch
     int p, jbits, sweep;
     float h, lambda_w, lambda_v;
 };
@@ -265,16 +265,38 @@ __global__ void __launch_bounds__(kSgdThreads, 4) sgd_chunk_kernel(const SgdChun
     float4 *sw = smem4 + warp * L::WARP;
     float4 *s_item = sw + L::ITEMS + g * L::ITEM_STRIDE;
     float4 *s_rows = sw + L::ROWS + g * L::ROW_STRIDE;
-    float2 *s_scale_all = reinterpret_cast<float2 *>(sw + L::SCALES);
-    float2 *s_scale = s_scale_all + g * L::ITEM_STRIDE;
+    float4 *s_scale_all = sw + L::SCALES;
+    float4 *s_scale = s_scale_all + g * L::ITEM_STRIDE;
     float4 *s_wpiece = smem4 + L::WPIECE;  // [warp][head/tail][KP4+1]
     float4 *s_cpiece = smem4 + L::CPIECE;
     int *s_wflag = reinterpret_cast<int *>(smem4 + L::TOTAL);
 
-    const int2 cm = a.chunk_map[blockIdx.x];
+    // Chunks are handed out in sweep order by a ticket counter, so a CTA that holds a ticket knows that
+    // every earlier chunk has been taken by a CTA that is running or done: waiting for earlier tiles of
+    // the same column block can therefore not deadlock.  The wait is bounded all the same; on a
+    // time-out the error flag makes every CTA leave and the host reports the failure.
+    __shared__ int s_ticket, s_go;
+    if (tid == 0) s_ticket = atomicAdd(a.sync, 1);
+    __syncthreads();
+    const int chunk = s_ticket;
+    const int4 cm = a.chunk_map[chunk];
     const int64_t t = cm.x;
     const int r = (int)(t % a.p), s = (int)(t / a.p);
     const int c = (r + s) % a.p;
+    if (tid == 0) {
+        int go = 1;
+        const volatile int *done = a.sync + 2 + c;
+        const volatile int *err = a.sync + 1;
+        for (int spin = 0; *done < cm.z; ++spin) {
+            if (*err != 0 || spin > kSgdSpinLimit) { go = 0; break; }
+            __nanosleep(100);
+        }
+        if (!go) atomicExch(a.sync + 1, 1);
+        __threadfence();
+        s_go = go;
+    }
+    __syncthreads();
+    if (!s_go) return;
     const bool tail_mode = a.sweep == 1 && r > c;
     const int64_t tb = a.tile_ptr[t], te = a.tile_ptr[t + 1];
     const int64_t cb = tb + (int64_t)cm.y * kChunk;
@@ -294,10 +316,10 @@ __global__ void __launch_bounds__(kSgdThreads, 4) sgd_chunk_kernel(const SgdChun
     // the column state this tile acts on (u-parts and scale pairs), shifted to the column block
     float4 *U4 = reinterpret_cast<float4 *>(tail_mode ? a.Tb : a.V) + (size_t)col0 * KP4;
     float *uw = (tail_mode ? a.Tw : a.w) + col0;
-    float2 *Sc = (tail_mode ? a.TS : a.S) + col0;
+    float4 *Sc = (tail_mode ? a.TS : a.S) + col0;
 
     // column state <- run o column state, given the column's scale pair (lanes of one group)
-    auto apply = [&](uint32_t jl, const C &x, float2 sc) {
+    auto apply = [&](uint32_t jl, const C &x, float4 sc) {
         const float sg = fmaf(sc.x, x.D, sc.x + x.D);
         const float inv = __frcp_rn(1.0f + sg);
 #pragma unroll
@@ -307,13 +329,13 @@ __global__ void __launch_bounds__(kSgdThreads, 4) sgd_chunk_kernel(const SgdChun
         if (l == 0) {
             const float sgw = fmaf(sc.y, x.Dw, sc.y + x.Dw);
             red_add1(uw + jl, x.Bw * __frcp_rn(1.0f + sgw));
-            Sc[jl] = make_float2(sg, sgw);
+            Sc[jl] = make_float4(sg, sgw, 0.f, 0.f);
         }
     };
-    // the same with the scale pair fetched from global memory (an L2 hit after the first launch)
+    // the same with the scale pair fetched from L2 (never through L1: another SM wrote it in this launch)
     auto apply_fetch = [&](uint32_t jl, const C &x) {
         if (jl == kNoCol) return;
-        apply(jl, x, Sc[jl]);
+        apply(jl, x, __ldcg(Sc + jl));
     };
 
     // ---------------- warp phase ----------------
@@ -392,7 +414,7 @@ __global__ void __launch_bounds__(kSgdThreads, 4) sgd_chunk_kernel(const SgdChun
             bool ends;
             if (at + 1 < cnt) ends = nextcol != jq[q];
             else ends = after_known && after != jq[q];
-            if (at < cnt && ends) cp_async8(s_scale_all + (at / S) * L::ITEM_STRIDE + (at % S), Sc + jq[q]);
+            if (at < cnt && ends) cp_async16(s_scale_all + (at / S) * L::ITEM_STRIDE + (at % S), Sc + jq[q]);
         }
         __syncwarp();
         // 2. gather the rows a_i of the pass
@@ -501,6 +523,7 @@ __global__ void __launch_bounds__(kSgdThreads, 4) sgd_chunk_kernel(const SgdChun
         comp_store<LG, NV>(s_wpiece + (warp * 2 + 1) * (KP4 + 1), wcarry, last_col, l);
         if (l == 0) s_wflag[warp] = wflag ? 1 : 0;
     }
+    __threadfence();  // this warp's state updates are ordered before the tile's completion signal below
     __syncthreads();
     if (warp != 0) return;
 
@@ -540,10 +563,13 @@ __global__ void __launch_bounds__(kSgdThreads, 4) sgd_chunk_kernel(const SgdChun
         // the tile starts and ends in this chunk: its head piece belongs to no column, and the end
         // of the tile closes the run that is still open
         if (g == 0) apply_fetch(ctailcol, ccarry);
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) atomicAdd(a.sync + 2 + c, 1);  // this tile of column block c is done
         return;
     }
     {
-        float4 *rec4 = reinterpret_cast<float4 *>(a.records) + (size_t)blockIdx.x * REC4;
+        float4 *rec4 = reinterpret_cast<float4 *>(a.records) + (size_t)chunk * REC4;
         if (lane < LG) {
             if (l == 0) {
                 rec4[0] = cflag ? s_cpiece[KP4] : make_float4(0.f, 0.f, 0.f, __uint_as_float(kNoCol));
@@ -566,7 +592,7 @@ __global__ void __launch_bounds__(kSgdThreads, 4) sgd_chunk_kernel(const SgdChun
     last = __shfl_sync(0xFFFFFFFFu, last, 0);
     if (!last) return;
     __threadfence();
-    const float4 *base4 = reinterpret_cast<const float4 *>(a.records) + ((size_t)blockIdx.x - (size_t)cm.y) * REC4;
+    const float4 *base4 = reinterpret_cast<const float4 *>(a.records) + ((size_t)chunk - (size_t)cm.y) * REC4;
     C tcarry;
     comp_identity(tcarry);
     bool tflag = false;
@@ -598,7 +624,12 @@ __global__ void __launch_bounds__(kSgdThreads, 4) sgd_chunk_kernel(const SgdChun
     }
     const uint32_t ttailcol = __float_as_uint(__ldcg(base4 + (size_t)(nchunks - 1) * REC4 + 1).w);
     if (g == 0) apply_fetch(ttailcol, tcarry);  // the end of the tile closes the last run
-    if (lane == 0) a.tile_count[t] = 0;
+    __threadfence();
+    __syncwarp();
+    if (lane == 0) {
+        a.tile_count[t] = 0;
+        atomicAdd(a.sync + 2 + c, 1);  // this tile of column block c is done
+    }
 }
 
 // End of the SGD phase: back from the scaled state to plain parameters,
@@ -606,8 +637,8 @@ __global__ void __launch_bounds__(kSgdThreads, 4) sgd_chunk_kernel(const SgdChun
 // where T_j = (D_T, ub_j) is the tail composite (identity unless the launch order was the row-block
 // sweep), and reset of the scale pairs and of T_j.  Two kernels because the first reads the scale
 // pairs that the second clears.
-__global__ void __launch_bounds__(kThreads) sgd_finalize_v_kernel(float *V, float *Tb, const float2 *S,
-                                                                  const float2 *TS, int64_t d, int kp4) {
+__global__ void __launch_bounds__(kThreads) sgd_finalize_v_kernel(float *V, float *Tb, const float4 *S,
+                                                                  const float4 *TS, int64_t d, int kp4) {
     const int64_t total = d * kp4;
     float4 *V4 = reinterpret_cast<float4 *>(V);
     float4 *Tb4 = reinterpret_cast<float4 *>(Tb);
@@ -626,16 +657,16 @@ __global__ void __launch_bounds__(kThreads) sgd_finalize_v_kernel(float *V, floa
         V4[i] = y;
     }
 }
-__global__ void __launch_bounds__(kThreads) sgd_finalize_w_kernel(float *w, float *Tw, float2 *S, float2 *TS, int64_t d) {
+__global__ void __launch_bounds__(kThreads) sgd_finalize_w_kernel(float *w, float *Tw, float4 *S, float4 *TS, int64_t d) {
     for (int64_t j = (int64_t)blockIdx.x * kThreads + threadIdx.x; j < d; j += (int64_t)gridDim.x * kThreads) {
         float wj = w[j];
         wj = fmaf(S[j].y, wj, wj);
-        S[j] = make_float2(0.f, 0.f);
+        S[j] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (Tw != nullptr) {
             wj += Tw[j];
             wj = fmaf(TS[j].y, wj, wj);
             Tw[j] = 0.f;
-            TS[j] = make_float2(0.f, 0.f);
+            TS[j] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
         w[j] = wj;
     }
