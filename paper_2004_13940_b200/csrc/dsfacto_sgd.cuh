@@ -26,7 +26,7 @@ namespace dsf {
 
 constexpr int kSgdThreads = 128;  // 4 warps per CTA
 constexpr int kSgdWarps = kSgdThreads / 32;
-constexpr int kWarpEntries = 512;                 // entries per warp
+constexpr int kWarpEntries = 1024;                // entries per warp
 constexpr int kChunk = kSgdWarps * kWarpEntries;  // entries per CTA
 constexpr int kSgdSpinLimit = 1 << 22;            // polls (about 100 ns each) before a dependency wait gives up
 
