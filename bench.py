@@ -33,7 +33,7 @@ UNIT = "updates/s"
 ORACLE_SAMPLE_ROWS = 1_000_000
 # dram__bytes_read.sum + dram__bytes_write.sum of sgd_chunk_kernel per stored entry, from the ncu capture
 # summarised in profiles/ (None once the kernel has changed since the counters were taken)
-SGD_DRAM_BYTES_PER_ENTRY = None
+SGD_DRAM_BYTES_PER_ENTRY = 20.1
 
 
 def peaks():
@@ -142,6 +142,33 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def take_turns(rank, world, barrier, fn):
+    """Runs fn() on one rank at a time (rank order), a barrier after each turn; returns this rank's result.
+    Used for the loads, so that the host-side bucketing buffers of the replicas never coexist."""
+    out = None
+    for turn in range(world):
+        if turn == rank:
+            out = fn()
+        barrier()
+    return out
+
+
+def max_over_ranks(values, world, device):
+    """Element-wise maximum of a list of floats over all ranks (identity for one rank)."""
+    if world == 1:
+        return [float(v) for v in values]
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(v) for v in values], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.tolist()]
+
+
+def whole_job_rate(world, units_per_rank, steps, ms):
+    """Units all replicas processed per second, given the slowest rank's time for `steps` steps."""
+    return world * units_per_rank * steps / (ms * 1e-3)
+
+
 def workload_config(name, sample_rows=None):
     from paper_2004_13940_b200 import workloads as W
     c = W.CONFIGS[name]
@@ -192,15 +219,13 @@ def run_ours(args):
         return g
 
     # ranks load one after another so that the host-side bucketing buffers never coexist
-    g = None
-    t_load = 0.0
-    for turn in range(world):
-        if turn == rank:
-            t0 = time.perf_counter()
-            g = new_handle()
-            g.load_csr(wl.indptr, wl.indices, wl.values, wl.y)
-            t_load = time.perf_counter() - t0
-        barrier()
+    def first_load():
+        t0 = time.perf_counter()
+        gg = new_handle()
+        gg.load_csr(wl.indptr, wl.indices, wl.values, wl.y)
+        return gg, time.perf_counter() - t0
+
+    g, t_load = take_turns(rank, world, barrier, first_load)
 
     for _ in range(args.warmup):
         g.epoch()
@@ -224,25 +249,20 @@ def run_ours(args):
     g.close()
 
     # ---- e2e: host buffers -> load_csr -> epoch -> objective, through the C ABI ----
-    e2e_ms = 0.0
-    for turn in range(world):
-        if turn == rank:
-            torch.cuda.synchronize()
-            t0 = time.perf_counter()
-            for _ in range(args.e2e_steps):
-                h = new_handle()
-                h.load_csr(wl.indptr, wl.indices, wl.values, wl.y)
-                h.epoch()
-                _ = h.objective()
-                h.close()
-            torch.cuda.synchronize()
-            e2e_ms = 1e3 * (time.perf_counter() - t0)
-        barrier()
+    def e2e_leg():
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            hh = new_handle()
+            hh.load_csr(wl.indptr, wl.indices, wl.values, wl.y)
+            hh.epoch()
+            _ = hh.objective()
+            hh.close()
+        torch.cuda.synchronize()
+        return 1e3 * (time.perf_counter() - t0)
 
-    if world > 1:
-        t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, e2e_ms = float(t[0]), float(t[1])
+    e2e_ms = take_turns(rank, world, barrier, e2e_leg)
+    ms, e2e_ms = max_over_ranks([ms, e2e_ms], world, "cuda")
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -260,20 +280,20 @@ def run_ours(args):
     sgd_bytes = sgd_gather if sweep == "round" else sgd_floor
     ref_bytes = 8 * nnz + 8 * (n + 1) + 4 * d * (K + 2) + 4 * n * K + 8 * n
     sgd_s, ref_s = phase[1] * 1e-3, phase[2] * 1e-3
-    traffic = None if SGD_DRAM_BYTES_PER_ENTRY is None else SGD_DRAM_BYTES_PER_ENTRY * nnz / p
-    roof = {"bound": "hbm", "kernel": "sgd_chunk_kernel", "launches_per_step": p, "sweep": sweep,
+    traffic = None if SGD_DRAM_BYTES_PER_ENTRY is None else SGD_DRAM_BYTES_PER_ENTRY * nnz   # one launch per sweep
+    roof = {"bound": "hbm", "kernel": "sgd_chunk_kernel", "launches_per_step": 1, "sweep": sweep,
             "achieved": sgd_bytes / sgd_s / 1e9, "peak": peak, "unit": "GB/s", "frac": sgd_bytes / sgd_s / 1e9 / peak,
             "peak_kind": "of " + peak_kind, "traffic": traffic,
-            "algorithmic_bytes_per_launch": sgd_bytes / p, "avg_launch_us": 1e6 * sgd_s / p,
+            "algorithmic_bytes_per_launch": sgd_bytes, "avg_launch_us": 1e6 * sgd_s,
             "model": ("gather: nnz*(8+4K+4) + 8d(K+1)" if sweep == "round" else "stream floor: 8nnz + 4n(K+1) + 8d(K+1)")
-                     + ", per launch = 1/p of it",
+                     + "; one launch covers the whole sweep",
             "gather_model": {"bytes_per_step": sgd_gather, "achieved": sgd_gather / sgd_s / 1e9,
                              "frac": sgd_gather / sgd_s / 1e9 / peak},
             "refresh_kernel": {"algorithmic_bytes_per_step": ref_bytes, "ms": phase[2],
                                "achieved": ref_bytes / ref_s / 1e9, "frac": ref_bytes / ref_s / 1e9 / peak}}
-    value = world * nnz * args.steps / (ms * 1e-3)
+    value = whole_job_rate(world, nnz, args.steps, ms)
     h2d = (wl.indptr.nbytes + wl.indices.nbytes + wl.values.nbytes + wl.y.nbytes + 8 * nnz + 8 * (p * p + 1))
-    e2e = {"value": world * nnz * args.e2e_steps / (e2e_ms * 1e-3) if args.e2e_steps > 0 else None, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+    e2e = {"value": whole_job_rate(world, nnz, args.e2e_steps, e2e_ms) if args.e2e_steps > 0 else None, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
            "d2h_bytes_per_step": 32, "steps": args.e2e_steps, "ms_per_step": e2e_ms / max(args.e2e_steps, 1),
            "what": "dsfacto_create + dsfacto_load_csr (host bucketing, H2D) + dsfacto_epoch + dsfacto_objective"}
     cfg = workload_config(args.workload)
