@@ -85,6 +85,24 @@ void dev_free(T *&ptr) {
     ptr = nullptr;
 }
 
+// Large host scratch without the zero fill of std::vector: the pages are first touched by the
+// parallel passes that write them.
+template <typename T>
+struct HostBuf {
+    T *p = nullptr;
+    HostBuf() = default;
+    HostBuf(const HostBuf &) = delete;
+    HostBuf &operator=(const HostBuf &) = delete;
+    ~HostBuf() { std::free(p); }
+    bool alloc(size_t count) {
+        std::free(p);
+        p = static_cast<T *>(std::malloc((count ? count : 1) * sizeof(T)));
+        return p != nullptr;
+    }
+    T *data() { return p; }
+    T &operator[](size_t i) { return p[i]; }
+};
+
 // ---- SplitMix64 (Steele, Lea, Flood 2014), random access to the c-th output ----
 inline uint64_t splitmix64_output(uint64_t seed, uint64_t c) {
     uint64_t z = seed + (c + 1) * 0x9E3779B97F4A7C15ull;
@@ -339,7 +357,7 @@ int validate_csr(int64_t m, int32_t d, const int64_t *indptr, const int32_t *ind
 // by local column inside every tile.
 // ---------------------------------------------------------------------------------------------
 int bucket_tiles(dsfacto *h, const int64_t *indptr, const int32_t *indices, const float *values,
-                 std::vector<uint2> &ent, std::vector<float> &xw) {
+                 HostBuf<uint2> &ent, HostBuf<float> &xw) {
     const int64_t n = h->n, nnz = indptr[n];
     const int32_t d = h->d, p = h->p;
     const int64_t nt = (int64_t)p * p;
@@ -365,14 +383,13 @@ int bucket_tiles(dsfacto *h, const int64_t *indptr, const int32_t *indices, cons
     rs[T] = n;
 
     std::vector<uint32_t> counts;
-    std::vector<uint2> tmp_e;
-    std::vector<float> tmp_x;
+    HostBuf<uint2> tmp_e;
+    HostBuf<float> tmp_x;
     try {
         counts.assign((size_t)T * nt, 0u);
-        tmp_e.resize((size_t)std::max<int64_t>(nnz, 1));
-        if (wide) tmp_x.resize((size_t)std::max<int64_t>(nnz, 1));
-        ent.resize((size_t)std::max<int64_t>(nnz, 1));
-        if (wide) xw.resize((size_t)std::max<int64_t>(nnz, 1));
+        if (!tmp_e.alloc((size_t)nnz) || (wide && !tmp_x.alloc((size_t)nnz)) || !ent.alloc((size_t)nnz) ||
+            (wide && !xw.alloc((size_t)nnz)))
+            return DSFACTO_ERR_OOM;
     } catch (const std::bad_alloc &) {
         return DSFACTO_ERR_OOM;
     }
@@ -585,31 +602,40 @@ int dsfacto_load_csr(dsfacto_t *h, const int64_t *indptr, const int32_t *indices
 
     CU_TRY(h, cudaStreamSynchronize(h->stream));
     free_data(h);
-    std::vector<uint2> ent;
-    std::vector<float> xw;
-    if ((rc = bucket_tiles(h, indptr, indices, values, ent, xw))) return rc;
     h->nnz = nnz;
     h->refresh_grid = refresh_grid_for(h, n);
-
     const size_t cnt = (size_t)std::max<int64_t>(nnz, 1);
+    cudaStream_t st = h->stream;
+    // the CSR copy for the recompute pass goes out first: from page-locked caller memory it overlaps
+    // the host bucketing below
     if ((rc = dev_alloc(h, &h->d_indptr, (size_t)n + 1)) || (rc = dev_alloc(h, &h->d_idx, cnt)) ||
-        (rc = dev_alloc(h, &h->d_val, cnt)) || (rc = dev_alloc(h, &h->d_y, (size_t)n)) ||
-        (rc = dev_alloc(h, &h->d_A, (size_t)n * h->Kp)) || (rc = dev_alloc(h, &h->d_G, (size_t)n)) ||
-        (rc = dev_alloc(h, &h->d_tile_ptr, h->tile_ptr.size())) || (rc = dev_alloc(h, &h->d_ent, cnt)) ||
-        (rc = dev_alloc(h, &h->d_partials, 2 * ((size_t)h->refresh_grid + (size_t)h->norm_grid)))) {
+        (rc = dev_alloc(h, &h->d_val, cnt)) || (rc = dev_alloc(h, &h->d_y, (size_t)n))) {
         free_data(h);
         return rc;
     }
-    if (h->wide && (rc = dev_alloc(h, &h->d_xw, cnt))) { free_data(h); return rc; }
-    cudaStream_t st = h->stream;
     CU_TRY(h, cudaMemcpyAsync(h->d_indptr, indptr, sizeof(int64_t) * ((size_t)n + 1), cudaMemcpyHostToDevice, st));
     if (nnz > 0) {
         CU_TRY(h, cudaMemcpyAsync(h->d_idx, indices, sizeof(int32_t) * (size_t)nnz, cudaMemcpyHostToDevice, st));
         CU_TRY(h, cudaMemcpyAsync(h->d_val, values, sizeof(float) * (size_t)nnz, cudaMemcpyHostToDevice, st));
+    }
+    CU_TRY(h, cudaMemcpyAsync(h->d_y, y, sizeof(float) * (size_t)n, cudaMemcpyHostToDevice, st));
+
+    HostBuf<uint2> ent;
+    HostBuf<float> xw;
+    if ((rc = bucket_tiles(h, indptr, indices, values, ent, xw))) { cudaStreamSynchronize(st); free_data(h); return rc; }
+    h->nnz = nnz;   // (free_data on an error path above resets it)
+    if ((rc = dev_alloc(h, &h->d_A, (size_t)n * h->Kp)) || (rc = dev_alloc(h, &h->d_G, (size_t)n)) ||
+        (rc = dev_alloc(h, &h->d_tile_ptr, h->tile_ptr.size())) || (rc = dev_alloc(h, &h->d_ent, cnt)) ||
+        (rc = dev_alloc(h, &h->d_partials, 2 * ((size_t)h->refresh_grid + (size_t)h->norm_grid))) ||
+        (h->wide && (rc = dev_alloc(h, &h->d_xw, cnt)))) {
+        cudaStreamSynchronize(st);
+        free_data(h);
+        return rc;
+    }
+    if (nnz > 0) {
         CU_TRY(h, cudaMemcpyAsync(h->d_ent, ent.data(), sizeof(uint2) * (size_t)nnz, cudaMemcpyHostToDevice, st));
         if (h->wide) CU_TRY(h, cudaMemcpyAsync(h->d_xw, xw.data(), sizeof(float) * (size_t)nnz, cudaMemcpyHostToDevice, st));
     }
-    CU_TRY(h, cudaMemcpyAsync(h->d_y, y, sizeof(float) * (size_t)n, cudaMemcpyHostToDevice, st));
     CU_TRY(h, cudaMemcpyAsync(h->d_tile_ptr, h->tile_ptr.data(), sizeof(int64_t) * h->tile_ptr.size(), cudaMemcpyHostToDevice, st));
     CU_TRY(h, cudaStreamSynchronize(st));
     if ((rc = build_sgd_plan(h))) { free_data(h); return rc; }
@@ -700,12 +726,9 @@ int dsfacto_get_tiles(dsfacto_t *h, int64_t *tile_ptr, int32_t *rows, int32_t *c
     const int64_t nt = (int64_t)h->p * h->p;
     if (tile_ptr) std::memcpy(tile_ptr, h->tile_ptr.data(), sizeof(int64_t) * ((size_t)nt + 1));
     if (!rows && !cols && !vals) return DSFACTO_OK;
-    std::vector<uint2> ent;
-    std::vector<float> xw;
-    try {
-        ent.resize((size_t)std::max<int64_t>(h->nnz, 1));
-        if (h->wide) xw.resize((size_t)std::max<int64_t>(h->nnz, 1));
-    } catch (const std::bad_alloc &) { return DSFACTO_ERR_OOM; }
+    HostBuf<uint2> ent;
+    HostBuf<float> xw;
+    if (!ent.alloc((size_t)h->nnz) || (h->wide && !xw.alloc((size_t)h->nnz))) return DSFACTO_ERR_OOM;
     if (h->nnz > 0) {
         CU_TRY(h, cudaMemcpyAsync(ent.data(), h->d_ent, sizeof(uint2) * (size_t)h->nnz, cudaMemcpyDeviceToHost, h->stream));
         if (h->wide) CU_TRY(h, cudaMemcpyAsync(xw.data(), h->d_xw, sizeof(float) * (size_t)h->nnz, cudaMemcpyDeviceToHost, h->stream));
@@ -725,8 +748,8 @@ int dsfacto_bucket_host(int64_t n, int32_t d, int32_t p, const int64_t *indptr, 
     dsfacto tmp;
     tmp.n = n; tmp.d = d; tmp.p = p;
     if ((rc = setup_partition(&tmp))) return rc;
-    std::vector<uint2> ent;
-    std::vector<float> xw;
+    HostBuf<uint2> ent;
+    HostBuf<float> xw;
     if ((rc = bucket_tiles(&tmp, indptr, indices, values, ent, xw))) return rc;
     std::memcpy(tile_ptr, tmp.tile_ptr.data(), sizeof(int64_t) * tmp.tile_ptr.size());
     unpack_tiles(&tmp, ent.data(), xw.data(), rows, cols, vals);
