@@ -24,7 +24,7 @@
 
 namespace dsf {
 
-constexpr int kSgdThreads = 128;  // 4 warps per CTA
+constexpr int kSgdThreads = 32;   // one warp per CTA: a finished warp frees its registers and shared memory at once
 constexpr int kSgdWarps = kSgdThreads / 32;
 constexpr int kWarpEntries = 1024;                // entries per warp
 constexpr int kChunk = kSgdWarps * kWarpEntries;  // entries per CTA
@@ -197,7 +197,7 @@ __device__ __forceinline__ void scan_step(bool hasb, const Comp<NV> &head, const
 }
 
 // ------------------------------------------------------------------------------------------
-// sgd_chunk_kernel: one CTA (4 warps) per chunk of kChunk consecutive entries of one tile.
+// sgd_chunk_kernel: one CTA per chunk of kChunk consecutive entries of one tile (kSgdWarps warps; 1 today).
 //
 // A launch covers tiles with pairwise disjoint column blocks: the p tiles of one inner round
 // (sweep 0) or the p tiles of one row block (sweep 1).  A tile's entries are sorted by (column,
@@ -249,7 +249,7 @@ struct SgdChunkArgs {
 };
 
 template <int LG, int NV, bool WIDE>
-__global__ void __launch_bounds__(kSgdThreads, 4) sgd_chunk_kernel(const SgdChunkArgs a) {
+__global__ void __launch_bounds__(kSgdThreads, 16) sgd_chunk_kernel(const SgdChunkArgs a) {
     typedef SgdSmem<LG, NV> L;
     constexpr int GW = L::GW, KP4 = L::KP4, PASS = L::PASS, S = L::S;
     constexpr int PP = kWarpEntries / PASS;
@@ -283,20 +283,6 @@ __global__ void __launch_bounds__(kSgdThreads, 4) sgd_chunk_kernel(const SgdChun
     const int64_t t = cm.x;
     const int r = (int)(t % a.p), s = (int)(t / a.p);
     const int c = (r + s) % a.p;
-    if (tid == 0) {
-        int go = 1;
-        const volatile int *done = a.sync + 2 + c;
-        const volatile int *err = a.sync + 1;
-        for (int spin = 0; *done < cm.z; ++spin) {
-            if (*err != 0 || spin > kSgdSpinLimit) { go = 0; break; }
-            __nanosleep(100);
-        }
-        if (!go) atomicExch(a.sync + 1, 1);
-        __threadfence();
-        s_go = go;
-    }
-    __syncthreads();
-    if (!s_go) return;
     const bool tail_mode = a.sweep == 1 && r > c;
     const int64_t tb = a.tile_ptr[t], te = a.tile_ptr[t + 1];
     const int64_t cb = tb + (int64_t)cm.y * kChunk;
@@ -368,6 +354,21 @@ __global__ void __launch_bounds__(kSgdThreads, 4) sgd_chunk_kernel(const SgdChun
     if (PP > 1) fetch_ent(1, ent1, xw1);
     fetch_g(0, ent0, g0);
 
+    // the first fetches are under way; now make sure the earlier tiles of this column block are done
+    if (tid == 0) {
+        int go = 1;
+        const volatile int *done = a.sync + 2 + c;
+        const volatile int *err = a.sync + 1;
+        for (int spin = 0; *done < cm.z; ++spin) {
+            if (*err != 0 || spin > kSgdSpinLimit) { go = 0; break; }
+            __nanosleep(100);
+        }
+        if (!go) atomicExch(a.sync + 1, 1);
+        __threadfence();
+        s_go = go;
+    }
+    __syncthreads();
+    if (!s_go) return;
     for (int pp = 0; pp < PP; ++pp) {
         if (pp * PASS >= wlen) break;
         const int cnt = (wlen - pp * PASS) < PASS ? (wlen - pp * PASS) : PASS;
