@@ -26,13 +26,13 @@ namespace dsf {
 
 constexpr int kSgdThreads = 32;   // one warp per CTA: a finished warp frees its registers and shared memory at once
 constexpr int kSgdWarps = kSgdThreads / 32;
-constexpr int kWarpEntries = 1024;                // entries per warp
+constexpr int kWarpEntries = 512;                 // entries per warp
 constexpr int kChunk = kSgdWarps * kWarpEntries;  // entries per CTA
 constexpr int kSgdSpinLimit = 1 << 22;            // polls (about 100 ns each) before a dependency wait gives up
 
-// entries of one warp pass: sized so that the gathered rows of A fill about 8 KB of shared memory
+// entries of one warp pass: sized so that the gathered rows of A fill about 4 KB of shared memory
 __host__ __device__ constexpr int sgd_pass_len(int LG, int NV) {
-    return 512 / (LG * NV) > 256 ? 256 : (512 / (LG * NV) < 8 ? 8 : 512 / (LG * NV));
+    return 256 / (LG * NV) > 256 ? 256 : (256 / (LG * NV) < 8 ? 8 : 256 / (LG * NV));
 }
 // floats per chunk record in global scratch: 3 header float4s + head offsets + tail offsets
 __host__ __device__ constexpr int chunk_record_floats(int Kp) { return 12 + 2 * Kp; }
@@ -249,7 +249,7 @@ struct SgdChunkArgs {
 };
 
 template <int LG, int NV, bool WIDE>
-__global__ void __launch_bounds__(kSgdThreads, 16) sgd_chunk_kernel(const SgdChunkArgs a) {
+__global__ void __launch_bounds__(kSgdThreads, 24) sgd_chunk_kernel(const SgdChunkArgs a) {
     typedef SgdSmem<LG, NV> L;
     constexpr int GW = L::GW, KP4 = L::KP4, PASS = L::PASS, S = L::S;
     constexpr int PP = kWarpEntries / PASS;
