@@ -39,7 +39,7 @@ struct dsfacto {
 
     std::vector<int64_t> row_start;  // p+1
     std::vector<int32_t> col_start;  // p+1
-    std::vector<int64_t> tile_ptr;   // p*p+1
+    std::vector<int64_t> tile_ptr;   // p*p+1, tiles in DEVICE order ("slots": the order the sweep visits them)
 
     // device
     float *d_w = nullptr, *d_V = nullptr, *d_A = nullptr, *d_G = nullptr, *d_y = nullptr, *d_val = nullptr, *d_xw = nullptr;
@@ -124,6 +124,37 @@ inline int bits_for(int64_t count) {  // bits needed for values in [0, count)
     return b;
 }
 
+// Device order of the tiles = the order in which the SGD sweep visits them, so that the entries a
+// launch works on at any moment are close together in memory.  Slot L*p + k holds, for the row-block
+// sweep, tile (r = p-1-L, c = k); for the round sweep, tile (r = k, round s = L), which is also the
+// canonical tile number s*p + r.
+inline int64_t tile_slot(const dsfacto *h, int64_t r, int64_t c) {
+    const int64_t p = h->p;
+    if (h->sweep == 1) return (p - 1 - r) * p + c;
+    int64_t s = c - r;
+    if (s < 0) s += p;
+    return s * p + r;
+}
+inline void slot_tile(const dsfacto *h, int64_t slot, int64_t &r, int64_t &c) {
+    const int64_t p = h->p;
+    if (h->sweep == 1) { r = p - 1 - slot / p; c = slot % p; }
+    else { r = slot % p; c = (r + slot / p) % p; }
+}
+// canonical tile_ptr (tile number s*p + r, s = (c - r) mod p) from the device-order one
+std::vector<int64_t> canonical_tile_ptr(const dsfacto *h) {
+    const int64_t p = h->p, nt = p * p;
+    std::vector<int64_t> cp((size_t)nt + 1, 0);
+    for (int64_t slot = 0; slot < nt; ++slot) {
+        int64_t r, c;
+        slot_tile(h, slot, r, c);
+        int64_t sr = c - r;
+        if (sr < 0) sr += p;
+        cp[(size_t)(sr * p + r) + 1] = h->tile_ptr[slot + 1] - h->tile_ptr[slot];
+    }
+    for (int64_t t = 0; t < nt; ++t) cp[t + 1] += cp[t];
+    return cp;
+}
+
 // partition: row block r = rows [ceil(r n / p), ceil((r+1) n / p)), i.e. floor(i p / n) = r; same for
 // columns.  Also chooses the packed (32-bit key) or wide entry layout.
 int setup_partition(dsfacto *h) {
@@ -150,20 +181,25 @@ int setup_partition(dsfacto *h) {
 }
 
 // canonical (global row, global column, value) lists from the packed device layout
-void unpack_tiles(const dsfacto *h, const uint2 *ent, const float *xw, int32_t *rows, int32_t *cols, float *vals) {
+void unpack_tiles(const dsfacto *h, const std::vector<int64_t> &canon_ptr, const uint2 *ent, const float *xw,
+                  int32_t *rows, int32_t *cols, float *vals) {
     const int64_t nt = (int64_t)h->p * h->p;
     const uint32_t jmask = h->jbits >= 32 ? 0xFFFFFFFFu : ((1u << h->jbits) - 1u);
 #pragma omp parallel for schedule(dynamic, 8)
-    for (int64_t t = 0; t < nt; ++t) {
-        const int64_t s = t / h->p, r = t % h->p, c = (r + s) % h->p;
-        for (int64_t q = h->tile_ptr[t]; q < h->tile_ptr[t + 1]; ++q) {
+    for (int64_t slot = 0; slot < nt; ++slot) {
+        int64_t r, c;
+        slot_tile(h, slot, r, c);
+        int64_t sr = c - r;
+        if (sr < 0) sr += h->p;
+        const int64_t shift = canon_ptr[(size_t)(sr * h->p + r)] - h->tile_ptr[slot];
+        for (int64_t q = h->tile_ptr[slot]; q < h->tile_ptr[slot + 1]; ++q) {
             uint32_t il, jl;
             float x;
             if (h->wide) { il = ent[q].x; jl = ent[q].y; x = xw[q]; }
             else { il = ent[q].x >> h->jbits; jl = ent[q].x & jmask; std::memcpy(&x, &ent[q].y, 4); }
-            if (rows) rows[q] = (int32_t)(h->row_start[r] + il);
-            if (cols) cols[q] = (int32_t)(h->col_start[c] + jl);
-            if (vals) vals[q] = x;
+            if (rows) rows[q + shift] = (int32_t)(h->row_start[r] + il);
+            if (cols) cols[q + shift] = (int32_t)(h->col_start[c] + jl);
+            if (vals) vals[q + shift] = x;
         }
     }
 }
@@ -233,11 +269,9 @@ int build_sgd_plan(dsfacto *h) {
         map.reserve((size_t)(h->nnz / kChunk + p * p / 4 + 16));
         for (int64_t L = 0; L < p; ++L) {
             for (int64_t k = 0; k < p; ++k) {
-                int64_t r, s;
-                if (h->sweep == 1) { r = p - 1 - L; s = ((k - r) % p + p) % p; }   // column block c = k
-                else { s = L; r = k; }
-                const int64_t t = s * p + r;
-                const int64_t c = (r + s) % p;
+                const int64_t t = L * p + k;   // slot
+                int64_t r, c;
+                slot_tile(h, t, r, c);
                 const int64_t cnt = h->tile_ptr[t + 1] - h->tile_ptr[t];
                 const int64_t nch = (cnt + kChunk - 1) / kChunk;
                 for (int64_t ci = 0; ci < nch; ++ci) map.push_back(make_int4((int)t, (int)ci, seen[c], 0));
@@ -251,7 +285,7 @@ int build_sgd_plan(dsfacto *h) {
     int rc;
     if ((rc = dev_alloc(h, &h->d_chunk_map, map.size())) ||
         (rc = dev_alloc(h, &h->d_records, map.size() * chunk_record_floats(h->Kp))) ||
-        (rc = dev_alloc(h, &h->d_tile_count, (size_t)(p * p))) || (rc = dev_alloc(h, &h->d_sync, (size_t)p + 2)))
+        (rc = dev_alloc(h, &h->d_tile_count, (size_t)(p * p))) || (rc = dev_alloc(h, &h->d_sync, sync_words((int)p))))
         return rc;
     CU_TRY(h, cudaMemsetAsync(h->d_tile_count, 0, sizeof(int) * (size_t)(p * p), h->stream));
     if (!map.empty())
@@ -270,7 +304,7 @@ void run_sgd_phase(dsfacto *h) {
     a.h = h->h; a.lambda_w = h->lambda_w; a.lambda_v = h->lambda_v;
     // One launch for the whole sweep: chunks are taken in sweep order (row block by row block, or round
     // by round) and a tile waits only for the earlier tiles of its own column block.
-    cudaMemsetAsync(h->d_sync, 0, sizeof(int) * ((size_t)h->p + 2), h->stream);
+    cudaMemsetAsync(h->d_sync, 0, sizeof(int) * sync_words(h->p), h->stream);
     a.chunk_map = h->d_chunk_map;
     a.sync = h->d_sync;
     if (h->total_chunks > 0) {
@@ -403,9 +437,7 @@ int bucket_tiles(dsfacto *h, const int64_t *indptr, const int32_t *indices, cons
         for (int64_t i = rs[k]; i < rs[k + 1]; ++i) {
             while (i >= h->row_start[r + 1]) ++r;
             for (int64_t e = indptr[i]; e < indptr[i + 1]; ++e) {
-                int64_t s = cb[indices[e]] - r;
-                if (s < 0) s += p;
-                cnt[s * p + r] += 1;
+                cnt[tile_slot(h, r, cb[indices[e]])] += 1;
             }
         }
     }
@@ -437,9 +469,7 @@ int bucket_tiles(dsfacto *h, const int64_t *indptr, const int32_t *indices, cons
             for (int64_t e = indptr[i]; e < indptr[i + 1]; ++e) {
                 const int32_t j = indices[e];
                 const int32_t c = cb[j];
-                int64_t s = c - r;
-                if (s < 0) s += p;
-                const int64_t at = off[s * p + r]++;
+                const int64_t at = off[tile_slot(h, r, c)]++;
                 const uint32_t jl = (uint32_t)(j - h->col_start[c]);
                 if (wide) { tmp_e[at] = make_uint2(il, jl); tmp_x[at] = values[e]; }
                 else {
@@ -459,8 +489,9 @@ int bucket_tiles(dsfacto *h, const int64_t *indptr, const int32_t *indices, cons
         for (int64_t t = 0; t < nt; ++t) {
             const int64_t b = h->tile_ptr[t], e = h->tile_ptr[t + 1];
             if (b == e) continue;
-            const int64_t s = t / p, r = t % p;
-            const int64_t c = (r + s) % p;
+            int64_t r, c;
+            slot_tile(h, t, r, c);
+            (void)r;
             const int64_t width = h->col_start[c + 1] - h->col_start[c];
             hist.assign((size_t)width + 1, 0);
             for (int64_t q = b; q < e; ++q) {
@@ -657,7 +688,7 @@ int dsfacto_epoch(dsfacto_t *h) {
     int rc = run_refresh(h, true);
     if (rc) return rc;
     int sgd_error = 0;  // set by the SGD kernel if a dependency wait ran out (never seen; the state is then unusable)
-    CU_TRY(h, cudaMemcpy(&sgd_error, h->d_sync + 1, sizeof(int), cudaMemcpyDeviceToHost));
+    CU_TRY(h, cudaMemcpy(&sgd_error, h->d_sync + kSyncError, sizeof(int), cudaMemcpyDeviceToHost));
     if (sgd_error) { h->err = "stratum SGD: a wait for an earlier tile of the same column block timed out"; return DSFACTO_ERR_CUDA; }
     float t01 = 0, t12 = 0, t23 = 0;
     cudaEventElapsedTime(&t01, h->ev[0], h->ev[1]);
@@ -724,7 +755,8 @@ int dsfacto_get_tiles(dsfacto_t *h, int64_t *tile_ptr, int32_t *rows, int32_t *c
     if (!h) return DSFACTO_ERR_INVALID_ARG;
     if (!h->loaded) return DSFACTO_ERR_NO_DATA;
     const int64_t nt = (int64_t)h->p * h->p;
-    if (tile_ptr) std::memcpy(tile_ptr, h->tile_ptr.data(), sizeof(int64_t) * ((size_t)nt + 1));
+    const std::vector<int64_t> canon = canonical_tile_ptr(h);
+    if (tile_ptr) std::memcpy(tile_ptr, canon.data(), sizeof(int64_t) * ((size_t)nt + 1));
     if (!rows && !cols && !vals) return DSFACTO_OK;
     HostBuf<uint2> ent;
     HostBuf<float> xw;
@@ -734,7 +766,7 @@ int dsfacto_get_tiles(dsfacto_t *h, int64_t *tile_ptr, int32_t *rows, int32_t *c
         if (h->wide) CU_TRY(h, cudaMemcpyAsync(xw.data(), h->d_xw, sizeof(float) * (size_t)h->nnz, cudaMemcpyDeviceToHost, h->stream));
         CU_TRY(h, cudaStreamSynchronize(h->stream));
     }
-    unpack_tiles(h, ent.data(), xw.data(), rows, cols, vals);
+    unpack_tiles(h, canon, ent.data(), xw.data(), rows, cols, vals);
     return DSFACTO_OK;
 }
 
@@ -747,12 +779,14 @@ int dsfacto_bucket_host(int64_t n, int32_t d, int32_t p, const int64_t *indptr, 
     if (rc) return rc;
     dsfacto tmp;
     tmp.n = n; tmp.d = d; tmp.p = p;
+    tmp.sweep = 0;
     if ((rc = setup_partition(&tmp))) return rc;
     HostBuf<uint2> ent;
     HostBuf<float> xw;
     if ((rc = bucket_tiles(&tmp, indptr, indices, values, ent, xw))) return rc;
-    std::memcpy(tile_ptr, tmp.tile_ptr.data(), sizeof(int64_t) * tmp.tile_ptr.size());
-    unpack_tiles(&tmp, ent.data(), xw.data(), rows, cols, vals);
+    const std::vector<int64_t> canon = canonical_tile_ptr(&tmp);
+    std::memcpy(tile_ptr, canon.data(), sizeof(int64_t) * canon.size());
+    unpack_tiles(&tmp, canon, ent.data(), xw.data(), rows, cols, vals);
     return DSFACTO_OK;
 }
 

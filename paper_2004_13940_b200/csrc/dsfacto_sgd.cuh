@@ -29,6 +29,13 @@ constexpr int kSgdWarps = kSgdThreads / 32;
 constexpr int kWarpEntries = 512;                 // entries per warp
 constexpr int kChunk = kSgdWarps * kWarpEntries;  // entries per CTA
 constexpr int kSgdSpinLimit = 1 << 22;            // polls (about 100 ns each) before a dependency wait gives up
+// Words of the launch's synchronisation array.  The ticket counter takes one atomic per CTA and the
+// progress counters are polled by waiting CTAs, so every word sits in a 128-byte line of its own.
+constexpr int kSyncStride = 32;                   // ints between two words
+constexpr int kSyncTicket = 0;                    // next chunk to hand out
+constexpr int kSyncError = kSyncStride;           // set when a dependency wait ran out
+__host__ __device__ constexpr size_t sync_done(int c) { return (size_t)(2 + c) * kSyncStride; }  // finished tiles of column block c
+__host__ __device__ constexpr size_t sync_words(int p) { return (size_t)(2 + p) * kSyncStride; }
 
 // entries of one warp pass: sized so that the gathered rows of A fill about 4 KB of shared memory
 __host__ __device__ constexpr int sgd_pass_len(int LG, int NV) {
@@ -225,7 +232,7 @@ __device__ __forceinline__ void scan_step(bool hasb, const Comp<NV> &head, const
 // from L2 after first touch.
 // ------------------------------------------------------------------------------------------
 struct SgdChunkArgs {
-    const int64_t *tile_ptr;   // p*p+1, tile t = s*p + r
+    const int64_t *tile_ptr;   // p*p+1, tiles in sweep order (slots)
     const uint2 *ent;          // packed: {(i_local << jbits) | j_local, bits of x}; wide: {i_local, j_local}
     const float *xw;           // wide layout only: x per entry
     const int64_t *row_start;  // p+1
@@ -238,12 +245,12 @@ struct SgdChunkArgs {
     float *Tw;                 // d        u-part of the w offset of T_j      (sweep 1)
     float *Tb;                 // d * Kp   u-part of the v offset of T_j      (sweep 1)
     float4 *TS;                // d        {D, Dw, -, -} of T_j               (sweep 1)
-    const int4 *chunk_map;     // per chunk, in sweep order: {tile t, chunk index inside the tile, number
+    const int4 *chunk_map;     // per chunk, in sweep order: {tile slot, chunk index inside the tile, number
                                // of earlier non-empty tiles of the same column block, -}
     float *records;            // chunk_record_floats(Kp) floats per chunk
     int *tile_count;           // p*p, all zero between launches
-    int *sync;                 // [0] ticket counter, [1] error flag, [2 + c] finished tiles of column block c;
-                               // all zero at launch
+    int *sync;                 // sync_words(p) ints: ticket counter, error flag, finished tiles per column
+                               // block; all zero at launch
     int p, jbits, sweep;
     float h, lambda_w, lambda_v;
 };
@@ -276,13 +283,14 @@ __global__ void __launch_bounds__(kSgdThreads, 24) sgd_chunk_kernel(const SgdChu
     // the same column block can therefore not deadlock.  The wait is bounded all the same; on a
     // time-out the error flag makes every CTA leave and the host reports the failure.
     __shared__ int s_ticket, s_go;
-    if (tid == 0) s_ticket = atomicAdd(a.sync, 1);
+    if (tid == 0) s_ticket = atomicAdd(a.sync + kSyncTicket, 1);
     __syncthreads();
     const int chunk = s_ticket;
     const int4 cm = a.chunk_map[chunk];
-    const int64_t t = cm.x;
-    const int r = (int)(t % a.p), s = (int)(t / a.p);
-    const int c = (r + s) % a.p;
+    const int64_t t = cm.x;  // tile slot: position of the tile in sweep order (the device order of tiles)
+    int r, c;
+    if (a.sweep == 1) { r = a.p - 1 - (int)(t / a.p); c = (int)(t % a.p); }
+    else { r = (int)(t % a.p); c = (r + (int)(t / a.p)) % a.p; }
     const bool tail_mode = a.sweep == 1 && r > c;
     const int64_t tb = a.tile_ptr[t], te = a.tile_ptr[t + 1];
     const int64_t cb = tb + (int64_t)cm.y * kChunk;
@@ -357,13 +365,13 @@ __global__ void __launch_bounds__(kSgdThreads, 24) sgd_chunk_kernel(const SgdChu
     // the first fetches are under way; now make sure the earlier tiles of this column block are done
     if (tid == 0) {
         int go = 1;
-        const volatile int *done = a.sync + 2 + c;
-        const volatile int *err = a.sync + 1;
+        const volatile int *done = a.sync + sync_done(c);
+        const volatile int *err = a.sync + kSyncError;
         for (int spin = 0; *done < cm.z; ++spin) {
             if (*err != 0 || spin > kSgdSpinLimit) { go = 0; break; }
             __nanosleep(100);
         }
-        if (!go) atomicExch(a.sync + 1, 1);
+        if (!go) atomicExch(a.sync + kSyncError, 1);
         __threadfence();
         s_go = go;
     }
@@ -524,7 +532,9 @@ __global__ void __launch_bounds__(kSgdThreads, 24) sgd_chunk_kernel(const SgdChu
         comp_store<LG, NV>(s_wpiece + (warp * 2 + 1) * (KP4 + 1), wcarry, last_col, l);
         if (l == 0) s_wflag[warp] = wflag ? 1 : 0;
     }
-    __threadfence();  // this warp's state updates are ordered before the tile's completion signal below
+    // with several warps, each orders its own state updates before the tile's completion signal below
+    // (warp 0 fences again before it signals)
+    if (NW > 1) __threadfence();
     __syncthreads();
     if (warp != 0) return;
 
@@ -566,7 +576,7 @@ __global__ void __launch_bounds__(kSgdThreads, 24) sgd_chunk_kernel(const SgdChu
         if (g == 0) apply_fetch(ctailcol, ccarry);
         __threadfence();
         __syncwarp();
-        if (lane == 0) atomicAdd(a.sync + 2 + c, 1);  // this tile of column block c is done
+        if (lane == 0) atomicAdd(a.sync + sync_done(c), 1);  // this tile of column block c is done
         return;
     }
     {
@@ -597,31 +607,48 @@ __global__ void __launch_bounds__(kSgdThreads, 24) sgd_chunk_kernel(const SgdChu
     C tcarry;
     comp_identity(tcarry);
     bool tflag = false;
-    for (int k0 = 0; k0 < nchunks; k0 += GW) {
-        const int k = k0 + g;
-        bool hasb = false;
-        uint32_t headcol = kNoCol;
-        C head, cur, closing;
-        comp_identity(head);
-        comp_identity(cur);
+    // The next tile of this column block waits for this loop, so the records (and the scale pair of each
+    // record's head column) of step k0 + GW are fetched before step k0 is scanned: one memory latency
+    // for the whole loop instead of two per step.
+    struct Rec {
+        bool hasb;
+        uint32_t headcol;
+        C head, cur;
+        float4 sc;
+    };
+    auto load_rec = [&](int k, Rec &x) {
+        x.hasb = false;
+        x.headcol = kNoCol;
+        comp_identity(x.head);
+        comp_identity(x.cur);
+        x.sc = make_float4(0.f, 0.f, 0.f, 0.f);
         if (k < nchunks) {
             const float4 *rec4 = base4 + (size_t)k * REC4;
             const float4 hh = __ldcg(rec4 + 0);
             const float4 th = __ldcg(rec4 + 1);
-            hasb = __float_as_uint(__ldcg(rec4 + 2).x) != 0u;
-            head.D = hh.x; head.Dw = hh.y; head.Bw = hh.z;
-            headcol = __float_as_uint(hh.w);
-            cur.D = th.x; cur.Dw = th.y; cur.Bw = th.z;
+            x.hasb = __float_as_uint(__ldcg(rec4 + 2).x) != 0u;
+            x.head.D = hh.x; x.head.Dw = hh.y; x.head.Bw = hh.z;
+            x.headcol = __float_as_uint(hh.w);
+            x.cur.D = th.x; x.cur.Dw = th.y; x.cur.Bw = th.z;
 #pragma unroll
             for (int v = 0; v < NV; ++v) {
-                head.B[v] = __ldcg(rec4 + 3 + v * LG + l);
-                cur.B[v] = __ldcg(rec4 + 3 + KP4 + v * LG + l);
+                x.head.B[v] = __ldcg(rec4 + 3 + v * LG + l);
+                x.cur.B[v] = __ldcg(rec4 + 3 + KP4 + v * LG + l);
             }
+            // no chunk of this tile applies to a head column: its run is still open until this loop
+            if (x.hasb && x.headcol != kNoCol) x.sc = __ldcg(Sc + x.headcol);
         }
+    };
+    Rec nxt;
+    load_rec(g, nxt);
+    for (int k0 = 0; k0 < nchunks; k0 += GW) {
+        const Rec now = nxt;
+        if (k0 + GW < nchunks) load_rec(k0 + GW + g, nxt);
+        C closing;
         bool outer;
-        scan_step<LG, NV>(hasb, head, cur, tcarry, tflag, closing, outer);
+        scan_step<LG, NV>(now.hasb, now.head, now.cur, tcarry, tflag, closing, outer);
         // the first boundary of a tile is its start, whose head column is kNoCol: nothing to apply
-        if (hasb) apply_fetch(headcol, closing);
+        if (now.hasb && now.headcol != kNoCol) apply(now.headcol, closing, now.sc);
     }
     const uint32_t ttailcol = __float_as_uint(__ldcg(base4 + (size_t)(nchunks - 1) * REC4 + 1).w);
     if (g == 0) apply_fetch(ttailcol, tcarry);  // the end of the tile closes the last run
@@ -629,7 +656,7 @@ __global__ void __launch_bounds__(kSgdThreads, 24) sgd_chunk_kernel(const SgdChu
     __syncwarp();
     if (lane == 0) {
         a.tile_count[t] = 0;
-        atomicAdd(a.sync + 2 + c, 1);  // this tile of column block c is done
+        atomicAdd(a.sync + sync_done(c), 1);  // this tile of column block c is done
     }
 }
 
