@@ -112,6 +112,22 @@ __device__ __forceinline__ Comp<NV> comp_shfl_up(const Comp<NV> &c, int delta) {
 }
 
 template <int NV>
+__device__ __forceinline__ Comp<NV> comp_shfl_down(const Comp<NV> &c, int delta) {
+    Comp<NV> r;
+    r.D = __shfl_down_sync(0xFFFFFFFFu, c.D, delta);
+    r.Dw = __shfl_down_sync(0xFFFFFFFFu, c.Dw, delta);
+    r.Bw = __shfl_down_sync(0xFFFFFFFFu, c.Bw, delta);
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+        r.B[v].x = __shfl_down_sync(0xFFFFFFFFu, c.B[v].x, delta);
+        r.B[v].y = __shfl_down_sync(0xFFFFFFFFu, c.B[v].y, delta);
+        r.B[v].z = __shfl_down_sync(0xFFFFFFFFu, c.B[v].z, delta);
+        r.B[v].w = __shfl_down_sync(0xFFFFFFFFu, c.B[v].w, delta);
+    }
+    return r;
+}
+
+template <int NV>
 __device__ __forceinline__ Comp<NV> comp_shfl(const Comp<NV> &c, int src) {
     Comp<NV> r;
     r.D = __shfl_sync(0xFFFFFFFFu, c.D, src);
@@ -153,6 +169,13 @@ __device__ __forceinline__ void red_add4(float4 *p, float x, float y, float z, f
 }
 __device__ __forceinline__ void red_add1(float *p, float x) {
     asm volatile("red.global.add.f32 [%0], %1;" ::"l"(p), "f"(x) : "memory");
+}
+// 1 / x by the special-function unit alone (within one unit in the last place): it scales an increment,
+// so a correctly rounded reciprocal would buy nothing but instructions
+__device__ __forceinline__ float rcp_fast(float x) {
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
 }
 __device__ __forceinline__ void cp_async_wait_all() {
     asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;\n" ::: "memory");
@@ -260,7 +283,8 @@ __global__ void __launch_bounds__(kSgdThreads, 24) sgd_chunk_kernel(const SgdChu
     typedef SgdSmem<LG, NV> L;
     constexpr int GW = L::GW, KP4 = L::KP4, PASS = L::PASS, S = L::S;
     constexpr int PP = kWarpEntries / PASS;
-    constexpr int EPL = (PASS + 31) / 32;  // entries staged per lane and pass
+    constexpr int EPL = (S + LG - 1) / LG;  // entries a lane holds per pass: lane l of group g holds the
+                                            // entries g*S + l*EPL + q of the pass, q < EPL (those below S)
     constexpr int NW = kSgdWarps;
     constexpr int REC4 = chunk_record_floats(4 * KP4) / 4;
     static_assert(PASS * PP == kWarpEntries && S * GW == PASS, "a warp's entries must be whole passes");
@@ -315,14 +339,14 @@ __global__ void __launch_bounds__(kSgdThreads, 24) sgd_chunk_kernel(const SgdChu
     // column state <- run o column state, given the column's scale pair (lanes of one group)
     auto apply = [&](uint32_t jl, const C &x, float4 sc) {
         const float sg = fmaf(sc.x, x.D, sc.x + x.D);
-        const float inv = __frcp_rn(1.0f + sg);
+        const float inv = rcp_fast(1.0f + sg);
 #pragma unroll
         for (int v = 0; v < NV; ++v)
             red_add4(U4 + (size_t)jl * KP4 + v * LG + l, x.B[v].x * inv, x.B[v].y * inv, x.B[v].z * inv,
                      x.B[v].w * inv);
         if (l == 0) {
             const float sgw = fmaf(sc.y, x.Dw, sc.y + x.Dw);
-            red_add1(uw + jl, x.Bw * __frcp_rn(1.0f + sgw));
+            red_add1(uw + jl, x.Bw * rcp_fast(1.0f + sgw));
             Sc[jl] = make_float4(sg, sgw, 0.f, 0.f);
         }
     };
@@ -341,11 +365,13 @@ __global__ void __launch_bounds__(kSgdThreads, 24) sgd_chunk_kernel(const SgdChu
     // entry records are fetched two passes ahead and G one pass ahead, into registers
     uint2 ent0[EPL], ent1[EPL];
     float xw0[EPL], xw1[EPL], g0[EPL];
+    const int slot0 = l * EPL;          // this lane's first entry inside its group's S entries
+    const int at0 = g * S + slot0;      // ... and inside the pass
     auto fetch_ent = [&](int pp, uint2 (&e)[EPL], float (&xv)[EPL]) {
 #pragma unroll
         for (int q = 0; q < EPL; ++q) {
-            const int at = pp * PASS + lane + 32 * q;
-            if ((PASS >= 32 || lane < PASS) && at < wlen) {
+            const int at = pp * PASS + at0 + q;
+            if (slot0 + q < S && at < wlen) {
                 e[q] = entw[at];
                 if (WIDE) xv[q] = xww[at];
             }
@@ -354,8 +380,8 @@ __global__ void __launch_bounds__(kSgdThreads, 24) sgd_chunk_kernel(const SgdChu
     auto fetch_g = [&](int pp, const uint2 (&e)[EPL], float (&gv)[EPL]) {
 #pragma unroll
         for (int q = 0; q < EPL; ++q) {
-            const int at = pp * PASS + lane + 32 * q;
-            if ((PASS >= 32 || lane < PASS) && at < wlen) gv[q] = __ldg(Gr + (WIDE ? e[q].x : (e[q].x >> a.jbits)));
+            const int at = pp * PASS + at0 + q;
+            if (slot0 + q < S && at < wlen) gv[q] = __ldg(Gr + (WIDE ? e[q].x : (e[q].x >> a.jbits)));
         }
     };
     fetch_ent(0, ent0, xw0);
@@ -391,20 +417,34 @@ __global__ void __launch_bounds__(kSgdThreads, 24) sgd_chunk_kernel(const SgdChu
         uint32_t after = kNoCol;
         const bool after_known = (pp + 1 < PP) && ((pp + 1) * PASS < wlen);
         // 1. items of this pass from the prefetched registers
-        uint32_t jq[EPL];
+        uint32_t jq[EPL], ilq[EPL];
+        float eq[EPL], bq[EPL];
+        bool cont = true;  // every entry this lane holds continues the run that is open at the pass start
 #pragma unroll
         for (int q = 0; q < EPL; ++q) {
-            const int at = lane + 32 * q;
             jq[q] = kNoCol;
-            if (at < cnt) {
-                uint32_t il;
+            ilq[q] = 0u;
+            eq[q] = 0.f;
+            bq[q] = 0.f;
+            if (slot0 + q < S && at0 + q < cnt) {
                 float x;
-                if (WIDE) { il = ent0[q].x; jq[q] = ent0[q].y; x = xw0[q]; }
-                else { il = ent0[q].x >> a.jbits; jq[q] = ent0[q].x & jmask; x = __uint_as_float(ent0[q].y); }
+                if (WIDE) { ilq[q] = ent0[q].x; jq[q] = ent0[q].y; x = xw0[q]; }
+                else { ilq[q] = ent0[q].x >> a.jbits; jq[q] = ent0[q].x & jmask; x = __uint_as_float(ent0[q].y); }
                 const float gx = g0[q] * x;
-                sw[L::ITEMS + (at / S) * L::ITEM_STRIDE + (at % S)] =
-                    make_float4(a.h * (a.lambda_v - gx * x), -a.h * gx, __uint_as_float(il), __uint_as_float(jq[q]));
+                eq[q] = a.h * (a.lambda_v - gx * x);
+                bq[q] = -a.h * gx;
+                cont = cont && jq[q] == before;
             }
+        }
+        // A full pass inside one run (about two thirds of the passes on click-log data, where a few
+        // columns hold most entries) has no boundary: nothing is applied and nothing needs the staging
+        // in shared memory.  It takes the short way below.
+        const bool one_run = cnt == PASS && before != kNoCol && __all_sync(0xFFFFFFFFu, cont);
+        if (!one_run) {
+#pragma unroll
+            for (int q = 0; q < EPL; ++q)
+                if (slot0 + q < S && at0 + q < cnt)
+                    s_item[slot0 + q] = make_float4(eq[q], bq[q], __uint_as_float(ilq[q]), __uint_as_float(jq[q]));
         }
         // rotate the prefetch registers and start the next fetches
 #pragma unroll
@@ -412,18 +452,68 @@ __global__ void __launch_bounds__(kSgdThreads, 24) sgd_chunk_kernel(const SgdChu
         if (after_known) after = __shfl_sync(0xFFFFFFFFu, WIDE ? ent0[0].y : (ent0[0].x & jmask), 0);
         if (pp + 1 < PP) fetch_g(pp + 1, ent0, g0);
         if (pp + 2 < PP) fetch_ent(pp + 2, ent1, xw1);
+        if (one_run) {
+            // Each lane group composes its S entries, rows a_i straight from global memory to registers
+            // (entry u of the group sits in lane u / EPL of the group), then the groups' composites are
+            // joined in order and appended to the open run.
+            constexpr int UB = (S * NV <= 8) ? S : (8 / NV < 1 ? 1 : 8 / NV);  // rows requested before the first is used
+            C cur;
+            comp_identity(cur);
+#pragma unroll
+            for (int u0 = 0; u0 < S; u0 += UB) {
+                float4 av[UB][NV];
+                float eu[UB], bu[UB];
+#pragma unroll
+                for (int u = 0; u < UB; ++u) {
+                    const int src = (u0 + u) / EPL, reg = (u0 + u) % EPL;
+                    const uint32_t il = __shfl_sync(0xFFFFFFFFu, ilq[reg], src, LG);
+                    eu[u] = __shfl_sync(0xFFFFFFFFu, eq[reg], src, LG);
+                    bu[u] = __shfl_sync(0xFFFFFFFFu, bq[reg], src, LG);
+#pragma unroll
+                    for (int v = 0; v < NV; ++v) av[u][v] = __ldcg(A4 + (size_t)il * KP4 + v * LG + l);
+                }
+#pragma unroll
+                for (int u = 0; u < UB; ++u) {
+                    const float e = eu[u], b = bu[u];
+                    cur.D = fmaf(-e, cur.D, cur.D - e);
+                    cur.Dw = fmaf(-ew, cur.Dw, cur.Dw - ew);
+                    cur.Bw = fmaf(-ew, cur.Bw, cur.Bw + b);
+#pragma unroll
+                    for (int v = 0; v < NV; ++v) {
+                        cur.B[v].x = fmaf(b, av[u][v].x, fmaf(-e, cur.B[v].x, cur.B[v].x));
+                        cur.B[v].y = fmaf(b, av[u][v].y, fmaf(-e, cur.B[v].y, cur.B[v].y));
+                        cur.B[v].z = fmaf(b, av[u][v].z, fmaf(-e, cur.B[v].z, cur.B[v].z));
+                        cur.B[v].w = fmaf(b, av[u][v].w, fmaf(-e, cur.B[v].w, cur.B[v].w));
+                    }
+                }
+            }
+            if (GW > 1) {
+#pragma unroll
+                for (int delta = 1; delta < GW; delta <<= 1) {
+                    const C o = comp_shfl_down<NV>(cur, delta * LG);
+                    if ((g & (2 * delta - 1)) == 0) cur = compose<NV>(cur, o);
+                }
+                cur = comp_shfl<NV>(cur, l);  // group 0 holds the whole pass
+            }
+            wcarry = compose<NV>(wcarry, cur);
+            last_col = before;
+            continue;
+        }
         //    scale pairs of the columns whose runs end in this pass (an entry ends a run when the
         //    next entry has another column)
+        {
+            // the entry after this lane's last one is held by the next lane that holds entries
+            const int next_lane = (slot0 + EPL < S) ? lane + 1 : (g + 1) * LG;
+            const uint32_t first_of_next = __shfl_sync(0xFFFFFFFFu, jq[0], next_lane & 31);
 #pragma unroll
-        for (int q = 0; q < EPL; ++q) {
-            const int at = lane + 32 * q;
-            uint32_t nextcol = __shfl_down_sync(0xFFFFFFFFu, jq[q], 1);
-            const uint32_t wrap = __shfl_sync(0xFFFFFFFFu, q + 1 < EPL ? jq[q + 1 < EPL ? q + 1 : q] : kNoCol, 0);
-            if (lane == 31) nextcol = wrap;
-            bool ends;
-            if (at + 1 < cnt) ends = nextcol != jq[q];
-            else ends = after_known && after != jq[q];
-            if (at < cnt && ends) cp_async16(s_scale_all + (at / S) * L::ITEM_STRIDE + (at % S), Sc + jq[q]);
+            for (int q = 0; q < EPL; ++q) {
+                const int at = at0 + q;
+                const uint32_t nextcol = (q + 1 < EPL && slot0 + q + 1 < S) ? jq[q + 1 < EPL ? q + 1 : q] : first_of_next;
+                bool ends;
+                if (at + 1 < cnt) ends = nextcol != jq[q];
+                else ends = after_known && after != jq[q];
+                if (slot0 + q < S && at < cnt && ends) cp_async16(s_scale + slot0 + q, Sc + jq[q]);
+            }
         }
         __syncwarp();
         // 2. gather the rows a_i of the pass
