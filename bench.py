@@ -15,6 +15,7 @@ replicas (the path is single-GPU; no collective on the data path)."""
 from __future__ import annotations
 
 import argparse
+import datetime
 import json
 import os
 import statistics
@@ -33,7 +34,7 @@ UNIT = "updates/s"
 ORACLE_SAMPLE_ROWS = 1_000_000
 # dram__bytes_read.sum + dram__bytes_write.sum of sgd_chunk_kernel per stored entry, from the ncu capture
 # summarised in profiles/ (None once the kernel has changed since the counters were taken)
-SGD_DRAM_BYTES_PER_ENTRY = 20.1
+SGD_DRAM_BYTES_PER_ENTRY = 19.8
 
 
 def peaks():
@@ -47,7 +48,7 @@ def peaks():
 
 
 class ClockSampler:
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
@@ -58,12 +59,15 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
-                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
 
-    def stop(self):
+    def stop(self, t_begin=None, t_end=None):
+        """Ends the sampling; keeps the samples taken between the two datetimes (the timed region).
+        The sampler is started before the warm-up so that it is already running when the region
+        begins; a region shorter than the sampling period keeps the samples closest to it."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -72,21 +76,29 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
             out = ""
-        sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        rows = []   # (time, sm MHz, max MHz, active reasons)
         for line in out.splitlines():
             parts = [x.strip() for x in line.split(",")]
-            if len(parts) < 7:
+            if len(parts) < 8:
                 continue
             try:
-                sm.append(float(parts[0])); mx.append(float(parts[1]))
+                when = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f")
+                rows.append((when, float(parts[1]), float(parts[2]),
+                             [nm for nm, val in zip(names, parts[4:8]) if val.lower().startswith("active")]))
             except ValueError:
                 continue
-            for nm, val in zip(names, parts[3:7]):
-                if val.lower().startswith("active"):
-                    reasons.add(nm)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+        window = "timed region"
+        inside = [r for r in rows if t_begin is None or (t_begin <= r[0] <= t_end)]
+        if not inside and rows:
+            mid = t_begin + (t_end - t_begin) / 2
+            inside = sorted(rows, key=lambda r: abs((r[0] - mid).total_seconds()))[:3]
+            window = "nearest samples (region shorter than the sampling period)"
+        sm = [r[1] for r in inside]
+        reasons = sorted({nm for r in inside for nm in r[3]})
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(r[2] for r in inside) if inside else None,
+                "samples": len(sm), "window": window, "reasons": reasons}
 
 
 def oracle_leg(wl_name: str, rows: int, min_seconds: float, max_epochs: int):
@@ -227,13 +239,14 @@ def run_ours(args):
 
     g, t_load = take_turns(rank, world, barrier, first_load)
 
-    for _ in range(args.warmup):
-        g.epoch()
     sampler = ClockSampler(local)
-    launches0 = g.launch_count()
-    barrier(); torch.cuda.synchronize()
     if rank == 0:
         sampler.start()
+    for _ in range(args.warmup):
+        g.epoch()
+    launches0 = g.launch_count()
+    barrier(); torch.cuda.synchronize()
+    t_begin = datetime.datetime.now()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     phase = np.zeros(4)
     ev0.record(stream)
@@ -242,7 +255,7 @@ def run_ours(args):
         phase += np.asarray(g.last_epoch_ms())
     ev1.record(stream)
     torch.cuda.synchronize(); barrier()
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.stop(t_begin, datetime.datetime.now()) if rank == 0 else None
     ms = ev0.elapsed_time(ev1)
     launches = g.launch_count() - launches0
     objective = g.objective()
@@ -316,7 +329,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C4")
