@@ -22,6 +22,9 @@
  *                        staleness ...": the auxiliaries are recomputed after the update step)
  *   oracle_epoch         one outer iteration t of Algorithm 1 in its synchronous (DSGD-style) form:
  *                        the update loop, then the recompute loop
+ *   oracle_evaluate      the quantities the experiments plot on held-out rows (Section 5, the
+ *                        convergence figures): mean loss, and RMSE (regression) or accuracy
+ *                        (classification) of the scores eq. (fm_model2)
  *
  * Readings of points the paper leaves garbled or open (each also listed in the design notes):
  *   - update = gradient descent on eq. (fm_obj): theta <- theta - eta_s (G * df/dtheta + lambda theta);
@@ -260,4 +263,32 @@ int64_t oracle_column_epoch(int64_t n, int32_t d, int32_t K, int32_t p, int32_t 
     *wj_out = wj;
     free(a);
     return count;
+}
+
+/* Held-out evaluation (Section 5: the convergence figures plot objective, test RMSE for the
+ * regression sets and test accuracy for the classification sets).  m rows as CSR with labels y.
+ * out2[0] = (1/m) sum_i l(f_i, y_i) with the loss of the model;
+ * out2[1] = sqrt((1/m) sum_i (f_i - y_i)^2)          for the squared loss (RMSE),
+ *         = (1/m) #{ i : y_i f_i > 0 }                for the logistic loss (accuracy; the predicted
+ *           class is the sign of the score, and a score of exactly 0 predicts neither class).
+ * With decide_in_fp32 != 0 the sign test is taken on the score rounded to fp32, the precision in
+ * which the CUDA path holds its scores. */
+void oracle_evaluate(int64_t m, int32_t K, int32_t loss, const int64_t *indptr, const int32_t *indices,
+                     const float *values, const float *y, double w0, const double *w, const double *V,
+                     int32_t decide_in_fp32, double *out2) {
+    double suml = 0.0, sumsq = 0.0, correct = 0.0;
+    double *a = (double *)malloc(sizeof(double) * (size_t)(K > 0 ? K : 1));
+    for (int64_t i = 0; i < m; ++i) {
+        const double f = score_row(K, indptr[i + 1] - indptr[i], indices + indptr[i], values + indptr[i],
+                                   w0, w, V, a, NULL, NULL);
+        const double yi = (double)y[i];
+        suml += loss_value(loss, f, yi);
+        sumsq += (f - yi) * (f - yi);
+        const double fd = decide_in_fp32 ? (double)(float)f : f;
+        if (yi * fd > 0.0) correct += 1.0;
+    }
+    free(a);
+    out2[0] = m > 0 ? suml / (double)m : 0.0;
+    if (loss == ORACLE_SQUARED) out2[1] = m > 0 ? sqrt(sumsq / (double)m) : 0.0;
+    else out2[1] = m > 0 ? correct / (double)m : 0.0;
 }

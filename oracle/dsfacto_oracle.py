@@ -77,6 +77,18 @@ def score(indptr, indices, values, w0, w, V):
     return out
 
 
+def evaluate(loss, indptr, indices, values, y, w0, w, V, decide_in_fp32=True):
+    """Held-out mean loss and RMSE (squared loss) or accuracy (logistic loss) of the scores."""
+    indptr = np.ascontiguousarray(indptr, np.int64)
+    indices = np.ascontiguousarray(indices, np.int32)
+    values = np.ascontiguousarray(values, np.float32)
+    y = np.ascontiguousarray(y, np.float32)
+    out = np.zeros(2, np.float64)
+    lib().oracle_evaluate(_i64(len(indptr) - 1), _i32(V.shape[1]), _i32(loss), _p(indptr), _p(indices), _p(values),
+                          _p(y), _f64(w0), _p(w), _p(V), _i32(1 if decide_in_fp32 else 0), _p(out))
+    return float(out[0]), float(out[1])
+
+
 def column_epoch(wl_n, d, K, p, loss, eta_s, lambda_w, lambda_v, indptr, indices, values, y, w0, w, V, j):
     wj = ctypes.c_double(0.0)
     vj = np.empty(K, np.float64)
@@ -93,6 +105,7 @@ class Oracle:
         self.n, self.d, self.K, self.p, self.loss = int(n), int(d), int(K), int(p), int(loss)
         self.lambda_w, self.lambda_v, self.eta = float(lambda_w), float(lambda_v), float(eta)
         # per-nonzero step: eta / N (the objective is normalised by 1/N); literal_step keeps eta
+        self.literal_step = bool(literal_step)
         self.eta_s = self.eta if literal_step else self.eta / max(self.n, 1)
         self.w0, self.w, self.V = init_params(self.d, self.K, seed)
         self.loaded = False
@@ -154,3 +167,11 @@ class Oracle:
             indptr, indices, values = self.indptr, self.indices, self.values
         return score(np.ascontiguousarray(indptr, np.int64), np.ascontiguousarray(indices, np.int32),
                      np.ascontiguousarray(values, np.float32), self.w0, self.w, self.V)
+
+    def evaluate(self, indptr, indices, values, y, decide_in_fp32=True):
+        return evaluate(self.loss, indptr, indices, values, y, self.w0, self.w, self.V, decide_in_fp32)
+
+    def set_eta(self, eta):
+        """New learning rate for the following epochs (step-size schedules are the caller's)."""
+        self.eta = float(eta)
+        self.eta_s = self.eta if self.literal_step else self.eta / max(self.n, 1)

@@ -121,3 +121,41 @@ def test_init_is_seeded_normal_with_sigma_001():
     # 4-sigma tail fraction of a normal: 6.3e-5; a uniform or wrong-variance draw would miss this
     assert (np.abs(V) > 0.04).mean() < 5e-4 and (np.abs(V) > 0.02).mean() == pytest.approx(0.0455, rel=0.1)
     assert not np.array_equal(V, O.init_params(4000, 8, seed=2005)[2])
+
+
+@pytest.mark.parametrize("loss", [O.SQUARED, O.LOGISTIC])
+def test_heldout_evaluation_matches_library_metrics(loss):
+    # mean loss, RMSE and accuracy of held-out rows against scikit-learn's metric routines applied
+    # to brute-force pairwise scores (eq. (fm_model)); a flipped label must change the answer
+    from sklearn.metrics import accuracy_score, log_loss, mean_squared_error
+
+    rng = np.random.default_rng(40 + loss)
+    n, d, K = 23, 7, 3
+    X, mask, indptr, indices, vals, w0, w, V = tiny_problem(rng, n, d, K, 0.6)
+    f = fm_pairwise(X, mask, w0, w, V)
+    if loss == O.SQUARED:
+        y = (f + rng.standard_normal(n)).astype(np.float32)
+        mean_loss, rmse = O.evaluate(loss, indptr, indices, vals, y, w0, w, V)
+        mse = mean_squared_error(y.astype(np.float64), f)
+        assert rmse == pytest.approx(math.sqrt(mse), rel=1e-12)
+        assert mean_loss == pytest.approx(0.5 * mse, rel=1e-12)
+        y2 = y.copy(); y2[3] += 1.0
+        assert O.evaluate(loss, indptr, indices, vals, y2, w0, w, V)[1] != pytest.approx(rmse, rel=1e-6)
+    else:
+        y = np.where(rng.random(n) < 0.5, 1.0, -1.0).astype(np.float32)
+        mean_loss, acc = O.evaluate(loss, indptr, indices, vals, y, w0, w, V, decide_in_fp32=False)
+        assert acc == pytest.approx(accuracy_score(y, np.where(f > 0, 1.0, -1.0)), abs=1e-15)
+        prob = 1.0 / (1.0 + np.exp(-f))                                    # P(y = +1 | x) under the logistic model
+        assert mean_loss == pytest.approx(log_loss(y, prob, labels=[-1.0, 1.0]), rel=1e-10)
+        y2 = y.copy(); y2[3] = -y2[3]
+        assert abs(O.evaluate(loss, indptr, indices, vals, y2, w0, w, V)[1] - acc) == pytest.approx(1.0 / n, rel=1e-9)
+
+
+def test_heldout_accuracy_counts_zero_score_as_wrong():
+    # w = 0, V = 0, w0 = 0: every score is exactly 0, which predicts neither class
+    indptr = np.array([0, 1, 2], np.int64)
+    indices = np.array([0, 1], np.int32)
+    vals = np.array([1.0, 2.0], np.float32)
+    y = np.array([1.0, -1.0], np.float32)
+    mean_loss, acc = O.evaluate(O.LOGISTIC, indptr, indices, vals, y, 0.0, np.zeros(2), np.zeros((2, 2)))
+    assert acc == 0.0 and mean_loss == pytest.approx(math.log(2.0), rel=1e-15)
