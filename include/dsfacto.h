@@ -85,6 +85,22 @@ int dsfacto_epoch(dsfacto_t *h);
 int dsfacto_predict(dsfacto_t *h, int64_t m, const int64_t *indptr, const int32_t *indices,
                     const float *values, float *scores_out);
 
+/* Held-out evaluation, the quantities the convergence figures of Section 5 plot beside the
+ * objective: m >= 1 rows as CSR (same rules as dsfacto_load_csr; indptr must not be NULL) with labels
+ * y fp32[m] (finite; +-1 for the logistic loss), scored with the current parameters.
+ *   *mean_loss = (1/m) sum_i l(f(x_i), y_i) with the handle's loss;
+ *   *metric    = sqrt((1/m) sum_i (f(x_i) - y_i)^2)   (RMSE)       for DSFACTO_SQUARED,
+ *              = (1/m) #{ i : y_i f(x_i) > 0 }        (accuracy)   for DSFACTO_LOGISTIC; the predicted
+ *                class is the sign of the fp32 score, and a score of exactly 0 predicts neither class.
+ * Either output pointer may be NULL.  The training state (A, G, objective) is not touched. */
+int dsfacto_evaluate(dsfacto_t *h, int64_t m, const int64_t *indptr, const int32_t *indices,
+                     const float *values, const float *y, double *mean_loss, double *metric);
+
+/* Sets the learning rate eta (> 0, finite) used by the following epochs; the per-entry step becomes
+ * eta / n.  Step-size schedules (the experiments' file names mention a decay, the text does not define
+ * it) are left to the caller: call this between epochs. */
+int dsfacto_set_eta(dsfacto_t *h, float eta);
+
 /* Objective eq. (fm_obj) as of the last recompute pass (after load_csr, epoch or set_params). */
 int dsfacto_objective(dsfacto_t *h, double *out);
 

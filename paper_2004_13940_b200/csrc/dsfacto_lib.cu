@@ -229,9 +229,10 @@ void launch_sgd(dsfacto *h, const SgdChunkArgs &a, int grid) {
     else sgd_chunk_kernel<LG, NV, false><<<grid, kSgdThreads, bytes, h->stream>>>(a);
 }
 template <int LG, int NV>
-void launch_refresh(dsfacto *h, const RefreshArgs &a, bool train, int grid) {
-    if (train) refresh_kernel<LG, NV, true><<<grid, kThreads, 0, h->stream>>>(a);
-    else refresh_kernel<LG, NV, false><<<grid, kThreads, 0, h->stream>>>(a);
+void launch_refresh(dsfacto *h, const RefreshArgs &a, int mode, int grid) {
+    if (mode == kTrain) refresh_kernel<LG, NV, kTrain><<<grid, kThreads, 0, h->stream>>>(a);
+    else if (mode == kEvaluate) refresh_kernel<LG, NV, kEvaluate><<<grid, kThreads, 0, h->stream>>>(a);
+    else refresh_kernel<LG, NV, kScore><<<grid, kThreads, 0, h->stream>>>(a);
 }
 
 #define DSF_DISPATCH(h, FN, ...)                                   \
@@ -325,7 +326,7 @@ int run_refresh(dsfacto *h, bool timed) {
     a.n = h->n; a.indptr = h->d_indptr; a.idx = h->d_idx; a.val = h->d_val; a.y = h->d_y;
     a.w = h->d_w; a.V = h->d_V; a.A = h->d_A; a.G = h->d_G; a.f_out = nullptr;
     a.partials = h->d_partials; a.w0 = h->w0; a.loss = h->loss;
-    DSF_DISPATCH(h, launch_refresh, h, a, true, h->refresh_grid);
+    DSF_DISPATCH(h, launch_refresh, h, a, kTrain, h->refresh_grid);
     reduce2_kernel<<<1, kThreads, 0, h->stream>>>(h->d_partials, h->refresh_grid, h->d_scal);
     if (timed) cudaEventRecord(h->ev[2], h->stream);
     double *np = h->d_partials + 2 * (size_t)h->refresh_grid;
@@ -790,17 +791,19 @@ int dsfacto_bucket_host(int64_t n, int32_t d, int32_t p, const int64_t *indptr, 
     return DSFACTO_OK;
 }
 
-int dsfacto_predict(dsfacto_t *h, int64_t m, const int64_t *indptr, const int32_t *indices, const float *values,
-                    float *scores_out) {
-    if (!h || !scores_out || m < 0) return DSFACTO_ERR_INVALID_ARG;
-    if (m == 0) return DSFACTO_OK;
+// Scores m rows (training rows when indptr is NULL, otherwise a caller CSR copied to the device for
+// the call).  mode kScore: scores_out fp32[m].  mode kEvaluate: labels y (host) and sums2 = {sum of
+// losses, sum of squared errors or number of correct signs}.
+static int score_rows(dsfacto_t *h, int mode, int64_t m, const int64_t *indptr, const int32_t *indices,
+                      const float *values, const float *y, float *scores_out, double sums2[2]) {
     RefreshArgs a{};
     a.w = h->d_w; a.V = h->d_V; a.w0 = h->w0; a.loss = h->loss; a.n = m;
     int64_t *d_ip = nullptr;
     int32_t *d_ix = nullptr;
-    float *d_vl = nullptr, *d_f = nullptr;
+    float *d_vl = nullptr, *d_f = nullptr, *d_yy = nullptr;
+    double *d_part = nullptr;
     int rc = DSFACTO_OK;
-    auto cleanup = [&]() { dev_free(d_ip); dev_free(d_ix); dev_free(d_vl); dev_free(d_f); };
+    auto cleanup = [&]() { dev_free(d_ip); dev_free(d_ix); dev_free(d_vl); dev_free(d_f); dev_free(d_yy); dev_free(d_part); };
     if (!indptr) {
         if (!h->loaded) return DSFACTO_ERR_NO_DATA;
         if (m != h->n) return DSFACTO_ERR_INVALID_ARG;
@@ -822,15 +825,57 @@ int dsfacto_predict(dsfacto_t *h, int64_t m, const int64_t *indptr, const int32_
         }
         a.indptr = d_ip; a.idx = d_ix; a.val = d_vl;
     }
-    if ((rc = dev_alloc(h, &d_f, (size_t)m))) { cleanup(); return rc; }
-    a.f_out = d_f;
-    DSF_DISPATCH(h, launch_refresh, h, a, false, refresh_grid_for(h, m));
-    h->launches += 1;
-    cudaError_t e = cudaMemcpyAsync(scores_out, d_f, sizeof(float) * (size_t)m, cudaMemcpyDeviceToHost, h->stream);
+    const int grid = refresh_grid_for(h, m);
+    cudaError_t e = cudaSuccess;
+    if (mode == kScore) {
+        if ((rc = dev_alloc(h, &d_f, (size_t)m))) { cleanup(); return rc; }
+        a.f_out = d_f;
+        DSF_DISPATCH(h, launch_refresh, h, a, kScore, grid);
+        h->launches += 1;
+        e = cudaMemcpyAsync(scores_out, d_f, sizeof(float) * (size_t)m, cudaMemcpyDeviceToHost, h->stream);
+    } else {
+        if ((rc = dev_alloc(h, &d_yy, (size_t)m)) || (rc = dev_alloc(h, &d_part, 2 * (size_t)grid + 2))) { cleanup(); return rc; }
+        cudaMemcpyAsync(d_yy, y, sizeof(float) * (size_t)m, cudaMemcpyHostToDevice, h->stream);
+        a.y = d_yy; a.partials = d_part;
+        DSF_DISPATCH(h, launch_refresh, h, a, kEvaluate, grid);
+        reduce2_kernel<<<1, kThreads, 0, h->stream>>>(d_part, grid, d_part + 2 * (size_t)grid);
+        h->launches += 2;
+        e = cudaMemcpyAsync(sums2, d_part + 2 * (size_t)grid, 2 * sizeof(double), cudaMemcpyDeviceToHost, h->stream);
+    }
     if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
     if (e == cudaSuccess) e = cudaGetLastError();
     cleanup();
     if (e != cudaSuccess) { h->err = cudaGetErrorString(e); return DSFACTO_ERR_CUDA; }
+    return DSFACTO_OK;
+}
+
+int dsfacto_predict(dsfacto_t *h, int64_t m, const int64_t *indptr, const int32_t *indices, const float *values,
+                    float *scores_out) {
+    if (!h || !scores_out || m < 0) return DSFACTO_ERR_INVALID_ARG;
+    if (m == 0) return DSFACTO_OK;
+    return score_rows(h, kScore, m, indptr, indices, values, nullptr, scores_out, nullptr);
+}
+
+int dsfacto_evaluate(dsfacto_t *h, int64_t m, const int64_t *indptr, const int32_t *indices, const float *values,
+                     const float *y, double *mean_loss, double *metric) {
+    if (!h || !indptr || !y || m < 1) return DSFACTO_ERR_INVALID_ARG;
+    int bad = 0;
+#pragma omp parallel for schedule(static) reduction(| : bad)
+    for (int64_t i = 0; i < m; ++i)
+        if (!std::isfinite(y[i])) bad |= 1;
+    if (bad) return DSFACTO_ERR_INVALID_CSR;
+    double s[2] = {0.0, 0.0};
+    const int rc = score_rows(h, kEvaluate, m, indptr, indices, values, y, nullptr, s);
+    if (rc) return rc;
+    if (mean_loss) *mean_loss = s[0] / (double)m;
+    if (metric) *metric = h->loss == DSFACTO_SQUARED ? std::sqrt(s[1] / (double)m) : s[1] / (double)m;
+    return DSFACTO_OK;
+}
+
+int dsfacto_set_eta(dsfacto_t *h, float eta) {
+    if (!h || !(eta > 0.f) || !std::isfinite(eta)) return DSFACTO_ERR_INVALID_ARG;
+    h->eta = eta;
+    h->h = (float)((double)eta / (double)h->n);
     return DSFACTO_OK;
 }
 

@@ -9,8 +9,12 @@ namespace dsf {
 // Recompute pass (eq. (compute_a_jk), eq. (fm_model2), multiplier G): one lane group per row.
 //   a_ik = sum_j v_jk x_ij ; lin_i = sum_j w_j x_ij ; q_i = sum_j sum_k (v_jk x_ij)^2
 //   f_i = w0 + lin_i + 1/2 (sum_k a_ik^2 - q_i)
-// TRAIN: writes A, G and per-CTA fp64 partial sums {sum l_i, sum G_i}; otherwise writes f only.
+// MODE kScore: writes f only.  kTrain: writes A, G and per-CTA fp64 partial sums {sum l_i, sum G_i}.
+// kEvaluate (held-out rows with labels; the quantities of the convergence figures of Section 5):
+// writes nothing per row, per-CTA fp64 partial sums {sum l_i, sum t_i} with t_i = (f_i - y_i)^2 for
+// the squared loss (RMSE) and t_i = [y_i f_i > 0] for the logistic loss (accuracy).
 // ------------------------------------------------------------------------------------------
+enum { kScore = 0, kTrain = 1, kEvaluate = 2 };
 struct RefreshArgs {
     int64_t n;
     const int64_t *indptr;
@@ -27,7 +31,7 @@ struct RefreshArgs {
     int loss;
 };
 
-template <int LG, int NV, bool TRAIN>
+template <int LG, int NV, int MODE>
 __global__ void __launch_bounds__(kThreads) refresh_kernel(const RefreshArgs a) {
     constexpr int G = kThreads / LG;
     constexpr int KP4 = LG * NV;
@@ -36,6 +40,7 @@ __global__ void __launch_bounds__(kThreads) refresh_kernel(const RefreshArgs a) 
     const uint32_t gm = group_mask<LG>();
     const float4 *V4 = reinterpret_cast<const float4 *>(a.V);
     float4 *A4 = reinterpret_cast<float4 *>(a.A);
+    constexpr bool TRAIN = MODE == kTrain;
     double loss_sum = 0.0, g_sum = 0.0;
 
     for (int64_t row = (int64_t)blockIdx.x * G + g; row < a.n; row += (int64_t)gridDim.x * G) {
@@ -101,7 +106,7 @@ __global__ void __launch_bounds__(kThreads) refresh_kernel(const RefreshArgs a) 
         }
         if (l == 0) {
             const float f = a.w0 + lin + 0.5f * pair;
-            if (TRAIN) {
+            if (MODE != kScore) {
                 const float yy = a.y[row];
                 float li, gi;
                 if (a.loss == 0) {
@@ -112,15 +117,21 @@ __global__ void __launch_bounds__(kThreads) refresh_kernel(const RefreshArgs a) 
                     li = fmaxf(-m, 0.f) + log1pf(expf(-fabsf(m)));
                     gi = -yy / (1.f + expf(m));
                 }
-                a.G[row] = gi;
                 loss_sum += (double)li;
-                g_sum += (double)gi;
+                if (TRAIN) {
+                    a.G[row] = gi;
+                    g_sum += (double)gi;
+                } else if (a.loss == 0) {
+                    g_sum += (double)gi * (double)gi;      // (f - y)^2 for the RMSE
+                } else {
+                    g_sum += (yy * f > 0.f) ? 1.0 : 0.0;   // the sign of the score is the predicted class
+                }
             } else {
                 a.f_out[row] = f;
             }
         }
     }
-    if (TRAIN) {
+    if (MODE != kScore) {
         block_sum2(loss_sum, g_sum);
         if (threadIdx.x == 0) {
             a.partials[2 * blockIdx.x] = loss_sum;

@@ -24,6 +24,9 @@ SIGNATURES = {
     "dsfacto_load_csr": (ctypes.c_int, [_vp, _vp, _vp, _vp, _vp]),
     "dsfacto_epoch": (ctypes.c_int, [_vp]),
     "dsfacto_predict": (ctypes.c_int, [_vp, _c_i64, _vp, _vp, _vp, _vp]),
+    "dsfacto_evaluate": (ctypes.c_int, [_vp, _c_i64, _vp, _vp, _vp, _vp, ctypes.POINTER(ctypes.c_double),
+                                        ctypes.POINTER(ctypes.c_double)]),
+    "dsfacto_set_eta": (ctypes.c_int, [_vp, _c_f32]),
     "dsfacto_objective": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_double)]),
     "dsfacto_get_params": (ctypes.c_int, [_vp, _vp, _vp, _vp]),
     "dsfacto_set_params": (ctypes.c_int, [_vp, _vp, _vp, _vp]),
@@ -84,6 +87,17 @@ def dsfacto_epoch(h):
 
 def dsfacto_predict(h, m, indptr, indices, values, out):
     return lib().dsfacto_predict(h, m, _ptr(indptr), _ptr(indices), _ptr(values), _ptr(out))
+
+
+def dsfacto_evaluate(h, m, indptr, indices, values, y):
+    ml, mt = ctypes.c_double(), ctypes.c_double()
+    rc = lib().dsfacto_evaluate(h, m, _ptr(indptr), _ptr(indices), _ptr(values), _ptr(y), ctypes.byref(ml),
+                                ctypes.byref(mt))
+    return rc, ml.value, mt.value
+
+
+def dsfacto_set_eta(h, eta):
+    return lib().dsfacto_set_eta(h, eta)
 
 
 def dsfacto_objective(h):
@@ -212,6 +226,22 @@ class DSFacto:
         out = np.empty(max(m, 1), np.float32)[:m]
         self._check(dsfacto_predict(self._h, m, indptr, indices, values, out), "dsfacto_predict")
         return out
+
+    def evaluate(self, indptr, indices, values, y):
+        """Held-out (mean loss, RMSE or accuracy) of the rows given as CSR with labels y."""
+        indptr = np.ascontiguousarray(indptr, np.int64)
+        indices = np.ascontiguousarray(indices, np.int32)
+        values = np.ascontiguousarray(values, np.float32)
+        y = np.ascontiguousarray(y, np.float32)
+        m = indptr.shape[0] - 1
+        if y.shape != (m,):
+            raise ValueError("y must have one label per row")
+        rc, ml, mt = dsfacto_evaluate(self._h, m, indptr, indices, values, y)
+        self._check(rc, "dsfacto_evaluate")
+        return ml, mt
+
+    def set_eta(self, eta: float):
+        self._check(dsfacto_set_eta(self._h, float(eta)), "dsfacto_set_eta")
 
     def get_tiles(self):
         tile_ptr = np.empty(self.p * self.p + 1, np.int64)
