@@ -43,22 +43,42 @@ __global__ void __launch_bounds__(kThreads) refresh_kernel(const RefreshArgs a) 
     constexpr bool TRAIN = MODE == kTrain;
     double loss_sum = 0.0, g_sum = 0.0;
 
-    for (int64_t row = (int64_t)blockIdx.x * G + g; row < a.n; row += (int64_t)gridDim.x * G) {
-        const int64_t beg = a.indptr[row], end = a.indptr[row + 1];
+    // The row pointers of the next row are requested while the current row is processed, and its
+    // first batch of entries during the current row's last batch: a lane group never waits for the
+    // pointer -> entry -> factor-row chain at a row start, except at its very first row.
+    const int64_t row_first = (int64_t)blockIdx.x * G + g, row_step = (int64_t)gridDim.x * G;
+    int64_t nbeg = 0, nend = 0;
+    int32_t jn = 0;
+    float xn = 0.f;
+    if (row_first < a.n) {
+        nbeg = __ldg(a.indptr + row_first);
+        nend = __ldg(a.indptr + row_first + 1);
+        if (nbeg + l < nend) { jn = __ldg(a.idx + nbeg + l); xn = __ldg(a.val + nbeg + l); }
+    }
+    for (int64_t row = row_first; row < a.n; row += row_step) {
+        const int64_t beg = nbeg, end = nend;
+        const bool has_next = row + row_step < a.n;
+        if (has_next) {
+            nbeg = __ldg(a.indptr + row + row_step);
+            nend = __ldg(a.indptr + row + row_step + 1);
+        }
         float4 acc[NV];
 #pragma unroll
         for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
         float q = 0.f, lin = 0.f;
-        // this lane's entry of the next batch is fetched while the current batch is processed
-        int32_t jn = 0;
-        float xn = 0.f;
-        if (beg + l < end) { jn = __ldg(a.idx + beg + l); xn = __ldg(a.val + beg + l); }
+        if (beg >= end && has_next) {   // empty row: no batch below fetches the next row's entries
+            jn = 0; xn = 0.f;
+            if (nbeg + l < nend) { jn = __ldg(a.idx + nbeg + l); xn = __ldg(a.val + nbeg + l); }
+        }
         for (int64_t t0 = beg; t0 < end; t0 += LG) {
             const int32_t jm = jn;
             const float xm = xn;
-            const int64_t ahead = t0 + LG + l;
+            // this lane's entry of the next batch (of this row, or the first batch of the next row)
+            // is fetched while the current batch is processed
+            int64_t ahead = t0 + LG + l, ahead_end = end;
+            if (t0 + LG >= end) { ahead = nbeg + l; ahead_end = has_next ? nend : nbeg; }
             jn = 0; xn = 0.f;
-            if (ahead < end) { jn = __ldg(a.idx + ahead); xn = __ldg(a.val + ahead); }
+            if (ahead < ahead_end) { jn = __ldg(a.idx + ahead); xn = __ldg(a.val + ahead); }
             if (t0 + l < end) lin = fmaf(__ldg(a.w + jm), xm, lin);
             const int cnt = (int)((end - t0) < (int64_t)LG ? (end - t0) : (int64_t)LG);
             // the rows of up to UB entries are requested before any of them is used

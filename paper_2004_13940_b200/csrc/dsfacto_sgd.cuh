@@ -37,10 +37,16 @@ constexpr int kSyncError = kSyncStride;           // set when a dependency wait 
 __host__ __device__ constexpr size_t sync_done(int c) { return (size_t)(2 + c) * kSyncStride; }  // finished tiles of column block c
 __host__ __device__ constexpr size_t sync_words(int p) { return (size_t)(2 + p) * kSyncStride; }
 
-// entries of one warp pass: sized so that the gathered rows of A fill about 4 KB of shared memory
+// entries of one warp pass: sized so that the gathered rows of A fill about 4 KB of shared memory, but
+// never fewer than 16 entries: with 8-entry passes (rows of 512 bytes and more) the fixed cost of a
+// pass and its one exposed gather latency dominated (K = 128: 59.1 ms per sweep with 8, 46.7 with 16,
+// 54.6 with 32 on the 400 M-entry workload)
 __host__ __device__ constexpr int sgd_pass_len(int LG, int NV) {
-    return 256 / (LG * NV) > 256 ? 256 : (256 / (LG * NV) < 8 ? 8 : 256 / (LG * NV));
+    return 256 / (LG * NV) > 256 ? 256 : (256 / (LG * NV) < 16 ? 16 : 256 / (LG * NV));
 }
+// resident one-warp CTAs per SM the register budget is cut for: 24 for rows up to 256 bytes; wider
+// rows hold 16 entries per lane group in flight and are limited by shared memory anyway
+__host__ __device__ constexpr int sgd_min_ctas(int LG, int NV) { return LG * NV >= 32 ? 12 : 24; }
 // floats per chunk record in global scratch: 3 header float4s + head offsets + tail offsets
 __host__ __device__ constexpr int chunk_record_floats(int Kp) { return 12 + 2 * Kp; }
 
@@ -279,7 +285,7 @@ struct SgdChunkArgs {
 };
 
 template <int LG, int NV, bool WIDE>
-__global__ void __launch_bounds__(kSgdThreads, 24) sgd_chunk_kernel(const SgdChunkArgs a) {
+__global__ void __launch_bounds__(kSgdThreads, sgd_min_ctas(LG, NV)) sgd_chunk_kernel(const SgdChunkArgs a) {
     typedef SgdSmem<LG, NV> L;
     constexpr int GW = L::GW, KP4 = L::KP4, PASS = L::PASS, S = L::S;
     constexpr int PP = kWarpEntries / PASS;
