@@ -22,6 +22,8 @@
  *                        staleness ...": the auxiliaries are recomputed after the update step)
  *   oracle_epoch         one outer iteration t of Algorithm 1 in its synchronous (DSGD-style) form:
  *                        the update loop, then the recompute loop
+ *   oracle_epoch_segmented  the same epoch with the recompute loop run after every R inner rounds
+ *                        (Section 4.2: stale G, A slow convergence, hence the recompute)
  *   oracle_evaluate      the quantities the experiments plot on held-out rows (Section 5, the
  *                        convergence figures): mean loss, and RMSE (regression) or accuracy
  *                        (classification) of the scores eq. (fm_model2)
@@ -192,13 +194,13 @@ void oracle_refresh(int64_t n, int32_t d, int32_t K, int32_t loss, double lambda
     out3[2] = out3[1] + 0.5 * lambda_w * w2 + 0.5 * lambda_v * v2;
 }
 
-/* Update loop of Algorithm 1, synchronous form: rounds s = 0..p-1; in round s the p tiles
+/* Update loop of Algorithm 1, synchronous form, inner rounds s0 <= s < s1: in round s the p tiles
  * (r, (r+s) mod p) touch disjoint rows and disjoint columns, so they run in parallel.  Each stored
  * entry applies eqs. (dsfacto_sgdupdatew) / (dsfacto_sgdupdatev) once with frozen G_i, a_ik. */
-void oracle_sgd_phase(int32_t K, int32_t p, double eta_s, double lambda_w, double lambda_v,
-                      const int64_t *tile_ptr, const int32_t *rows, const int32_t *cols,
-                      const float *vals, const double *A, const double *G, double *w, double *V) {
-    for (int32_t s = 0; s < p; ++s) {
+void oracle_sgd_rounds(int32_t K, int32_t p, int32_t s0, int32_t s1, double eta_s, double lambda_w,
+                       double lambda_v, const int64_t *tile_ptr, const int32_t *rows, const int32_t *cols,
+                       const float *vals, const double *A, const double *G, double *w, double *V) {
+    for (int32_t s = s0; s < s1; ++s) {
 #pragma omp parallel for schedule(dynamic, 1)
         for (int32_t r = 0; r < p; ++r) {
             const int64_t t = (int64_t)s * p + r;
@@ -216,6 +218,13 @@ void oracle_sgd_phase(int32_t K, int32_t p, double eta_s, double lambda_w, doubl
     }
 }
 
+/* The whole update loop: rounds 0..p-1. */
+void oracle_sgd_phase(int32_t K, int32_t p, double eta_s, double lambda_w, double lambda_v,
+                      const int64_t *tile_ptr, const int32_t *rows, const int32_t *cols,
+                      const float *vals, const double *A, const double *G, double *w, double *V) {
+    oracle_sgd_rounds(K, p, 0, p, eta_s, lambda_w, lambda_v, tile_ptr, rows, cols, vals, A, G, w, V);
+}
+
 /* One epoch: w0 step with the frozen multipliers, the p strata, then the recompute pass. */
 void oracle_epoch(int64_t n, int32_t d, int32_t K, int32_t p, int32_t loss, double eta_s,
                   double lambda_w, double lambda_v, const int64_t *indptr, const int32_t *indices,
@@ -226,6 +235,28 @@ void oracle_epoch(int64_t n, int32_t d, int32_t K, int32_t p, int32_t loss, doub
     oracle_sgd_phase(K, p, eta_s, lambda_w, lambda_v, tile_ptr, rows, cols, vals, A, G, w, V);
     oracle_refresh(n, d, K, loss, lambda_w, lambda_v, indptr, indices, values, y, *w0, w, V, A, lin, q, f,
                    lossv, G, out3);
+}
+
+/* Second schedule: shorter staleness.  Section 4.2 ("Handling the staleness ...") recomputes G and A
+ * after the update step because stale auxiliaries slow convergence; this variant applies the same
+ * recompute after every `every` inner rounds instead of after all p (every <= 0 or >= p gives
+ * oracle_epoch).  Reading for w0, which belongs to no column block: before a segment of m rounds it
+ * takes the share m/p of its epoch step with the multipliers frozen for that segment,
+ * w0 <- w0 - eta_s (m/p) sum_i G_i, so that the shares add up to the one step of oracle_epoch. */
+void oracle_epoch_segmented(int64_t n, int32_t d, int32_t K, int32_t p, int32_t loss, int32_t every,
+                            double eta_s, double lambda_w, double lambda_v, const int64_t *indptr,
+                            const int32_t *indices, const float *values, const float *y,
+                            const int64_t *tile_ptr, const int32_t *rows, const int32_t *cols,
+                            const float *vals, double *w0, double *w, double *V, double *A, double *lin,
+                            double *q, double *f, double *lossv, double *G, double *out3) {
+    if (every <= 0 || every > p) every = p;
+    for (int32_t s0 = 0; s0 < p; s0 += every) {
+        const int32_t s1 = s0 + every < p ? s0 + every : p;
+        *w0 = *w0 - eta_s * ((double)(s1 - s0) / (double)p) * out3[0];
+        oracle_sgd_rounds(K, p, s0, s1, eta_s, lambda_w, lambda_v, tile_ptr, rows, cols, vals, A, G, w, V);
+        oracle_refresh(n, d, K, loss, lambda_w, lambda_v, indptr, indices, values, y, *w0, w, V, A, lin, q,
+                       f, lossv, G, out3);
+    }
 }
 
 /* The same epoch restricted to ONE column j, computed straight from the CSR data and the

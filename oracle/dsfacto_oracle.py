@@ -150,6 +150,18 @@ class Oracle:
         self.w0 = w0.value
         return self.objective
 
+    def epoch_segmented(self, every):
+        """One epoch with G, A recomputed after every `every` inner rounds (0: after all p)."""
+        w0 = ctypes.c_double(self.w0)
+        lib().oracle_epoch_segmented(_i64(self.n), _i32(self.d), _i32(self.K), _i32(self.p), _i32(self.loss),
+                                     _i32(every), _f64(self.eta_s), _f64(self.lambda_w), _f64(self.lambda_v),
+                                     _p(self.indptr), _p(self.indices), _p(self.values), _p(self.y),
+                                     _p(self.tile_ptr), _p(self.rows), _p(self.cols), _p(self.vals),
+                                     ctypes.byref(w0), _p(self.w), _p(self.V), _p(self.A), _p(self.lin), _p(self.q),
+                                     _p(self.f), _p(self.lossv), _p(self.G), _p(self.out3))
+        self.w0 = w0.value
+        return self.objective
+
     @property
     def sum_G(self):
         return float(self.out3[0])

@@ -206,3 +206,79 @@ def test_objective_decreases_on_small_workload():
     objs = [o.objective] + [o.epoch() for _ in range(wl.epochs)]
     assert all(b < a for a, b in zip(objs, objs[1:]))
     assert np.isfinite(objs).all()
+
+
+# ---- second schedule: auxiliaries recomputed after every R inner rounds ----
+
+def test_segmented_epoch_with_one_segment_is_the_plain_epoch():
+    for every in (0, 4, 9):
+        a, *_ = _setup(11, 30, 8, 3, 4, O.LOGISTIC)
+        b, *_ = _setup(11, 30, 8, 3, 4, O.LOGISTIC)
+        for _ in range(2):
+            a.epoch()
+            b.epoch_segmented(every)
+        assert a.w0 == b.w0 and np.array_equal(a.w, b.w) and np.array_equal(a.V, b.V)
+        assert a.objective == b.objective
+
+
+@pytest.mark.parametrize("loss,p,every", [(O.SQUARED, 4, 1), (O.LOGISTIC, 5, 2), (O.SQUARED, 3, 2)])
+def test_segmented_epoch_on_linear_model_is_block_gradient_descent(loss, p, every):
+    # V = 0 stays 0, and with lambda_w = 0 every segment is: G from the current (w0, w); then
+    # w[column block c] -= eta_s X[row block r, column block c]^T G[row block r] for the tiles
+    # (r, c = (r+s) mod p) of its rounds; w0 -= eta_s (rounds/p) sum G.  Written with dense numpy
+    # blocks, independent of the oracle's tile lists.
+    n, d, K = 26, 9, 2
+    rng = np.random.default_rng(91 + p)
+    X, mask, indptr, indices, vals, w0, w, V = tiny_problem(rng, n, d, K, 0.5)
+    y = (np.where(rng.random(n) < 0.5, 1.0, -1.0) if loss else rng.standard_normal(n)).astype(np.float32)
+    yd = y.astype(np.float64)
+    eta = 0.3
+    o = O.Oracle(n, d, K, p, loss, 0.0, 0.2, eta, seed=3)
+    o.w0, o.w[:], o.V[:] = w0, w, 0.0
+    o.load_csr(indptr, indices, vals, y)
+    o.epoch_segmented(every)
+    rb = np.arange(n) * p // n
+    cb = np.arange(d) * p // d
+    ww, ww0 = w.copy(), w0
+    for s0 in range(0, p, every):
+        s1 = min(s0 + every, p)
+        f = ww0 + X @ ww
+        G = f - yd if loss == O.SQUARED else -yd / (1 + np.exp(yd * f))
+        ww0 -= eta / n * (s1 - s0) / p * G.sum()
+        for s in range(s0, s1):
+            for r in range(p):
+                c = (r + s) % p
+                rows, cols = np.nonzero(rb == r)[0], np.nonzero(cb == c)[0]
+                ww[cols] -= eta / n * (X[np.ix_(rows, cols)].T @ G[rows])
+    assert not o.V.any()
+    np.testing.assert_allclose(o.w, ww, rtol=1e-12, atol=1e-15)
+    assert o.w0 == pytest.approx(ww0, rel=1e-13)
+    # and it is not the plain epoch: the later segments saw fresher multipliers
+    o2 = O.Oracle(n, d, K, p, loss, 0.0, 0.2, eta, seed=3)
+    o2.w0, o2.w[:], o2.V[:] = w0, w, 0.0
+    o2.load_csr(indptr, indices, vals, y)
+    o2.epoch()
+    assert np.abs(o2.w - o.w).max() > 1e-6
+
+
+def test_segmented_epoch_recomputes_auxiliaries_between_segments():
+    # after a segmented epoch the stored auxiliaries are consistent with the final parameters, and the
+    # factor rows differ from the plain epoch's (the second segment used a_i of the updated V)
+    a, X, mask, *_ = _setup(13, 40, 9, 3, 4, O.SQUARED)
+    b, *_ = _setup(13, 40, 9, 3, 4, O.SQUARED)
+    a.epoch()
+    b.epoch_segmented(2)
+    np.testing.assert_allclose(b.A, X @ b.V, rtol=1e-12, atol=1e-14)
+    assert np.abs(a.V - b.V).max() > 1e-9
+
+
+def test_segmented_schedule_converges_at_least_as_fast_on_small_workload():
+    wl = W.make("C1")
+    objs = {}
+    for every in (0, 1):
+        o = O.Oracle(wl.n, wl.d, wl.K, wl.p, wl.loss, wl.lambda_w, wl.lambda_v, 2.0, wl.init_seed)
+        o.load_csr(wl.indptr, wl.indices, wl.values, wl.y)
+        for _ in range(10):
+            o.epoch_segmented(every)
+        objs[every] = o.objective
+    assert np.isfinite(objs[1]) and objs[1] <= objs[0] * 1.001
