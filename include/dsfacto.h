@@ -101,6 +101,17 @@ int dsfacto_evaluate(dsfacto_t *h, int64_t m, const int64_t *indptr, const int32
  * it) are left to the caller: call this between epochs. */
 int dsfacto_set_eta(dsfacto_t *h, float eta);
 
+/* Second schedule, for shorter staleness (Section 4.2, "Handling the staleness ...": stale G and A
+ * slow convergence, which is why they are recomputed after the update step).  rounds = 0 (default):
+ * the recompute pass runs once per epoch, after all p inner rounds, as in Algorithm 1.  rounds = R >= 1:
+ * dsfacto_epoch cuts the p inner rounds into segments of R consecutive rounds (the last may be
+ * shorter) and runs the recompute pass after every segment; before a segment of m rounds w0 takes the
+ * share m/p of its step, w0 <- w0 - (eta/n) (m/p) sum_i G_i, with the multipliers frozen for that
+ * segment.  R >= p is the default schedule.  An epoch then costs ceil(p/R) recompute passes.
+ * Must be called before dsfacto_load_csr (DSFACTO_ERR_INVALID_ARG afterwards): a value > 0 makes the
+ * load store the tiles round by round, and the handle keeps that order even if 0 is set later. */
+int dsfacto_set_refresh_every(dsfacto_t *h, int32_t rounds);
+
 /* Objective eq. (fm_obj) as of the last recompute pass (after load_csr, epoch or set_params). */
 int dsfacto_objective(dsfacto_t *h, double *out);
 

@@ -49,6 +49,7 @@ struct dsfacto {
     double *d_partials = nullptr, *d_scal = nullptr;
     // stratum SGD launch plan: launch L covers chunks [launch_ptr[L], launch_ptr[L+1]) of chunk_map
     int sweep = 1;  // 1: a launch is a row block (p-1 .. 0); 0: a launch is an inner round (0 .. p-1)
+    int refresh_every = 0;  // > 0: G, A recomputed after every that many inner rounds (needs the round sweep)
     std::vector<int64_t> launch_ptr;
     int4 *d_chunk_map = nullptr;
     int *d_sync = nullptr;     // ticket, error flag, per-column-block progress of the fused SGD launch
@@ -295,21 +296,27 @@ int build_sgd_plan(dsfacto *h) {
     return DSFACTO_OK;
 }
 
-// the p strata of one epoch, then the return from the scaled state to plain parameters
-void run_sgd_phase(dsfacto *h) {
+// The strata [L0, L1) of one epoch (inner rounds for the round sweep, row blocks for the row-block
+// sweep; the whole sweep is [0, p)), then the return from the scaled state to plain parameters.
+void run_sgd_phase(dsfacto *h, int64_t L0, int64_t L1) {
     SgdChunkArgs a{};
     a.tile_ptr = h->d_tile_ptr; a.ent = h->d_ent; a.xw = h->d_xw; a.row_start = h->d_row_start;
     a.col_start = h->d_col_start; a.A = h->d_A; a.G = h->d_G; a.w = h->d_w; a.V = h->d_V;
     a.S = h->d_S; a.Tb = h->d_Tb; a.Tw = h->d_Tw; a.TS = h->d_TS; a.records = h->d_records; a.tile_count = h->d_tile_count;
     a.p = h->p; a.jbits = h->jbits; a.sweep = h->sweep;
     a.h = h->h; a.lambda_w = h->lambda_w; a.lambda_v = h->lambda_v;
-    // One launch for the whole sweep: chunks are taken in sweep order (row block by row block, or round
-    // by round) and a tile waits only for the earlier tiles of its own column block.
-    cudaMemsetAsync(h->d_sync, 0, sizeof(int) * sync_words(h->p), h->stream);
+    // One launch for the whole range: chunks are taken in sweep order (row block by row block, or round
+    // by round) and a tile waits only for the earlier tiles of its own column block.  The counters of
+    // finished tiles are cumulative over the sweep, so they are cleared at its first launch only; the
+    // ticket counter restarts with every launch.
+    if (L0 == 0) cudaMemsetAsync(h->d_sync, 0, sizeof(int) * sync_words(h->p), h->stream);
+    else cudaMemsetAsync(h->d_sync + kSyncTicket, 0, sizeof(int), h->stream);
     a.chunk_map = h->d_chunk_map;
     a.sync = h->d_sync;
-    if (h->total_chunks > 0) {
-        DSF_DISPATCH(h, launch_sgd, h, a, (int)h->total_chunks);
+    a.chunk_base = (int)h->launch_ptr[(size_t)L0];
+    const int64_t chunks = h->launch_ptr[(size_t)L1] - h->launch_ptr[(size_t)L0];
+    if (chunks > 0) {
+        DSF_DISPATCH(h, launch_sgd, h, a, (int)chunks);
         h->launches += 1;
     }
     {   // back from the scaled state to plain (w, V); folds the tail composites in after a row-block sweep
@@ -682,21 +689,42 @@ int dsfacto_epoch(dsfacto_t *h) {
     if (!h->loaded) return DSFACTO_ERR_NO_DATA;
     cudaStream_t st = h->stream;
     CU_TRY(h, cudaEventRecord(h->ev[0], st));
-    // w0 step with the frozen multipliers
-    h->w0 = (float)((double)h->w0 - (double)h->h * h->g_sum);
-    run_sgd_phase(h);
-    CU_TRY(h, cudaEventRecord(h->ev[1], st));
-    int rc = run_refresh(h, true);
-    if (rc) return rc;
+    const int64_t p = h->p;
+    const int64_t every = (h->refresh_every > 0 && h->refresh_every < p) ? h->refresh_every : p;
+    float t01 = 0, t12 = 0, t23 = 0;
+    int rc = DSFACTO_OK;
+    for (int64_t L0 = 0; L0 < p; L0 += every) {
+        const int64_t L1 = std::min(L0 + every, p);
+        if (L0 > 0) CU_TRY(h, cudaEventRecord(h->ev[0], st));
+        // w0 step with the frozen multipliers: the share of the epoch's step that belongs to these rounds
+        h->w0 = (float)((double)h->w0 - (double)h->h * ((double)(L1 - L0) / (double)p) * h->g_sum);
+        run_sgd_phase(h, L0, L1);
+        CU_TRY(h, cudaEventRecord(h->ev[1], st));
+        rc = run_refresh(h, true);
+        if (rc) return rc;
+        float a01 = 0, a12 = 0, a23 = 0;
+        cudaEventElapsedTime(&a01, h->ev[0], h->ev[1]);
+        cudaEventElapsedTime(&a12, h->ev[1], h->ev[2]);
+        cudaEventElapsedTime(&a23, h->ev[2], h->ev[3]);
+        t01 += a01; t12 += a12; t23 += a23;
+    }
     int sgd_error = 0;  // set by the SGD kernel if a dependency wait ran out (never seen; the state is then unusable)
     CU_TRY(h, cudaMemcpy(&sgd_error, h->d_sync + kSyncError, sizeof(int), cudaMemcpyDeviceToHost));
     if (sgd_error) { h->err = "stratum SGD: a wait for an earlier tile of the same column block timed out"; return DSFACTO_ERR_CUDA; }
-    float t01 = 0, t12 = 0, t23 = 0;
-    cudaEventElapsedTime(&t01, h->ev[0], h->ev[1]);
-    cudaEventElapsedTime(&t12, h->ev[1], h->ev[2]);
-    cudaEventElapsedTime(&t23, h->ev[2], h->ev[3]);
     h->ms[0] = t01 + t12 + t23; h->ms[1] = t01; h->ms[2] = t12; h->ms[3] = t23;
     return std::isfinite(h->objective) ? DSFACTO_OK : DSFACTO_ERR_DIVERGED;
+}
+
+int dsfacto_set_refresh_every(dsfacto_t *h, int32_t rounds) {
+    if (!h || rounds < 0) return DSFACTO_ERR_INVALID_ARG;
+    if (h->loaded) return DSFACTO_ERR_INVALID_ARG;   // the tile order on the device is fixed by dsfacto_load_csr
+    h->refresh_every = rounds;
+    if (rounds > 0 && h->sweep != 0) {
+        // inner rounds must be launches of their own: switch to the round sweep (no tail composites)
+        h->sweep = 0;
+        dev_free(h->d_Tb); dev_free(h->d_Tw); dev_free(h->d_TS);
+    }
+    return DSFACTO_OK;
 }
 
 int dsfacto_objective(dsfacto_t *h, double *out) {

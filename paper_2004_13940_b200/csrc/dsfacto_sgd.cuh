@@ -278,9 +278,11 @@ struct SgdChunkArgs {
                                // of earlier non-empty tiles of the same column block, -}
     float *records;            // chunk_record_floats(Kp) floats per chunk
     int *tile_count;           // p*p, all zero between launches
-    int *sync;                 // sync_words(p) ints: ticket counter, error flag, finished tiles per column
-                               // block; all zero at launch
+    int *sync;                 // sync_words(p) ints: ticket counter (zero at launch), error flag, finished
+                               // tiles per column block (zero at the first launch of a sweep, kept between
+                               // the launches of one sweep)
     int p, jbits, sweep;
+    int chunk_base;            // first chunk of this launch in chunk_map (a launch may cover a range of rounds)
     float h, lambda_w, lambda_v;
 };
 
@@ -315,7 +317,7 @@ __global__ void __launch_bounds__(kSgdThreads, sgd_min_ctas(LG, NV)) sgd_chunk_k
     __shared__ int s_ticket, s_go;
     if (tid == 0) s_ticket = atomicAdd(a.sync + kSyncTicket, 1);
     __syncthreads();
-    const int chunk = s_ticket;
+    const int chunk = a.chunk_base + s_ticket;
     const int4 cm = a.chunk_map[chunk];
     const int64_t t = cm.x;  // tile slot: position of the tile in sweep order (the device order of tiles)
     int r, c;

@@ -27,6 +27,7 @@ SIGNATURES = {
     "dsfacto_evaluate": (ctypes.c_int, [_vp, _c_i64, _vp, _vp, _vp, _vp, ctypes.POINTER(ctypes.c_double),
                                         ctypes.POINTER(ctypes.c_double)]),
     "dsfacto_set_eta": (ctypes.c_int, [_vp, _c_f32]),
+    "dsfacto_set_refresh_every": (ctypes.c_int, [_vp, _c_i32]),
     "dsfacto_objective": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_double)]),
     "dsfacto_get_params": (ctypes.c_int, [_vp, _vp, _vp, _vp]),
     "dsfacto_set_params": (ctypes.c_int, [_vp, _vp, _vp, _vp]),
@@ -98,6 +99,10 @@ def dsfacto_evaluate(h, m, indptr, indices, values, y):
 
 def dsfacto_set_eta(h, eta):
     return lib().dsfacto_set_eta(h, eta)
+
+
+def dsfacto_set_refresh_every(h, rounds):
+    return lib().dsfacto_set_refresh_every(h, rounds)
 
 
 def dsfacto_objective(h):
@@ -242,6 +247,10 @@ class DSFacto:
 
     def set_eta(self, eta: float):
         self._check(dsfacto_set_eta(self._h, float(eta)), "dsfacto_set_eta")
+
+    def set_refresh_every(self, rounds: int):
+        """G, A recomputed after every `rounds` inner rounds (0: once per epoch).  Before load_csr."""
+        self._check(dsfacto_set_refresh_every(self._h, int(rounds)), "dsfacto_set_refresh_every")
 
     def get_tiles(self):
         tile_ptr = np.empty(self.p * self.p + 1, np.int64)
