@@ -31,8 +31,11 @@ struct RefreshArgs {
     int loss;
 };
 
+// Rows of 128 bytes and more keep 8 float4s per lane in flight and would take 88 to 100 registers:
+// capped at 80 so that three CTAs stay resident (K = 128: 27.1 -> 22.3 ms per pass on 400 M entries;
+// a cap of 64 registers spills too much: 24.5 ms).  Narrower rows fit 64 registers and four CTAs.
 template <int LG, int NV, int MODE>
-__global__ void __launch_bounds__(kThreads) refresh_kernel(const RefreshArgs a) {
+__global__ void __launch_bounds__(kThreads, (LG >= 8 ? 3 : 4)) refresh_kernel(const RefreshArgs a) {
     constexpr int G = kThreads / LG;
     constexpr int KP4 = LG * NV;
     const int g = threadIdx.x / LG;
