@@ -1,0 +1,59 @@
+"""The three ways dsfacto_load_csr builds the tile lists on the device give the same lists, bit for
+bit, as the oracle's bucketing: the plain host bucketer, the row-block bucketer, and the streamed
+load (row blocks bucketed into page-locked staging memory and copied block by block), which large
+loads take by default and which DSFACTO_LOAD=stream forces on small ones."""
+import numpy as np
+import pytest
+
+from oracle import dsfacto_oracle as O
+from paper_2004_13940_b200 import dsfacto as D
+from paper_2004_13940_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("mode", ["stream", "simple", None])
+@pytest.mark.parametrize("name,kw", [("C3", {}), ("C4s", {}), ("C4s", {"p": 200}), ("C5s", {"p": 64}), ("C2", {"p": 40}),
+                                     ("C1", {"p": 2500})])
+def test_load_paths_give_the_oracle_tiles_and_epochs(monkeypatch, mode, name, kw):
+    if mode is None:
+        monkeypatch.delenv("DSFACTO_LOAD", raising=False)
+    else:
+        monkeypatch.setenv("DSFACTO_LOAD", mode)
+    wl = W.make(name, **kw)
+    o = O.Oracle(wl.n, wl.d, wl.K, wl.p, wl.loss, wl.lambda_w, wl.lambda_v, wl.eta, wl.init_seed)
+    o.load_csr(wl.indptr, wl.indices, wl.values, wl.y)
+    with D.DSFacto(wl.n, wl.d, wl.K, wl.p, wl.loss, wl.lambda_w, wl.lambda_v, wl.eta, wl.init_seed) as g:
+        g.load_csr(wl.indptr, wl.indices, wl.values, wl.y)
+        tp, rows, cols, vals = g.get_tiles()
+        assert np.array_equal(tp, o.tile_ptr)
+        assert np.array_equal(rows, o.rows) and np.array_equal(cols, o.cols) and np.array_equal(vals, o.vals)
+        want, got = o.epoch(), g.epoch()
+        assert got == pytest.approx(want, rel=1e-4)
+        # a second load on the same handle (staging memory is reused) replaces the data set
+        g.load_csr(wl.indptr, wl.indices, wl.values, wl.y)
+        tp2, rows2, cols2, vals2 = g.get_tiles()
+        assert np.array_equal(tp2, tp) and np.array_equal(rows2, rows) and np.array_equal(cols2, cols)
+
+
+def test_streamed_load_of_the_wide_entry_layout(monkeypatch):
+    # 2^16 rows x 2^17 columns per tile: local ids need 33 bits, so entries travel as {row, column} + value
+    monkeypatch.setenv("DSFACTO_LOAD", "stream")
+    rng = np.random.default_rng(5)
+    n, d, p, K = 1 << 21, 1 << 22, 32, 4
+    per_row = 3
+    indices = np.sort(rng.integers(0, d, size=(n, per_row)), axis=1).astype(np.int32)
+    keep = np.ones_like(indices, bool)
+    keep[:, 1:] = indices[:, 1:] != indices[:, :-1]
+    indptr = np.concatenate([[0], np.cumsum(keep.sum(1))]).astype(np.int64)
+    idx = indices[keep]
+    vals = rng.standard_normal(idx.shape[0]).astype(np.float32)
+    y = rng.standard_normal(n).astype(np.float32)
+    o = O.Oracle(n, d, K, p, O.SQUARED, 1e-3, 1e-3, 0.01, 7)
+    o.load_csr(indptr, idx, vals, y)
+    with D.DSFacto(n, d, K, p, D.SQUARED, 1e-3, 1e-3, 0.01, 7) as g:
+        g.load_csr(indptr, idx, vals, y)
+        tp, rows, cols, v = g.get_tiles()
+        assert np.array_equal(tp, o.tile_ptr) and np.array_equal(rows, o.rows) and np.array_equal(cols, o.cols)
+        assert np.array_equal(v, o.vals)
+        assert g.epoch() == pytest.approx(o.epoch(), rel=1e-4)
