@@ -312,7 +312,7 @@ def run_ours(args):
     h2d = (wl.indptr.nbytes + wl.indices.nbytes + wl.values.nbytes + wl.y.nbytes + 8 * nnz + 8 * (p * p + 1))
     e2e = {"value": whole_job_rate(world, nnz, args.e2e_steps, e2e_ms) if args.e2e_steps > 0 else None, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
            "d2h_bytes_per_step": 32, "steps": args.e2e_steps, "ms_per_step": e2e_ms / max(args.e2e_steps, 1),
-           "what": "dsfacto_create + dsfacto_load_csr (host bucketing, H2D) + dsfacto_epoch + dsfacto_objective"}
+           "what": "dsfacto_create + dsfacto_load_csr (host bucketing streamed to the device, H2D) + dsfacto_epoch + dsfacto_objective"}
     cfg = workload_config(args.workload)
     if args.refresh_every > 0:
         cfg["refresh_every"] = args.refresh_every

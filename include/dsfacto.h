@@ -66,7 +66,15 @@ int dsfacto_create(dsfacto_t **out, int64_t n, int32_t d, int32_t K, int32_t p, 
  * pattern": row block of row i is floor(i*p/n), column block of column j is floor(j*p/d); tile
  * (r,c) belongs to round s = (c-r) mod p; tiles ordered by (s, r); inside a tile entries ordered
  * by (column, row)), copies CSR and tiles to the device and runs the recompute pass once, so that
- * A, G and the objective of the initial parameters exist.  Replaces any earlier data set. */
+ * A, G and the objective of the initial parameters exist.  Replaces any earlier data set.
+ * Loads of 2^24 stored entries and more (with p at least twice the number of host threads) are
+ * streamed: each host thread buckets one row block at a time into page-locked staging memory and
+ * copies it to its place on the device while the other row blocks are being bucketed.  That staging
+ * memory (two row blocks per host thread) is allocated on the first such load and kept by the process
+ * for later loads; streamed loads of one process run one at a time.  The environment variable
+ * DSFACTO_LOAD=stream streams smaller loads too, DSFACTO_LOAD=simple never streams.  The resulting tile
+ * lists are the same bit for bit on every path.  Page-locked caller arrays make the CSR copy overlap
+ * the bucketing. */
 int dsfacto_load_csr(dsfacto_t *h, const int64_t *indptr, const int32_t *indices,
                      const float *values, const float *y);
 
