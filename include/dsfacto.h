@@ -72,7 +72,8 @@ int dsfacto_create(dsfacto_t **out, int64_t n, int32_t d, int32_t K, int32_t p, 
  * copies it to its place on the device while the other row blocks are being bucketed.  That staging
  * memory (two row blocks per host thread) is allocated on the first such load and kept by the process
  * for later loads; streamed loads of one process run one at a time.  The environment variable
- * DSFACTO_LOAD=stream streams smaller loads too, DSFACTO_LOAD=simple never streams.  The resulting tile
+ * DSFACTO_LOAD=stream streams smaller loads too, DSFACTO_LOAD=simple never streams; if the staging
+ * memory cannot be had, the load falls back to one copy from pageable memory.  The resulting tile
  * lists are the same bit for bit on every path.  Page-locked caller arrays make the CSR copy overlap
  * the bucketing. */
 int dsfacto_load_csr(dsfacto_t *h, const int64_t *indptr, const int32_t *indices,

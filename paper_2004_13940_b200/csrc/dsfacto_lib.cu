@@ -668,8 +668,11 @@ StagingArena g_staging;
 // place in the device arrays while the other row blocks are being bucketed, so that neither a host
 // copy of the whole entry array nor a copy from pageable memory is needed.  d_ent (and d_xw) must be
 // allocated; tile_ptr is set.  Returns after all copies have completed.
+// *no_staging is set when the page-locked staging memory could not be had; nothing has been copied
+// then and the caller takes the non-streamed way.
 int stream_tiles_by_row_block(dsfacto *h, const std::vector<int32_t> &cb, int64_t longest, const int64_t *indptr,
-                              const int32_t *indices, const float *values) {
+                              const int32_t *indices, const float *values, bool *no_staging) {
+    *no_staging = false;
     int T = omp_get_max_threads();
     if (T > 64) T = 64;
     const size_t per_entry = sizeof(uint2) + (h->wide ? sizeof(float) : 0);
@@ -680,7 +683,14 @@ int stream_tiles_by_row_block(dsfacto *h, const std::vector<int32_t> &cb, int64_
         if (g_staging.ptr) cudaFreeHost(g_staging.ptr);
         g_staging.ptr = nullptr;
         g_staging.bytes = 0;
-        CU_TRY(h, cudaHostAlloc(&g_staging.ptr, need, cudaHostAllocPortable));
+        const char *env = std::getenv("DSFACTO_LOAD");   // "nostaging": behave as if the allocation had failed (tests)
+        const bool refuse = env && std::strcmp(env, "nostaging") == 0;
+        if (refuse || cudaHostAlloc(&g_staging.ptr, need, cudaHostAllocPortable) != cudaSuccess) {
+            cudaGetLastError();   // not an error of the load: page-locked memory is a limited resource
+            g_staging.ptr = nullptr;
+            *no_staging = true;
+            return DSFACTO_ERR_OOM;
+        }
         g_staging.bytes = need;
     }
     char *arena = static_cast<char *>(g_staging.ptr);
@@ -901,7 +911,8 @@ int dsfacto_load_csr(dsfacto_t *h, const int64_t *indptr, const int32_t *indices
     const bool by_row_block = use_row_block_bucketer(h);
     const char *load_env = std::getenv("DSFACTO_LOAD");
     const bool streamed = by_row_block && nnz > 0 &&
-                          (nnz >= kStreamedLoadMinEntries || (load_env && std::strcmp(load_env, "stream") == 0)) &&
+                          (nnz >= kStreamedLoadMinEntries ||
+                           (load_env && (std::strcmp(load_env, "stream") == 0 || std::strcmp(load_env, "nostaging") == 0))) &&
                           !(load_env && std::strcmp(load_env, "simple") == 0);
     if (streamed) {
         try { column_blocks(h, cb); } catch (const std::bad_alloc &) { cudaStreamSynchronize(st); free_data(h); return DSFACTO_ERR_OOM; }
@@ -920,9 +931,17 @@ int dsfacto_load_csr(dsfacto_t *h, const int64_t *indptr, const int32_t *indices
         free_data(h);
         return rc;
     }
+    bool copy_from_host = !streamed;
     if (streamed) {
-        if ((rc = stream_tiles_by_row_block(h, cb, longest, indptr, indices, values))) { cudaStreamSynchronize(st); free_data(h); return rc; }
-    } else if (nnz > 0) {
+        bool no_staging = false;
+        rc = stream_tiles_by_row_block(h, cb, longest, indptr, indices, values, &no_staging);
+        if (rc && no_staging) {   // no page-locked memory to be had: bucket into pageable memory, one copy
+            rc = bucket_tiles_by_row_block(h, indptr, indices, values, ent, xw);
+            copy_from_host = true;
+        }
+        if (rc) { cudaStreamSynchronize(st); free_data(h); return rc; }
+    }
+    if (copy_from_host && nnz > 0) {
         CU_TRY(h, cudaMemcpyAsync(h->d_ent, ent.data(), sizeof(uint2) * (size_t)nnz, cudaMemcpyHostToDevice, st));
         if (h->wide) CU_TRY(h, cudaMemcpyAsync(h->d_xw, xw.data(), sizeof(float) * (size_t)nnz, cudaMemcpyHostToDevice, st));
     }

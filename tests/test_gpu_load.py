@@ -1,7 +1,9 @@
 """The three ways dsfacto_load_csr builds the tile lists on the device give the same lists, bit for
 bit, as the oracle's bucketing: the plain host bucketer, the row-block bucketer, and the streamed
 load (row blocks bucketed into page-locked staging memory and copied block by block), which large
-loads take by default and which DSFACTO_LOAD=stream forces on small ones."""
+loads take by default and which DSFACTO_LOAD=stream forces on small ones.  DSFACTO_LOAD=nostaging makes
+the streamed load behave as if no page-locked memory could be had, which must end in the row-block
+bucketer with one copy, not in an error."""
 import numpy as np
 import pytest
 
@@ -12,7 +14,7 @@ from paper_2004_13940_b200 import workloads as W
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("mode", ["stream", "simple", None])
+@pytest.mark.parametrize("mode", ["stream", "nostaging", "simple", None])
 @pytest.mark.parametrize("name,kw", [("C3", {}), ("C4s", {}), ("C4s", {"p": 200}), ("C5s", {"p": 64}), ("C2", {"p": 40}),
                                      ("C1", {"p": 2500})])
 def test_load_paths_give_the_oracle_tiles_and_epochs(monkeypatch, mode, name, kw):
