@@ -1,14 +1,15 @@
 """Parity at the size bench.py times: C4 in full (45 M rows, 1.755 G stored entries, p = 512, K = 16),
-same launch configuration as the bench.
+same launch configuration as the bench; and C5 in full (4 M rows, 400 M stored entries, p = 256,
+K = 128) the same way.
 
 The oracle cannot run a whole epoch at this size in seconds, so the comparison is on outputs it can
 compute one by one, each from the data and the seeded initial parameters alone (nothing the CUDA
 path produced is fed to it):
   * the first recompute pass: every G_i, every a_i, mean loss, sum of G and the objective, from the
     oracle's refresh routine over the full CSR;
-  * after one epoch: w0, and (w_j, v_j) of sampled columns - the hottest column (about 9 M entries,
-    present in every tile of its column block), mid-frequency and rare ones, the first and the last
-    id - from the oracle's one-column epoch, which visits that column's rows in the stratified
+  * after one epoch: w0, and (w_j, v_j) of sampled columns - for C4 the hottest column (about 9 M
+    entries, present in every tile of its column block), mid-frequency and rare ones, the first and
+    the last id - from the oracle's one-column epoch, which visits that column's rows in the stratified
     order (pinned against the full oracle epoch on small cases in tests/test_oracle_sgd.py).
 Tolerances are those of tests/test_gpu_parity.py."""
 import ctypes
@@ -33,7 +34,19 @@ def _enough_memory():
 
 @pytest.mark.skipif(not _enough_memory(), reason="needs about 110 GB of host memory")
 def test_c4_full_size_first_refresh_and_sampled_columns():
-    wl = W.make("C4")
+    _full_size_check("C4", per_row=39, popularity_rows=2_000_000, ranks=(0, 40, 2000), most_entries=None, moved=(1e-4, 1e-5))
+
+
+def test_c5_full_size_first_refresh_and_sampled_columns():
+    # the columns present in nearly every row would take the one-column oracle minutes at K = 128
+    # (it scores every row that holds the column): sample columns of up to 60 k entries.  The per-entry
+    # step of this workload is 1.25e-8, so one epoch moves a column by 1e-7 to 1e-5 only.
+    _full_size_check("C5", per_row=100, popularity_rows=400_000, ranks=(3000, 20000, 100000), most_entries=60_000,
+                     moved=(1e-7, 1e-8))
+
+
+def _full_size_check(name, per_row, popularity_rows, ranks, most_entries, moved):
+    wl = W.make(name)
     n, d, K, p = wl.n, wl.d, wl.K, wl.p
     eta_s = wl.eta / n
 
@@ -67,7 +80,7 @@ def test_c4_full_size_first_refresh_and_sampled_columns():
     assert tile_ptr[0] == 0 and tile_ptr[-1] == wl.nnz and np.all(np.diff(tile_ptr) >= 0)
     sizes = np.diff(tile_ptr).reshape(p, p)                 # [round s, row block r]
     rows_per_block = np.diff((np.arange(p + 1) * n + p - 1) // p)
-    assert np.array_equal(sizes.sum(0), rows_per_block * 39)
+    assert np.array_equal(sizes.sum(0), rows_per_block * per_row)
 
     # ---- one epoch ----
     obj0 = g.objective()
@@ -77,11 +90,12 @@ def test_c4_full_size_first_refresh_and_sampled_columns():
     g.close()
     assert w0_gpu == pytest.approx(w0 - eta_s * out3[0], rel=1e-5, abs=1e-7)
 
-    counts = np.bincount(wl.indices[: 39 * 2_000_000], minlength=d)   # popularity from the first 2 M rows
+    counts = np.bincount(wl.indices[: per_row * popularity_rows], minlength=d)   # popularity from the first rows
     order = np.argsort(-counts)
     present = order[counts[order] > 0]
-    sample = [int(present[0]), int(present[40]), int(present[2000]), int(present[len(present) // 2]),
-              int(present[-1]), 0, d - 23]
+    if most_entries is not None:
+        present = present[counts[present] * (n / popularity_rows) <= most_entries]
+    sample = [int(present[min(k, len(present) - 1)]) for k in ranks] + [int(present[len(present) // 2]), int(present[-1]), 0, d - 23]
     dw_max = dv_max = 0.0
     for j in sample:
         wj, vj, cnt = O.column_epoch(n, d, K, p, wl.loss, eta_s, wl.lambda_w, wl.lambda_v, wl.indptr, wl.indices,
@@ -93,4 +107,4 @@ def test_c4_full_size_first_refresh_and_sampled_columns():
         assert abs((w_gpu[j] - w[j]) - dw) <= 2e-3 * abs(dw) + 2e-7, (j, cnt)
         assert np.abs((V_gpu[j].astype(np.float64) - V[j]) - dv).max() <= 2e-3 * np.abs(dv).max() + 2e-7, (j, cnt)
         dw_max, dv_max = max(dw_max, abs(dw)), max(dv_max, np.abs(dv).max())
-    assert dw_max > 1e-4 and dv_max > 1e-5                  # the sampled columns did move
+    assert dw_max > moved[0] and dv_max > moved[1]          # the sampled columns did move
