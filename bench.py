@@ -34,7 +34,7 @@ UNIT = "updates/s"
 ORACLE_SAMPLE_ROWS = 1_000_000
 # dram__bytes_read.sum + dram__bytes_write.sum of sgd_chunk_kernel per stored entry, from the ncu capture
 # summarised in profiles/ (None once the kernel has changed since the counters were taken)
-SGD_DRAM_BYTES_PER_ENTRY = 19.8
+SGD_DRAM_BYTES_PER_ENTRY = 20.1
 
 
 def peaks():
