@@ -57,6 +57,7 @@ struct dsfacto {
     int4 *d_chunk_map = nullptr;
     int *d_sync = nullptr;     // ticket, error flag, per-column-block progress of the fused SGD launch
     int64_t total_chunks = 0;
+    int chunk_len = kChunk;    // entries per chunk of the stratum SGD launches
     float *d_records = nullptr, *d_Tb = nullptr, *d_Tw = nullptr;
     float4 *d_S = nullptr, *d_TS = nullptr;  // scale pairs of the scaled column state (zero outside the SGD phase)
     int *d_tile_count = nullptr;
@@ -303,14 +304,24 @@ int build_sgd_plan(dsfacto *h) {
     try {
         h->launch_ptr.assign((size_t)p + 1, 0);
         seen.assign((size_t)p, 0);
-        map.reserve((size_t)(h->nnz / kChunk + p * p / 4 + 16));
+        // Chunk length: kChunk when the data set keeps the GPU busy for many rounds of resident CTAs;
+        // otherwise the epoch is a chain of p dependent tiles per column block and is as long as p times
+        // the time one tile takes, so tiles are cut into short chunks that run side by side.
+        h->chunk_len = kChunk;
+        if (h->nnz / kChunk < (int64_t)h->sm_count * 24 * 16) h->chunk_len = std::max(128, sgd_pass_len(h->LG, h->NV));
+        if (const char *env = std::getenv("DSFACTO_CHUNK")) {
+            const int v = std::atoi(env);
+            if (v >= 16 && v <= kChunk) h->chunk_len = v;
+        }
+        const int64_t clen = h->chunk_len;
+        map.reserve((size_t)(h->nnz / clen + p * p / 4 + 16));
         for (int64_t L = 0; L < p; ++L) {
             for (int64_t k = 0; k < p; ++k) {
                 const int64_t t = L * p + k;   // slot
                 int64_t r, c;
                 slot_tile(h, t, r, c);
                 const int64_t cnt = h->tile_ptr[t + 1] - h->tile_ptr[t];
-                const int64_t nch = (cnt + kChunk - 1) / kChunk;
+                const int64_t nch = (cnt + clen - 1) / clen;
                 for (int64_t ci = 0; ci < nch; ++ci) map.push_back(make_int4((int)t, (int)ci, seen[c], 0));
                 if (nch > 0) seen[c] += 1;
             }
@@ -349,6 +360,7 @@ void run_sgd_phase(dsfacto *h, int64_t L0, int64_t L1) {
     a.chunk_map = h->d_chunk_map;
     a.sync = h->d_sync;
     a.chunk_base = (int)h->launch_ptr[(size_t)L0];
+    a.chunk_len = h->chunk_len;
     const int64_t chunks = h->launch_ptr[(size_t)L1] - h->launch_ptr[(size_t)L0];
     if (chunks > 0) {
         DSF_DISPATCH(h, launch_sgd, h, a, (int)chunks);

@@ -27,7 +27,7 @@ namespace dsf {
 constexpr int kSgdThreads = 32;   // one warp per CTA: a finished warp frees its registers and shared memory at once
 constexpr int kSgdWarps = kSgdThreads / 32;
 constexpr int kWarpEntries = 512;                 // entries per warp
-constexpr int kChunk = kSgdWarps * kWarpEntries;  // entries per CTA
+constexpr int kChunk = kSgdWarps * kWarpEntries;  // entries per CTA, at most (a launch may use shorter chunks)
 constexpr int kSgdSpinLimit = 1 << 22;            // polls (about 100 ns each) before a dependency wait gives up
 // Words of the launch's synchronisation array.  The ticket counter takes one atomic per CTA and the
 // progress counters are polled by waiting CTAs, so every word sits in a 128-byte line of its own.
@@ -283,6 +283,8 @@ struct SgdChunkArgs {
                                // the launches of one sweep)
     int p, jbits, sweep;
     int chunk_base;            // first chunk of this launch in chunk_map (a launch may cover a range of rounds)
+    int chunk_len;             // entries per chunk, <= kChunk: short chunks for small data sets, whose epoch is a
+                               // chain of dependent tiles and is as long as p times the time one tile takes
     float h, lambda_w, lambda_v;
 };
 
@@ -325,8 +327,8 @@ __global__ void __launch_bounds__(kSgdThreads, sgd_min_ctas(LG, NV)) sgd_chunk_k
     else { r = (int)(t % a.p); c = (r + (int)(t / a.p)) % a.p; }
     const bool tail_mode = a.sweep == 1 && r > c;
     const int64_t tb = a.tile_ptr[t], te = a.tile_ptr[t + 1];
-    const int64_t cb = tb + (int64_t)cm.y * kChunk;
-    const int64_t ce = (cb + kChunk < te) ? cb + kChunk : te;
+    const int64_t cb = tb + (int64_t)cm.y * a.chunk_len;
+    const int64_t ce = (cb + a.chunk_len < te) ? cb + a.chunk_len : te;
     const int64_t wb = cb + (int64_t)warp * kWarpEntries;
     const int64_t we = (wb + kWarpEntries < ce) ? wb + kWarpEntries : ce;
     const int64_t row0 = a.row_start[r];
@@ -637,7 +639,7 @@ __global__ void __launch_bounds__(kSgdThreads, sgd_min_ctas(LG, NV)) sgd_chunk_k
     if (warp != 0) return;
 
     // ---------------- chunk phase: warp 0 joins the warps ----------------
-    const int nchunks = (int)((te - tb + kChunk - 1) / kChunk);
+    const int nchunks = (int)((te - tb + a.chunk_len - 1) / a.chunk_len);
     C ccarry;
     comp_identity(ccarry);
     bool cflag = false;
