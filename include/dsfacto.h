@@ -161,7 +161,8 @@ int dsfacto_set_stream(dsfacto_t *h, void *cuda_stream);
 
 /* Device time of the last dsfacto_epoch from CUDA events on the handle's stream, in milliseconds:
  * ms[0] whole epoch, ms[1] the p strata (update loop), ms[2] recompute pass (refresh + residual +
- * loss sums), ms[3] parameter norms + final reduction. */
+ * loss sums), ms[3] parameter norms + final reduction.  With dsfacto_set_refresh_every each figure is
+ * the sum over the segments of the epoch. */
 int dsfacto_last_epoch_ms(dsfacto_t *h, float ms[4]);
 
 /* Number of kernels this handle has launched since creation. */
