@@ -269,3 +269,20 @@ def test_status_codes_on_device():
     rcs = [D.dsfacto_epoch(g._h) for _ in range(12)]
     assert D.ERR_DIVERGED in rcs and all(rc in (D.OK, D.ERR_DIVERGED) for rc in rcs)
     g.close()
+
+
+@pytest.mark.parametrize("chunk", [16, 100, 200, 512])
+@pytest.mark.parametrize("name", ["C3", "C4s", "C5s"])
+def test_any_chunk_length_gives_the_same_epoch(monkeypatch, name, chunk):
+    # the chunk length of the stratum SGD launches is a tuning parameter (DSFACTO_CHUNK overrides the
+    # choice made at load time): whole passes, partial passes and chunks shorter than a pass must all
+    # reproduce the oracle's epoch
+    monkeypatch.setenv("DSFACTO_CHUNK", str(chunk))
+    wl = W.make(name)
+    o, g = make_pair(wl)
+    for _ in range(2):
+        before = (o.w0, o.w.copy(), o.V.copy())
+        want, got = o.epoch(), g.epoch()
+        assert got == pytest.approx(want, rel=1e-4)
+        check_params(o, g, before)
+    g.close()
