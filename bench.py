@@ -101,23 +101,6 @@ class ClockSampler:
                 "samples": len(sm), "window": window, "reasons": reasons}
 
 
-def gather_ceiling(K):
-    """Rows per second of the stand-alone gather micro-benchmark for the row size nearest to 4K bytes."""
-    try:
-        from paper_2004_13940_b200 import build as B
-        out = subprocess.run([str(B.build_tools())], capture_output=True, text=True, timeout=120).stdout
-        want = "K=16, all of V" if K <= 32 else "K=128, all of V"
-        for line in out.splitlines():
-            if line.startswith(want):
-                parts = line.split()
-                return {"table": want, "gathered_GBps": float(parts[parts.index("GB/s") - 1]),
-                        "rows_per_s": float(parts[parts.index("G") - 1]) * 1e9,
-                        "what": "uniformly random rows, ld.global.cg, nothing else (csrc/tools/gather_ceiling.cu)"}
-    except Exception as exc:   # the number is context only
-        return {"error": str(exc)}
-    return None
-
-
 def oracle_leg(wl_name: str, rows: int, min_seconds: float, max_epochs: int):
     """Times oracle epochs (as the oracle stands) on the first `rows` rows' worth of the workload."""
     from oracle import dsfacto_oracle as O
@@ -325,9 +308,6 @@ def run_ours(args):
                              "frac": sgd_gather / sgd_s / 1e9 / peak},
             "refresh_kernel": {"algorithmic_bytes_per_step": ref_bytes, "ms": phase[2],
                                "achieved": ref_bytes / ref_s / 1e9, "frac": ref_bytes / ref_s / 1e9 / peak}}
-    # context for the fraction above: what a pure gather of L2-resident factor rows reaches on this device
-    # (the access both hot kernels are made of), measured now by the package's micro-benchmark
-    roof["gather_ceiling"] = gather_ceiling(K) if (world == 1 and not args.no_gather_ceiling and not args.no_cpu_baseline) else None
     value = whole_job_rate(world, nnz, args.steps, ms)
     h2d = (wl.indptr.nbytes + wl.indices.nbytes + wl.values.nbytes + wl.y.nbytes + 8 * nnz + 8 * (p * p + 1))
     e2e = {"value": whole_job_rate(world, nnz, args.e2e_steps, e2e_ms) if args.e2e_steps > 0 else None, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
@@ -368,7 +348,6 @@ def main():
     ap.add_argument("--oracle-seconds", type=float, default=10.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-pin", dest="pin", action="store_false")
-    ap.add_argument("--no-gather-ceiling", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

@@ -301,12 +301,10 @@ int64_t oracle_column_epoch(int64_t n, int32_t d, int32_t K, int32_t p, int32_t 
  * out2[0] = (1/m) sum_i l(f_i, y_i) with the loss of the model;
  * out2[1] = sqrt((1/m) sum_i (f_i - y_i)^2)          for the squared loss (RMSE),
  *         = (1/m) #{ i : y_i f_i > 0 }                for the logistic loss (accuracy; the predicted
- *           class is the sign of the score, and a score of exactly 0 predicts neither class).
- * With decide_in_fp32 != 0 the sign test is taken on the score rounded to fp32, the precision in
- * which the CUDA path holds its scores. */
+ *           class is the sign of the score, and a score of exactly 0 predicts neither class). */
 void oracle_evaluate(int64_t m, int32_t K, int32_t loss, const int64_t *indptr, const int32_t *indices,
                      const float *values, const float *y, double w0, const double *w, const double *V,
-                     int32_t decide_in_fp32, double *out2) {
+                     double *out2) {
     double suml = 0.0, sumsq = 0.0, correct = 0.0;
     double *a = (double *)malloc(sizeof(double) * (size_t)(K > 0 ? K : 1));
     for (int64_t i = 0; i < m; ++i) {
@@ -315,8 +313,7 @@ void oracle_evaluate(int64_t m, int32_t K, int32_t loss, const int64_t *indptr, 
         const double yi = (double)y[i];
         suml += loss_value(loss, f, yi);
         sumsq += (f - yi) * (f - yi);
-        const double fd = decide_in_fp32 ? (double)(float)f : f;
-        if (yi * fd > 0.0) correct += 1.0;
+        if (yi * f > 0.0) correct += 1.0;
     }
     free(a);
     out2[0] = m > 0 ? suml / (double)m : 0.0;

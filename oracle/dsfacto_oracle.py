@@ -77,7 +77,7 @@ def score(indptr, indices, values, w0, w, V):
     return out
 
 
-def evaluate(loss, indptr, indices, values, y, w0, w, V, decide_in_fp32=True):
+def evaluate(loss, indptr, indices, values, y, w0, w, V):
     """Held-out mean loss and RMSE (squared loss) or accuracy (logistic loss) of the scores."""
     indptr = np.ascontiguousarray(indptr, np.int64)
     indices = np.ascontiguousarray(indices, np.int32)
@@ -85,7 +85,7 @@ def evaluate(loss, indptr, indices, values, y, w0, w, V, decide_in_fp32=True):
     y = np.ascontiguousarray(y, np.float32)
     out = np.zeros(2, np.float64)
     lib().oracle_evaluate(_i64(len(indptr) - 1), _i32(V.shape[1]), _i32(loss), _p(indptr), _p(indices), _p(values),
-                          _p(y), _f64(w0), _p(w), _p(V), _i32(1 if decide_in_fp32 else 0), _p(out))
+                          _p(y), _f64(w0), _p(w), _p(V), _p(out))
     return float(out[0]), float(out[1])
 
 
@@ -180,8 +180,8 @@ class Oracle:
         return score(np.ascontiguousarray(indptr, np.int64), np.ascontiguousarray(indices, np.int32),
                      np.ascontiguousarray(values, np.float32), self.w0, self.w, self.V)
 
-    def evaluate(self, indptr, indices, values, y, decide_in_fp32=True):
-        return evaluate(self.loss, indptr, indices, values, y, self.w0, self.w, self.V, decide_in_fp32)
+    def evaluate(self, indptr, indices, values, y):
+        return evaluate(self.loss, indptr, indices, values, y, self.w0, self.w, self.V)
 
     def set_eta(self, eta):
         """New learning rate for the following epochs (step-size schedules are the caller's)."""

@@ -16,7 +16,6 @@ INCLUDE = ROOT / "include"
 
 LIB_CUDA = PKG / "libdsfacto.so"
 LIB_WORKLOADS = PKG / "_workloads_gen.so"
-BIN_GATHER = PKG / "gather_ceiling.bin"
 
 NVCC_ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 
@@ -64,17 +63,6 @@ def build_workloads(force: bool = False) -> Path:
     return LIB_WORKLOADS
 
 
-def build_tools(force: bool = False) -> Path:
-    """The stand-alone gather micro-benchmark (csrc/tools/gather_ceiling.cu)."""
-    src = CSRC / "tools" / "gather_ceiling.cu"
-    if force or _stale(BIN_GATHER, [src]):
-        tmp = BIN_GATHER.with_suffix(".bin.tmp%d" % os.getpid())
-        _run([_nvcc(), "-O3", "-std=c++17", "-lineinfo", *NVCC_ARCH, "-o", tmp, src])
-        os.replace(tmp, BIN_GATHER)
-    return BIN_GATHER
-
-
 def build_all(force: bool = False) -> None:
     build_workloads(force)
     build_cuda(force)
-    build_tools(force)

@@ -143,7 +143,7 @@ def test_heldout_evaluation_matches_library_metrics(loss):
         assert O.evaluate(loss, indptr, indices, vals, y2, w0, w, V)[1] != pytest.approx(rmse, rel=1e-6)
     else:
         y = np.where(rng.random(n) < 0.5, 1.0, -1.0).astype(np.float32)
-        mean_loss, acc = O.evaluate(loss, indptr, indices, vals, y, w0, w, V, decide_in_fp32=False)
+        mean_loss, acc = O.evaluate(loss, indptr, indices, vals, y, w0, w, V)
         assert acc == pytest.approx(accuracy_score(y, np.where(f > 0, 1.0, -1.0)), abs=1e-15)
         prob = 1.0 / (1.0 + np.exp(-f))                                    # P(y = +1 | x) under the logistic model
         assert mean_loss == pytest.approx(log_loss(y, prob, labels=[-1.0, 1.0]), rel=1e-10)
