@@ -34,7 +34,7 @@ UNIT = "updates/s"
 ORACLE_SAMPLE_ROWS = 1_000_000
 # dram__bytes_read.sum + dram__bytes_write.sum of sgd_chunk_kernel per stored entry, from the ncu capture
 # summarised in profiles/ (None once the kernel has changed since the counters were taken)
-SGD_DRAM_BYTES_PER_ENTRY = 20.1
+SGD_DRAM_BYTES_PER_ENTRY = None
 
 
 def peaks():
@@ -298,7 +298,7 @@ def run_ours(args):
     sgd_s, ref_s = phase[1] * 1e-3, phase[2] * 1e-3
     # the counters were taken on the default schedule (row-block sweep, one launch per sweep)
     traffic = None if (SGD_DRAM_BYTES_PER_ENTRY is None or sweep != "rowblock") else SGD_DRAM_BYTES_PER_ENTRY * nnz
-    roof = {"bound": "hbm", "kernel": "sgd_chunk_kernel", "launches_per_step": segments, "sweep": sweep,
+    roof = {"bound": "hbm", "kernel": "sgd_sweep_kernel", "launches_per_step": segments, "sweep": sweep,
             "achieved": sgd_bytes / sgd_s / 1e9, "peak": peak, "unit": "GB/s", "frac": sgd_bytes / sgd_s / 1e9 / peak,
             "peak_kind": "of " + peak_kind, "traffic": traffic,
             "algorithmic_bytes_per_launch": sgd_bytes / segments, "avg_launch_us": 1e6 * sgd_s / segments,

@@ -54,13 +54,18 @@ struct dsfacto {
     int sweep = 1;  // 1: a launch is a row block (p-1 .. 0); 0: a launch is an inner round (0 .. p-1)
     int refresh_every = 0;  // > 0: G, A recomputed after every that many inner rounds (needs the round sweep)
     std::vector<int64_t> launch_ptr;
-    int4 *d_chunk_map = nullptr;
-    int *d_sync = nullptr;     // ticket, error flag, per-column-block progress of the fused SGD launch
-    int64_t total_chunks = 0;
-    int chunk_len = kChunk;    // entries per chunk of the stratum SGD launches
+    ChunkDesc *d_desc = nullptr;   // chunk descriptors in sweep order
+    int *d_sync = nullptr;     // ticket, error word, per-column-block progress of the fused SGD launch
+    int64_t total_chunks = 0, long_runs = 0, slice_records = 0;
+    int chunk_len = kChunkMax;  // most entries a chunk of the stratum SGD launches holds
+    int chunk_override = 0;     // > 0: chunk length forced by dsfacto_debug_set (tests)
+    int sgd_grid = 0;           // CTAs of the persistent stratum SGD launch
+    int spin_limit = kSgdSpinLimit;  // polls before a wait for an earlier tile gives up
+    int debug_extra_need = 0;   // tests: added to the `need` of the first chunk, so that its wait runs out
+    bool failed = false;        // an SGD launch gave up; the parameters are unusable until they are set again
     float *d_records = nullptr, *d_Tb = nullptr, *d_Tw = nullptr;
-    float4 *d_S = nullptr, *d_TS = nullptr;  // scale pairs of the scaled column state (zero outside the SGD phase)
-    int *d_tile_count = nullptr;
+    float2 *d_S = nullptr, *d_TS = nullptr;  // scale records of the scaled column state (zero outside the SGD phase)
+    int *d_tile_count = nullptr, *d_run_count = nullptr;
     int refresh_grid = 0, norm_grid = 0;
 
     double loss_sum = 0, g_sum = 0, w2 = 0, v2 = 0, objective = 0;
@@ -227,7 +232,8 @@ void unpack_tiles(const dsfacto *h, const std::vector<int64_t> &canon_ptr, const
 void free_data(dsfacto *h) {
     dev_free(h->d_A); dev_free(h->d_G); dev_free(h->d_y); dev_free(h->d_val); dev_free(h->d_xw);
     dev_free(h->d_indptr); dev_free(h->d_tile_ptr); dev_free(h->d_idx); dev_free(h->d_ent);
-    dev_free(h->d_partials); dev_free(h->d_chunk_map); dev_free(h->d_records); dev_free(h->d_tile_count); dev_free(h->d_sync);
+    dev_free(h->d_partials); dev_free(h->d_desc); dev_free(h->d_records); dev_free(h->d_tile_count); dev_free(h->d_run_count);
+    dev_free(h->d_sync);
     h->launch_ptr.clear();
     h->loaded = false;
     h->nnz = 0;
@@ -237,16 +243,27 @@ void free_data(dsfacto *h) {
 // kernel dispatch over the factor-row layout
 // ---------------------------------------------------------------------------------------------
 template <int LG, int NV>
-void launch_sgd(dsfacto *h, const SgdChunkArgs &a, int grid) {
-    constexpr int bytes = SgdSmem<LG, NV>::BYTES;
-    static bool opted_in = false;  // more than 48 KB of dynamic shared memory needs an opt-in per kernel
-    if (!opted_in) {
-        cudaFuncSetAttribute(sgd_chunk_kernel<LG, NV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-        cudaFuncSetAttribute(sgd_chunk_kernel<LG, NV, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-        opted_in = true;
+void launch_sgd(dsfacto *h, const SgdArgs &a, int64_t chunks) {
+    const size_t bytes = (size_t)kSgdWarps * sgd_warp_smem<LG, NV>(h->wide, h->chunk_len);
+    // The launch is persistent: as many CTAs as stay resident (fewer if there are fewer chunks), each warp
+    // taking chunks from the ticket counter until none is left.  More than 48 KB of dynamic shared memory
+    // needs an opt-in per kernel; the residency depends on the chunk length, so both are redone per load.
+    if (h->sgd_grid == 0) {
+        int per_sm = 0;
+        if (h->wide) {
+            cudaFuncSetAttribute(sgd_sweep_kernel<LG, NV, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sgd_sweep_kernel<LG, NV, true>, kSgdThreads, bytes);
+        } else {
+            cudaFuncSetAttribute(sgd_sweep_kernel<LG, NV, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sgd_sweep_kernel<LG, NV, false>, kSgdThreads, bytes);
+        }
+        if (per_sm < 1) per_sm = 1;
+        h->sgd_grid = h->sm_count * per_sm;
     }
-    if (h->wide) sgd_chunk_kernel<LG, NV, true><<<grid, kSgdThreads, bytes, h->stream>>>(a);
-    else sgd_chunk_kernel<LG, NV, false><<<grid, kSgdThreads, bytes, h->stream>>>(a);
+    const int64_t want = (chunks + kSgdWarps - 1) / kSgdWarps;
+    const int grid = (int)std::min<int64_t>(h->sgd_grid, std::max<int64_t>(want, 1));
+    if (h->wide) sgd_sweep_kernel<LG, NV, true><<<grid, kSgdThreads, bytes, h->stream>>>(a);
+    else sgd_sweep_kernel<LG, NV, false><<<grid, kSgdThreads, bytes, h->stream>>>(a);
 }
 template <int LG, int NV>
 void launch_refresh(dsfacto *h, const RefreshArgs &a, int mode, int grid) {
@@ -295,49 +312,157 @@ int refresh_grid_for(const dsfacto *h, int64_t rows) {
     return (int)want;
 }
 
-// Launch plan of the stratum SGD phase: which tiles each launch covers and how they split into
-// chunks of kChunk entries.  Tiles of one launch have pairwise disjoint column blocks.
-int build_sgd_plan(dsfacto *h) {
-    const int64_t p = h->p;
-    std::vector<int4> map;
-    std::vector<int> seen;  // non-empty tiles met so far per column block
+// ---------------------------------------------------------------------------------------------
+// Launch plan of the stratum SGD phase.  While a tile is bucketed its column counts are at hand, and
+// the tile is cut into chunks right there: whole runs (all entries of one column inside the tile) are
+// packed greedily into chunks of at most chunk_len entries, and a run longer than that becomes slices
+// of its own.  The per-tile pieces are put in sweep order afterwards (finish_sgd_plan).
+// ---------------------------------------------------------------------------------------------
+struct TilePlanner {          // one per host thread
+    std::vector<ChunkDesc> descs;
+    bool failed = false;      // out of host memory
+};
+struct TileDescRef {          // where the chunks of a tile sit
+    int32_t owner = 0, count = 0;
+    int64_t first = 0;
+};
+struct SgdPlanBuild {
+    std::vector<TilePlanner> planners;
+    std::vector<TileDescRef> refs;   // per tile slot
+};
+
+// Chunk length: kChunkMax when the data set keeps the GPU busy for many rounds of resident warps;
+// otherwise the epoch is a chain of p dependent tiles per column block and is as long as p times the
+// time one tile takes, so tiles are cut into short chunks that run side by side.
+void choose_chunk_len(dsfacto *h, int64_t nnz) {
+    h->chunk_len = kChunkMax;
+    if (nnz / kChunkMax < (int64_t)h->sm_count * 24 * 16) h->chunk_len = 128;
+    if (h->chunk_override > 0) h->chunk_len = h->chunk_override;
+    if (const char *env = std::getenv("DSFACTO_CHUNK")) {
+        const int v = std::atoi(env);
+        if (v >= 16 && v <= kChunkMax) h->chunk_len = v;
+    }
+    h->sgd_grid = 0;   // residency is recomputed at the next launch
+}
+
+// col_end[j] = number of entries of the tile whose local column is <= j; tile_begin = position of the
+// tile's first entry in the entry array
+void plan_tile(const dsfacto *h, SgdPlanBuild *pb, int owner, int64_t slot, int64_t tile_begin, const int64_t *col_end,
+               int64_t width) {
+    if (!pb) return;
+    TilePlanner &tp = pb->planners[(size_t)owner];
+    const int64_t L = h->chunk_len;
+    const size_t first = tp.descs.size();
+    try {
+        auto emit = [&](int64_t off, int64_t len, int flags, int64_t jl, int64_t slice, int64_t nslices) {
+            ChunkDesc d{};
+            d.ent_off = tile_begin + off;
+            d.len = (int32_t)len;
+            d.flags = flags;
+            d.jl = (int32_t)jl;
+            d.slice = (int32_t)slice;
+            d.nslices = (int32_t)nslices;
+            tp.descs.push_back(d);
+        };
+        int64_t cur0 = 0, cur = 0, prev = 0;   // open chunk of whole runs [cur0, cur0 + cur); end of the last column
+        for (int64_t j = 0; j < width; ++j) {
+            const int64_t end = col_end[j], len = end - prev;
+            if (len == 0) continue;
+            if (len > L) {
+                if (cur > 0) emit(cur0, cur, 0, 0, 0, 0);
+                cur = 0;
+                int64_t ns = (len + L - 1) / L;
+                int64_t per = ((len + ns - 1) / ns + 31) & ~(int64_t)31;   // slices of whole passes, about equal
+                if (per > L) per = L;
+                ns = (len + per - 1) / per;
+                for (int64_t k = 0; k < ns; ++k)
+                    emit(prev + k * per, std::min(per, len - k * per), kChunkSlice, j, k, ns);
+            } else if (cur + len > L) {
+                emit(cur0, cur, 0, 0, 0, 0);
+                cur0 = prev;
+                cur = len;
+            } else {
+                if (cur == 0) cur0 = prev;
+                cur += len;
+            }
+            prev = end;
+        }
+        if (cur > 0) emit(cur0, cur, 0, 0, 0, 0);
+    } catch (const std::bad_alloc &) {
+        tp.failed = true;
+        return;
+    }
+    TileDescRef &ref = pb->refs[(size_t)slot];
+    ref.owner = owner;
+    ref.first = (int64_t)first;
+    ref.count = (int32_t)(tp.descs.size() - first);
+}
+
+bool init_plan_build(const dsfacto *h, SgdPlanBuild &pb, int threads) {
+    try {
+        pb.planners.assign((size_t)std::max(threads, 1), TilePlanner());
+        pb.refs.assign((size_t)h->p * h->p, TileDescRef());
+    } catch (const std::bad_alloc &) { return false; }
+    return true;
+}
+
+// Puts the chunks in sweep order, fills in what depends on it (earlier tiles of the column block, run
+// and record numbers, launch ranges) and copies the plan to the device.
+int finish_sgd_plan(dsfacto *h, SgdPlanBuild &pb) {
+    const int64_t p = h->p, nt = p * p;
+    for (const TilePlanner &tp : pb.planners)
+        if (tp.failed) return DSFACTO_ERR_OOM;
+    int64_t total = 0;
+    for (int64_t t = 0; t < nt; ++t) total += pb.refs[(size_t)t].count;
+    if (total >= (int64_t)kTicketStop / 2) return DSFACTO_ERR_INVALID_ARG;
+    HostBuf<ChunkDesc> all;
+    std::vector<int> seen;   // non-empty tiles met so far per column block
+    if (!all.alloc((size_t)total)) return DSFACTO_ERR_OOM;
     try {
         h->launch_ptr.assign((size_t)p + 1, 0);
         seen.assign((size_t)p, 0);
-        // Chunk length: kChunk when the data set keeps the GPU busy for many rounds of resident CTAs;
-        // otherwise the epoch is a chain of p dependent tiles per column block and is as long as p times
-        // the time one tile takes, so tiles are cut into short chunks that run side by side.
-        h->chunk_len = kChunk;
-        if (h->nnz / kChunk < (int64_t)h->sm_count * 24 * 16) h->chunk_len = std::max(128, sgd_pass_len(h->LG, h->NV));
-        if (const char *env = std::getenv("DSFACTO_CHUNK")) {
-            const int v = std::atoi(env);
-            if (v >= 16 && v <= kChunk) h->chunk_len = v;
-        }
-        const int64_t clen = h->chunk_len;
-        map.reserve((size_t)(h->nnz / clen + p * p / 4 + 16));
-        for (int64_t L = 0; L < p; ++L) {
-            for (int64_t k = 0; k < p; ++k) {
-                const int64_t t = L * p + k;   // slot
-                int64_t r, c;
-                slot_tile(h, t, r, c);
-                const int64_t cnt = h->tile_ptr[t + 1] - h->tile_ptr[t];
-                const int64_t nch = (cnt + clen - 1) / clen;
-                for (int64_t ci = 0; ci < nch; ++ci) map.push_back(make_int4((int)t, (int)ci, seen[c], 0));
-                if (nch > 0) seen[c] += 1;
-            }
-            h->launch_ptr[L + 1] = (int64_t)map.size();
-        }
     } catch (const std::bad_alloc &) { return DSFACTO_ERR_OOM; }
-    if (map.size() >= ((size_t)1 << 31)) return DSFACTO_ERR_INVALID_ARG;
-    h->total_chunks = (int64_t)map.size();
+    int64_t pos = 0, runs = 0, recs = 0, cur_run = 0, cur_rec0 = 0;
+    for (int64_t slot = 0; slot < nt; ++slot) {
+        int64_t r, c;
+        slot_tile(h, slot, r, c);
+        const TileDescRef &ref = pb.refs[(size_t)slot];
+        const bool tail = h->sweep == 1 && r > c;
+        for (int32_t q = 0; q < ref.count; ++q) {
+            ChunkDesc d = pb.planners[(size_t)ref.owner].descs[(size_t)(ref.first + q)];
+            d.row0 = (int32_t)h->row_start[(size_t)r];
+            d.col0 = h->col_start[(size_t)c];
+            d.cblock = (int32_t)c;
+            d.need = seen[(size_t)c];
+            d.tile = (int32_t)slot;
+            d.nchunks = ref.count;
+            if (tail) d.flags |= kChunkTail;
+            if (d.flags & kChunkSlice) {
+                if (d.slice == 0) { cur_run = runs++; cur_rec0 = recs; recs += d.nslices; }
+                d.run_id = (int32_t)cur_run;
+                d.rec0 = (int32_t)cur_rec0;
+            }
+            all[(size_t)pos++] = d;
+        }
+        if (ref.count > 0) seen[(size_t)c] += 1;
+        if ((slot + 1) % p == 0) h->launch_ptr[(size_t)((slot + 1) / p)] = pos;
+    }
+    if (recs >= ((int64_t)1 << 31)) return DSFACTO_ERR_INVALID_ARG;
+    h->total_chunks = total;
+    h->long_runs = runs;
+    h->slice_records = recs;
+    if (h->debug_extra_need > 0 && total > 0) all[0].need += h->debug_extra_need;
     int rc;
-    if ((rc = dev_alloc(h, &h->d_chunk_map, map.size())) ||
-        (rc = dev_alloc(h, &h->d_records, map.size() * chunk_record_floats(h->Kp))) ||
-        (rc = dev_alloc(h, &h->d_tile_count, (size_t)(p * p))) || (rc = dev_alloc(h, &h->d_sync, sync_words((int)p))))
+    if ((rc = dev_alloc(h, &h->d_desc, (size_t)total)) ||
+        (rc = dev_alloc(h, &h->d_records, (size_t)recs * slice_record_floats(h->Kp))) ||
+        (rc = dev_alloc(h, &h->d_run_count, (size_t)runs)) || (rc = dev_alloc(h, &h->d_tile_count, (size_t)nt)) ||
+        (rc = dev_alloc(h, &h->d_sync, sync_words((int)p))))
         return rc;
-    CU_TRY(h, cudaMemsetAsync(h->d_tile_count, 0, sizeof(int) * (size_t)(p * p), h->stream));
-    if (!map.empty())
-        CU_TRY(h, cudaMemcpyAsync(h->d_chunk_map, map.data(), sizeof(int4) * map.size(), cudaMemcpyHostToDevice, h->stream));
+    CU_TRY(h, cudaMemsetAsync(h->d_tile_count, 0, sizeof(int) * (size_t)nt, h->stream));
+    CU_TRY(h, cudaMemsetAsync(h->d_run_count, 0, sizeof(int) * (size_t)std::max<int64_t>(runs, 1), h->stream));
+    CU_TRY(h, cudaMemsetAsync(h->d_sync, 0, sizeof(int) * sync_words((int)p), h->stream));
+    if (total > 0)
+        CU_TRY(h, cudaMemcpyAsync(h->d_desc, all.data(), sizeof(ChunkDesc) * (size_t)total, cudaMemcpyHostToDevice, h->stream));
     CU_TRY(h, cudaStreamSynchronize(h->stream));
     return DSFACTO_OK;
 }
@@ -345,31 +470,33 @@ int build_sgd_plan(dsfacto *h) {
 // The strata [L0, L1) of one epoch (inner rounds for the round sweep, row blocks for the row-block
 // sweep; the whole sweep is [0, p)), then the return from the scaled state to plain parameters.
 void run_sgd_phase(dsfacto *h, int64_t L0, int64_t L1) {
-    SgdChunkArgs a{};
-    a.tile_ptr = h->d_tile_ptr; a.ent = h->d_ent; a.xw = h->d_xw; a.row_start = h->d_row_start;
-    a.col_start = h->d_col_start; a.A = h->d_A; a.G = h->d_G; a.w = h->d_w; a.V = h->d_V;
-    a.S = h->d_S; a.Tb = h->d_Tb; a.Tw = h->d_Tw; a.TS = h->d_TS; a.records = h->d_records; a.tile_count = h->d_tile_count;
-    a.p = h->p; a.jbits = h->jbits; a.sweep = h->sweep;
-    a.h = h->h; a.lambda_w = h->lambda_w; a.lambda_v = h->lambda_v;
+    SgdArgs a{};
+    a.ent = h->d_ent; a.xw = h->d_xw; a.A = h->d_A; a.G = h->d_G; a.w = h->d_w; a.V = h->d_V;
+    a.S = h->d_S; a.Tb = h->d_Tb; a.Tw = h->d_Tw; a.TS = h->d_TS; a.records = h->d_records;
+    a.tile_count = h->d_tile_count; a.run_count = h->d_run_count;
+    a.jbits = h->jbits; a.chunk_len = h->chunk_len; a.spin_limit = h->spin_limit;
+    a.h = h->h; a.lambda_v = h->lambda_v;
+    const double ew = (double)h->h * (double)h->lambda_w;
+    const double log1m_ew = std::log1p(-ew);           // log(1 - ew); -inf / NaN for absurd steps, which then diverge
+    a.kappa_w = (float)(-log1m_ew / std::log(2.0));
     // One launch for the whole range: chunks are taken in sweep order (row block by row block, or round
     // by round) and a tile waits only for the earlier tiles of its own column block.  The counters of
     // finished tiles are cumulative over the sweep, so they are cleared at its first launch only; the
     // ticket counter restarts with every launch.
     if (L0 == 0) cudaMemsetAsync(h->d_sync, 0, sizeof(int) * sync_words(h->p), h->stream);
     else cudaMemsetAsync(h->d_sync + kSyncTicket, 0, sizeof(int), h->stream);
-    a.chunk_map = h->d_chunk_map;
     a.sync = h->d_sync;
-    a.chunk_base = (int)h->launch_ptr[(size_t)L0];
-    a.chunk_len = h->chunk_len;
     const int64_t chunks = h->launch_ptr[(size_t)L1] - h->launch_ptr[(size_t)L0];
+    a.desc = h->d_desc + h->launch_ptr[(size_t)L0];
+    a.nchunks = (int)chunks;
     if (chunks > 0) {
-        DSF_DISPATCH(h, launch_sgd, h, a, (int)chunks);
+        DSF_DISPATCH(h, launch_sgd, h, a, chunks);
         h->launches += 1;
     }
     {   // back from the scaled state to plain (w, V); folds the tail composites in after a row-block sweep
         const int grid = h->sm_count * 8;
         sgd_finalize_v_kernel<<<grid, kThreads, 0, h->stream>>>(h->d_V, h->d_Tb, h->d_S, h->d_TS, h->d, h->Kp / 4);
-        sgd_finalize_w_kernel<<<grid, kThreads, 0, h->stream>>>(h->d_w, h->d_Tw, h->d_S, h->d_TS, h->d);
+        sgd_finalize_w_kernel<<<grid, kThreads, 0, h->stream>>>(h->d_w, h->d_Tw, h->d_S, h->d_TS, h->d, log1m_ew);
         h->launches += 2;
     }
 }
@@ -446,7 +573,7 @@ int validate_csr(int64_t m, int32_t d, const int64_t *indptr, const int32_t *ind
 // by local column inside every tile.
 // ---------------------------------------------------------------------------------------------
 int bucket_tiles(dsfacto *h, const int64_t *indptr, const int32_t *indices, const float *values,
-                 HostBuf<uint2> &ent, HostBuf<float> &xw) {
+                 HostBuf<uint2> &ent, HostBuf<float> &xw, SgdPlanBuild *pb) {
     const int64_t n = h->n, nnz = indptr[n];
     const int32_t d = h->d, p = h->p;
     const int64_t nt = (int64_t)p * p;
@@ -560,6 +687,7 @@ int bucket_tiles(dsfacto *h, const int64_t *indptr, const int32_t *indices, cons
                 ent[at] = tmp_e[q];
                 if (wide) xw[at] = tmp_x[q];
             }
+            plan_tile(h, pb, omp_get_thread_num(), t, b, hist.data(), width);   // hist[j] is now the end of column j
         }
     }
     return DSFACTO_OK;
@@ -576,6 +704,8 @@ struct RowBlockScratch {
     HostBuf<uint2> tmp_e;
     HostBuf<float> tmp_x;
     std::vector<int64_t> fill, hist;
+    SgdPlanBuild *plan = nullptr;   // where the chunks of the bucketed tiles go (none: bucketing only)
+    int owner = 0;                  // this thread's planner
 };
 
 bool use_row_block_bucketer(const dsfacto *h) {
@@ -647,6 +777,7 @@ void bucket_row_block(const dsfacto *h, int64_t r, const std::vector<int32_t> &c
             out_e[at] = tmp_e[q];
             if (wide) out_x[at] = tmp_x[q];
         }
+        plan_tile(h, sc.plan, sc.owner, (p - 1 - r) * p + c, tp[c], sc.hist.data(), width);   // hist[j]: end of column j
     }
 }
 
@@ -657,7 +788,7 @@ bool alloc_row_block_scratch(const dsfacto *h, RowBlockScratch &sc, int64_t long
 
 // host-only form: the whole entry array in host memory
 int bucket_tiles_by_row_block(dsfacto *h, const int64_t *indptr, const int32_t *indices, const float *values,
-                              HostBuf<uint2> &ent, HostBuf<float> &xw) {
+                              HostBuf<uint2> &ent, HostBuf<float> &xw, SgdPlanBuild *pb) {
     const int64_t nnz = indptr[h->n];
     std::vector<int32_t> cb;
     try { column_blocks(h, cb); } catch (const std::bad_alloc &) { return DSFACTO_ERR_OOM; }
@@ -667,6 +798,8 @@ int bucket_tiles_by_row_block(dsfacto *h, const int64_t *indptr, const int32_t *
 #pragma omp parallel
     {
         RowBlockScratch sc;
+        sc.plan = pb;
+        sc.owner = omp_get_thread_num();
         if (!alloc_row_block_scratch(h, sc, longest)) {
 #pragma omp atomic write
             failed = 1;
@@ -701,7 +834,7 @@ StagingArena g_staging;
 // *no_staging is set when the page-locked staging memory could not be had; nothing has been copied
 // then and the caller takes the non-streamed way.
 int stream_tiles_by_row_block(dsfacto *h, const std::vector<int32_t> &cb, int64_t longest, const int64_t *indptr,
-                              const int32_t *indices, const float *values, bool *no_staging) {
+                              const int32_t *indices, const float *values, bool *no_staging, SgdPlanBuild *pb) {
     *no_staging = false;
     int T = omp_get_max_threads();
     if (T > 64) T = 64;
@@ -729,6 +862,8 @@ int stream_tiles_by_row_block(dsfacto *h, const std::vector<int32_t> &cb, int64_
     {
         const int k = omp_get_thread_num();
         RowBlockScratch sc;
+        sc.plan = pb;
+        sc.owner = k;
         cudaStream_t st = nullptr;
         cudaEvent_t ev[2] = {nullptr, nullptr};
         bool used[2] = {false, false};
@@ -871,14 +1006,14 @@ int dsfacto_create(dsfacto_t **out, int64_t n, int32_t d, int32_t K, int32_t p, 
     h->norm_grid = h->sm_count * 8;
     if (const char *env = std::getenv("DSFACTO_SWEEP")) h->sweep = (std::strcmp(env, "round") == 0) ? 0 : 1;
     if ((rc = dev_alloc(h, &h->d_S, (size_t)d))) return fail(rc);
-    if (cudaMemset(h->d_S, 0, sizeof(float4) * (size_t)d) != cudaSuccess) return fail(DSFACTO_ERR_CUDA);
+    if (cudaMemset(h->d_S, 0, sizeof(float2) * (size_t)d) != cudaSuccess) return fail(DSFACTO_ERR_CUDA);
     if (h->sweep == 1) {
         if ((rc = dev_alloc(h, &h->d_Tb, (size_t)d * h->Kp)) || (rc = dev_alloc(h, &h->d_Tw, (size_t)d)) ||
             (rc = dev_alloc(h, &h->d_TS, (size_t)d)))
             return fail(rc);
         if (cudaMemset(h->d_Tb, 0, sizeof(float) * (size_t)d * h->Kp) != cudaSuccess ||
             cudaMemset(h->d_Tw, 0, sizeof(float) * (size_t)d) != cudaSuccess ||
-            cudaMemset(h->d_TS, 0, sizeof(float4) * (size_t)d) != cudaSuccess)
+            cudaMemset(h->d_TS, 0, sizeof(float2) * (size_t)d) != cudaSuccess)
             return fail(DSFACTO_ERR_CUDA);
     }
     *out = h;
@@ -944,6 +1079,9 @@ int dsfacto_load_csr(dsfacto_t *h, const int64_t *indptr, const int32_t *indices
     HostBuf<float> xw;
     std::vector<int32_t> cb;
     int64_t longest = 0;
+    choose_chunk_len(h, nnz);
+    SgdPlanBuild pb;   // the chunks of the stratum SGD launches are cut while the tiles are bucketed
+    if (!init_plan_build(h, pb, omp_get_max_threads())) { cudaStreamSynchronize(st); free_data(h); return DSFACTO_ERR_OOM; }
     const bool by_row_block = use_row_block_bucketer(h);
     const char *load_env = std::getenv("DSFACTO_LOAD");
     const bool streamed = by_row_block && nnz > 0 &&
@@ -954,15 +1092,15 @@ int dsfacto_load_csr(dsfacto_t *h, const int64_t *indptr, const int32_t *indices
         try { column_blocks(h, cb); } catch (const std::bad_alloc &) { cudaStreamSynchronize(st); free_data(h); return DSFACTO_ERR_OOM; }
         longest = count_tiles_by_row_block(h, cb, indptr, indices);
     } else {
-        rc = by_row_block ? bucket_tiles_by_row_block(h, indptr, indices, values, ent, xw)
-                          : bucket_tiles(h, indptr, indices, values, ent, xw);
+        rc = by_row_block ? bucket_tiles_by_row_block(h, indptr, indices, values, ent, xw, &pb)
+                          : bucket_tiles(h, indptr, indices, values, ent, xw, &pb);
         if (rc) { cudaStreamSynchronize(st); free_data(h); return rc; }
     }
     h->nnz = nnz;   // (free_data on an error path above resets it)
     if ((rc = dev_alloc(h, &h->d_A, (size_t)n * h->Kp)) || (rc = dev_alloc(h, &h->d_G, (size_t)n)) ||
-        (rc = dev_alloc(h, &h->d_tile_ptr, h->tile_ptr.size())) || (rc = dev_alloc(h, &h->d_ent, cnt)) ||
+        (rc = dev_alloc(h, &h->d_tile_ptr, h->tile_ptr.size())) || (rc = dev_alloc(h, &h->d_ent, cnt + 4)) ||
         (rc = dev_alloc(h, &h->d_partials, 2 * ((size_t)h->refresh_grid + (size_t)h->norm_grid))) ||
-        (h->wide && (rc = dev_alloc(h, &h->d_xw, cnt)))) {
+        (h->wide && (rc = dev_alloc(h, &h->d_xw, cnt + 4)))) {
         cudaStreamSynchronize(st);
         free_data(h);
         return rc;
@@ -970,9 +1108,10 @@ int dsfacto_load_csr(dsfacto_t *h, const int64_t *indptr, const int32_t *indices
     bool copy_from_host = !streamed;
     if (streamed) {
         bool no_staging = false;
-        rc = stream_tiles_by_row_block(h, cb, longest, indptr, indices, values, &no_staging);
+        rc = stream_tiles_by_row_block(h, cb, longest, indptr, indices, values, &no_staging, &pb);
         if (rc && no_staging) {   // no page-locked memory to be had: bucket into pageable memory, one copy
-            rc = bucket_tiles_by_row_block(h, indptr, indices, values, ent, xw);
+            if (!init_plan_build(h, pb, omp_get_max_threads())) { cudaStreamSynchronize(st); free_data(h); return DSFACTO_ERR_OOM; }
+            rc = bucket_tiles_by_row_block(h, indptr, indices, values, ent, xw, &pb);
             copy_from_host = true;
         }
         if (rc) { cudaStreamSynchronize(st); free_data(h); return rc; }
@@ -983,16 +1122,43 @@ int dsfacto_load_csr(dsfacto_t *h, const int64_t *indptr, const int32_t *indices
     }
     CU_TRY(h, cudaMemcpyAsync(h->d_tile_ptr, h->tile_ptr.data(), sizeof(int64_t) * h->tile_ptr.size(), cudaMemcpyHostToDevice, st));
     CU_TRY(h, cudaStreamSynchronize(st));
-    if ((rc = build_sgd_plan(h))) { free_data(h); return rc; }
+    if ((rc = finish_sgd_plan(h, pb))) { free_data(h); return rc; }
+    h->failed = false;
     h->loaded = true;
     rc = run_refresh(h, false);
     if (rc) return rc;
     return std::isfinite(h->objective) ? DSFACTO_OK : DSFACTO_ERR_DIVERGED;
 }
 
+// An SGD launch gave up (a bounded wait ran out, or a check of the debug build failed): the warps left
+// in the middle of the sweep, so the parameters and the scaled state are a mixture.  The bookkeeping of
+// the sweep is cleared and the handle refuses further epochs until the parameters are set again
+// (dsfacto_set_params with w and V) or a data set is loaded after that.
+static int sgd_gave_up(dsfacto *h, const int code[3]) {
+    h->failed = true;
+    char buf[160];
+    if (code[0] == 1) std::snprintf(buf, sizeof buf, "stratum SGD: a wait for an earlier tile of the same column block timed out");
+    else if (code[0] == 2) std::snprintf(buf, sizeof buf, "stratum SGD: a copy of entry records into shared memory did not arrive");
+    else std::snprintf(buf, sizeof buf, "stratum SGD: debug check %d failed (value %d)", code[1], code[2]);
+    h->err = buf;
+    const size_t d = (size_t)h->d;
+    cudaMemsetAsync(h->d_tile_count, 0, sizeof(int) * (size_t)h->p * h->p, h->stream);
+    cudaMemsetAsync(h->d_run_count, 0, sizeof(int) * (size_t)std::max<int64_t>(h->long_runs, 1), h->stream);
+    cudaMemsetAsync(h->d_sync, 0, sizeof(int) * sync_words(h->p), h->stream);
+    cudaMemsetAsync(h->d_S, 0, sizeof(float2) * d, h->stream);
+    if (h->d_TS) {
+        cudaMemsetAsync(h->d_TS, 0, sizeof(float2) * d, h->stream);
+        cudaMemsetAsync(h->d_Tw, 0, sizeof(float) * d, h->stream);
+        cudaMemsetAsync(h->d_Tb, 0, sizeof(float) * d * h->Kp, h->stream);
+    }
+    cudaStreamSynchronize(h->stream);
+    return DSFACTO_ERR_CUDA;
+}
+
 int dsfacto_epoch(dsfacto_t *h) {
     if (!h) return DSFACTO_ERR_INVALID_ARG;
     if (!h->loaded) return DSFACTO_ERR_NO_DATA;
+    if (h->failed) { h->err = "the last stratum SGD launch gave up: set the parameters again (dsfacto_set_params) first"; return DSFACTO_ERR_CUDA; }
     cudaStream_t st = h->stream;
     CU_TRY(h, cudaEventRecord(h->ev[0], st));
     const int64_t p = h->p;
@@ -1014,9 +1180,9 @@ int dsfacto_epoch(dsfacto_t *h) {
         cudaEventElapsedTime(&a23, h->ev[2], h->ev[3]);
         t01 += a01; t12 += a12; t23 += a23;
     }
-    int sgd_error = 0;  // set by the SGD kernel if a dependency wait ran out (never seen; the state is then unusable)
-    CU_TRY(h, cudaMemcpy(&sgd_error, h->d_sync + kSyncError, sizeof(int), cudaMemcpyDeviceToHost));
-    if (sgd_error) { h->err = "stratum SGD: a wait for an earlier tile of the same column block timed out"; return DSFACTO_ERR_CUDA; }
+    int sgd_error[3] = {0, 0, 0};  // set by the SGD kernel if one of its bounded waits ran out
+    CU_TRY(h, cudaMemcpy(sgd_error, h->d_sync + kSyncError, sizeof sgd_error, cudaMemcpyDeviceToHost));
+    if (sgd_error[0]) return sgd_gave_up(h, sgd_error);
     h->ms[0] = t01 + t12 + t23; h->ms[1] = t01; h->ms[2] = t12; h->ms[3] = t23;
     return std::isfinite(h->objective) ? DSFACTO_OK : DSFACTO_ERR_DIVERGED;
 }
@@ -1067,6 +1233,7 @@ int dsfacto_set_params(dsfacto_t *h, const float *w0, const float *w, const floa
         CU_TRY(h, cudaStreamSynchronize(h->stream));
     }
     if (V) { int rc = upload_V(h, V); if (rc) return rc; }
+    if (w && V) h->failed = false;   // a handle whose SGD launch gave up is usable again once w and V are replaced
     if (h->loaded) {
         int rc = run_refresh(h, false);
         if (rc) return rc;
@@ -1119,8 +1286,8 @@ int dsfacto_bucket_host(int64_t n, int32_t d, int32_t p, const int64_t *indptr, 
     if ((rc = setup_partition(&tmp))) return rc;
     HostBuf<uint2> ent;
     HostBuf<float> xw;
-    rc = tmp.sweep == 1 ? bucket_tiles_by_row_block(&tmp, indptr, indices, values, ent, xw)
-                        : bucket_tiles(&tmp, indptr, indices, values, ent, xw);
+    rc = tmp.sweep == 1 ? bucket_tiles_by_row_block(&tmp, indptr, indices, values, ent, xw, nullptr)
+                        : bucket_tiles(&tmp, indptr, indices, values, ent, xw, nullptr);
     if (rc) return rc;
     const std::vector<int64_t> canon = canonical_tile_ptr(&tmp);
     std::memcpy(tile_ptr, canon.data(), sizeof(int64_t) * canon.size());
@@ -1220,6 +1387,26 @@ int dsfacto_last_epoch_ms(dsfacto_t *h, float ms[4]) {
     if (!h || !ms) return DSFACTO_ERR_INVALID_ARG;
     for (int i = 0; i < 4; ++i) ms[i] = h->ms[i];
     return DSFACTO_OK;
+}
+
+int dsfacto_debug_set(dsfacto_t *h, int32_t key, int64_t value) {
+    if (!h) return DSFACTO_ERR_INVALID_ARG;
+    switch (key) {
+    case DSFACTO_DEBUG_SPIN_LIMIT:
+        if (value < 1 || value > kSgdSpinLimit) return DSFACTO_ERR_INVALID_ARG;
+        h->spin_limit = (int)value;
+        return DSFACTO_OK;
+    case DSFACTO_DEBUG_EXTRA_NEED:
+        if (value < 0 || value > 1000 || h->loaded) return DSFACTO_ERR_INVALID_ARG;
+        h->debug_extra_need = (int)value;
+        return DSFACTO_OK;
+    case DSFACTO_DEBUG_CHUNK_LEN:
+        if ((value != 0 && (value < 16 || value > kChunkMax)) || h->loaded) return DSFACTO_ERR_INVALID_ARG;
+        h->chunk_override = (int)value;
+        return DSFACTO_OK;
+    default:
+        return DSFACTO_ERR_INVALID_ARG;
+    }
 }
 
 int dsfacto_launch_count(dsfacto_t *h, int64_t *out) {

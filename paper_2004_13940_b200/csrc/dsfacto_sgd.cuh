@@ -4,171 +4,95 @@
 // (eqs. (dsfacto_sgdupdatew), (dsfacto_sgdupdatev) regrouped):
 //     v_j <- (1 - e) v_j + b a_i,   e = h (lambda_v - G_i x^2),  b = -h G_i x,  h = eta / n
 //     w_j <- (1 - ew) w_j + b,      ew = h lambda_w
-// so a run of entries of one column is a composition of affine maps.  A composite is kept as
-// (D, B) with D = (product of (1-e)) - 1 and B the accumulated offset, starting from the identity
-// (0, 0): the per-entry shrink e is often below half an ulp of 1, and summing it into D keeps it at
-// full relative precision instead of losing it against v_j.  Consecutive pieces combine as
-//     (D2,B2) o (D1,B1) = (D1 + D2 + D1 D2,  B1 + D2 B1 + B2)
-// and a finished run is applied once: v_j <- (1 + D) v_j + B.
+// The factor (1 - e) is the same for every k.  Writing P_t for the product of the factors of a
+// column's entries 1..t (in the stratified order), the entries t = 1..T of a column give
+//     v_T = P_T ( v_0 + sum_t (b_t / P_t) a_{i_t} ),
+// so only the scalar P depends on the order; the K-wide part is a weighted sum of rows of A whose
+// pieces join by addition.  P is kept as D = P - 1 (the per-entry shrink e is often below half an
+// ulp of 1), pieces combine as D1 + D2 + D1 D2.  For w the factor is the constant (1 - ew), so its
+// product over m entries is (1 - ew)^m and only the count m is carried.
 //
-// During the SGD phase the column state is held in scaled form, v_j = (1 + sigma_j) u_j (and the
-// same for w_j), with sigma_j = 0 at the start of the phase.  Applying a run then needs only the
-// 8-byte scale pair of the column:  sigma' = sigma + D + sigma D,  u_j += B / (1 + sigma'),
-// so the K-wide part is an add that nobody waits for (red.global.add; every column receives at
-// most one per launch, so the result does not depend on timing).  sgd_finalize_* turns the state
-// back into plain (w, V) at the end of the phase.  The scaled form breaks down only if some
-// 1 + sigma reaches zero, i.e. a step so large that a run wipes its column; the parameters then
-// become non-finite and the epoch reports divergence.
+// During the SGD phase the column state is held in scaled form, v_j = (1 + sigma_j) u_j and
+// w_j = (1 - ew)^{m_j} uw_j with sigma_j = 0, m_j = 0 at the start of the phase.  Applying a run of
+// entries with local sums U = sum_t (b_t / P_t) a_i, W = sum_t b_t (1 - ew)^{-t}, product D and
+// length m is then
+//     u_j += U / (1 + sigma_j),  uw_j += W (1 - ew)^{-m_j},  sigma_j <- sigma_j + D + sigma_j D,  m_j += m:
+// the K-wide part is an add that nobody waits for (red.global.add; every column receives at most one
+// per tile and tiles of a column block are ordered, so the result does not depend on timing).
+// sgd_finalize_* turns the state back into plain (w, V) at the end of the phase.  The scaled form
+// breaks down only if some 1 + sigma reaches zero, i.e. a step so large that a run wipes its column;
+// the parameters then become non-finite and the epoch reports divergence.
 #pragma once
 #include "dsfacto_common.cuh"
 
 namespace dsf {
 
-constexpr int kSgdThreads = 32;   // one warp per CTA: a finished warp frees its registers and shared memory at once
-constexpr int kSgdWarps = kSgdThreads / 32;
-constexpr int kWarpEntries = 512;                 // entries per warp
-constexpr int kChunk = kSgdWarps * kWarpEntries;  // entries per CTA, at most (a launch may use shorter chunks)
+constexpr int kSgdWarps = 2;                      // warps per CTA; every warp works on its own chunks
+constexpr int kSgdThreads = 32 * kSgdWarps;
+constexpr int kChunkMax = 512;                    // most entries a chunk may hold
 constexpr int kSgdSpinLimit = 1 << 22;            // polls (about 100 ns each) before a dependency wait gives up
-// Words of the launch's synchronisation array.  The ticket counter takes one atomic per CTA and the
-// progress counters are polled by waiting CTAs, so every word sits in a 128-byte line of its own.
+constexpr int kCopySpinLimit = 1 << 24;           // polls before the wait for a bulk copy into shared memory gives up
+constexpr int kTicketStop = 0x40000000;           // ticket counter value that makes every warp leave
+// Words of the launch's synchronisation array.  The ticket counter takes one atomic per chunk and the
+// progress counters are polled by waiting warps, so every word sits in a 128-byte line of its own.
 constexpr int kSyncStride = 32;                   // ints between two words
 constexpr int kSyncTicket = 0;                    // next chunk to hand out
-constexpr int kSyncError = kSyncStride;           // set when a dependency wait ran out
+constexpr int kSyncError = kSyncStride;           // set when a wait ran out (1: earlier tile, 2: bulk copy, 3: debug check)
 __host__ __device__ constexpr size_t sync_done(int c) { return (size_t)(2 + c) * kSyncStride; }  // finished tiles of column block c
 __host__ __device__ constexpr size_t sync_words(int p) { return (size_t)(2 + p) * kSyncStride; }
 
-// entries of one warp pass: sized so that the gathered rows of A fill about 4 KB of shared memory, but
-// never fewer than 16 entries: with 8-entry passes (rows of 512 bytes and more) the fixed cost of a
-// pass and its one exposed gather latency dominated (K = 128: 59.1 ms per sweep with 8, 46.7 with 16,
-// 54.6 with 32 on the 400 M-entry workload)
-__host__ __device__ constexpr int sgd_pass_len(int LG, int NV) {
-    return 256 / (LG * NV) > 256 ? 256 : (256 / (LG * NV) < 16 ? 16 : 256 / (LG * NV));
-}
-// resident one-warp CTAs per SM the register budget is cut for: 24 for rows up to 256 bytes; wider
-// rows hold 16 entries per lane group in flight and are limited by shared memory anyway
-__host__ __device__ constexpr int sgd_min_ctas(int LG, int NV) { return LG * NV >= 32 ? 12 : 24; }
-// floats per chunk record in global scratch: 3 header float4s + head offsets + tail offsets
-__host__ __device__ constexpr int chunk_record_floats(int Kp) { return 12 + 2 * Kp; }
-
-// shared-memory carve-up of one warp, in float4 units
-template <int LG, int NV>
-struct SgdSmem {
-    static constexpr int GW = 32 / LG;
-    static constexpr int KP4 = LG * NV;
-    static constexpr int PASS = sgd_pass_len(LG, NV);
-    static constexpr int S = PASS / GW;                  // entries a lane group walks per pass
-    static constexpr int ITEM_STRIDE = S + 1;            // +1: lane groups land in different banks
-    static constexpr int ROW_STRIDE = (S + (LG < 8 ? 1 : 0)) * KP4;
-    static constexpr int ITEMS = 0;                      // GW * ITEM_STRIDE   {e, b, row, j_local}
-    static constexpr int ROWS = ITEMS + GW * ITEM_STRIDE;  // GW * ROW_STRIDE  gathered rows a_i
-    static constexpr int SCALES = ROWS + GW * ROW_STRIDE;  // GW * ITEM_STRIDE float4: scale pair of the
-                                                         // column whose run starts at that entry
-    static constexpr int WARP = SCALES + GW * ITEM_STRIDE;  // float4s per warp
-    // per CTA, after the warps: per warp head/tail pieces, then the chunk head piece
-    static constexpr int WPIECE = kSgdWarps * WARP;      // kSgdWarps * 2 * (KP4+1)
-    static constexpr int CPIECE = WPIECE + kSgdWarps * 2 * (KP4 + 1);  // (KP4+1)
-    static constexpr int TOTAL = CPIECE + (KP4 + 1);
-    static constexpr int BYTES = TOTAL * 16 + 16 * kSgdWarps;  // + per-warp boundary flags
+// One unit of work of the sweep: a range of consecutive entries of one tile (entries of a tile are
+// sorted by (column, row)).  Either whole runs (all entries of a column inside the tile), or a slice
+// of one run that is longer than a chunk.  Built on the host when the tiles are bucketed.
+struct ChunkDesc {
+    int64_t ent_off;   // first entry in the entry array
+    int32_t len;       // entries, 1 .. chunk length
+    int32_t flags;     // kChunkSlice: slice of a long run; kChunkTail: the tile acts on the tail composite
+    int32_t row0;      // first row of the tile's row block
+    int32_t col0;      // first column of the tile's column block
+    int32_t cblock;    // column block (index of its progress counter)
+    int32_t need;      // earlier non-empty tiles of that column block, in sweep order
+    int32_t tile;      // tile slot (index of its chunk counter)
+    int32_t nchunks;   // chunks of the tile
+    int32_t run_id;    // slice: index of the long run (its join counter)
+    int32_t slice;     // slice: number of this slice inside the run
+    int32_t nslices;   // slice: slices of the run
+    int32_t rec0;      // slice: record index of slice 0 of the run
+    int32_t jl;        // slice: local column of the run
+    int32_t pad;
 };
+static_assert(sizeof(ChunkDesc) == 64, "a chunk descriptor is 16 ints");
+enum { kChunkSlice = 1, kChunkTail = 2 };
 
-template <int NV>
-struct Comp {
-    float D, Dw, Bw;
-    float4 B[NV];
+// lane layout and shared-memory staging of one warp
+template <int LG, int NV>
+struct SgdCfg {
+    static constexpr int GW = 32 / LG;               // lane groups per warp = rows worked on side by side
+    static constexpr int KP4 = LG * NV;              // float4s per factor row
+    // rows of A gathered per stage: at most 4 KB a stage
+    static constexpr int RST = KP4 <= 8 ? 32 : (KP4 <= 16 ? 16 : (KP4 <= 32 ? 8 : 4));
+    static constexpr int SP = 32 / RST;              // stages per 32-entry pass
+    static constexpr int NBUF = KP4 <= 8 ? 2 : 3;    // stages in the ring
+    static constexpr int PD = NBUF - 1;              // stages requested ahead
+    static constexpr int ROW4 = NBUF * RST * KP4;    // float4s of the row ring
 };
-
-template <int NV>
-__device__ __forceinline__ void comp_identity(Comp<NV> &c) {
-    c.D = 0.f; c.Dw = 0.f; c.Bw = 0.f;
-#pragma unroll
-    for (int v = 0; v < NV; ++v) c.B[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-}
-
-// second o first (first acts first)
-template <int NV>
-__device__ __forceinline__ Comp<NV> compose(const Comp<NV> &first, const Comp<NV> &second) {
-    Comp<NV> r;
-#pragma unroll
-    for (int v = 0; v < NV; ++v) {
-        r.B[v].x = fmaf(second.D, first.B[v].x, first.B[v].x) + second.B[v].x;
-        r.B[v].y = fmaf(second.D, first.B[v].y, first.B[v].y) + second.B[v].y;
-        r.B[v].z = fmaf(second.D, first.B[v].z, first.B[v].z) + second.B[v].z;
-        r.B[v].w = fmaf(second.D, first.B[v].w, first.B[v].w) + second.B[v].w;
-    }
-    r.Bw = fmaf(second.Dw, first.Bw, first.Bw) + second.Bw;
-    r.D = fmaf(first.D, second.D, first.D + second.D);
-    r.Dw = fmaf(first.Dw, second.Dw, first.Dw + second.Dw);
-    return r;
-}
-
-template <int NV>
-__device__ __forceinline__ Comp<NV> comp_shfl_up(const Comp<NV> &c, int delta) {
-    Comp<NV> r;
-    r.D = __shfl_up_sync(0xFFFFFFFFu, c.D, delta);
-    r.Dw = __shfl_up_sync(0xFFFFFFFFu, c.Dw, delta);
-    r.Bw = __shfl_up_sync(0xFFFFFFFFu, c.Bw, delta);
-#pragma unroll
-    for (int v = 0; v < NV; ++v) {
-        r.B[v].x = __shfl_up_sync(0xFFFFFFFFu, c.B[v].x, delta);
-        r.B[v].y = __shfl_up_sync(0xFFFFFFFFu, c.B[v].y, delta);
-        r.B[v].z = __shfl_up_sync(0xFFFFFFFFu, c.B[v].z, delta);
-        r.B[v].w = __shfl_up_sync(0xFFFFFFFFu, c.B[v].w, delta);
-    }
-    return r;
-}
-
-template <int NV>
-__device__ __forceinline__ Comp<NV> comp_shfl_down(const Comp<NV> &c, int delta) {
-    Comp<NV> r;
-    r.D = __shfl_down_sync(0xFFFFFFFFu, c.D, delta);
-    r.Dw = __shfl_down_sync(0xFFFFFFFFu, c.Dw, delta);
-    r.Bw = __shfl_down_sync(0xFFFFFFFFu, c.Bw, delta);
-#pragma unroll
-    for (int v = 0; v < NV; ++v) {
-        r.B[v].x = __shfl_down_sync(0xFFFFFFFFu, c.B[v].x, delta);
-        r.B[v].y = __shfl_down_sync(0xFFFFFFFFu, c.B[v].y, delta);
-        r.B[v].z = __shfl_down_sync(0xFFFFFFFFu, c.B[v].z, delta);
-        r.B[v].w = __shfl_down_sync(0xFFFFFFFFu, c.B[v].w, delta);
-    }
-    return r;
-}
-
-template <int NV>
-__device__ __forceinline__ Comp<NV> comp_shfl(const Comp<NV> &c, int src) {
-    Comp<NV> r;
-    r.D = __shfl_sync(0xFFFFFFFFu, c.D, src);
-    r.Dw = __shfl_sync(0xFFFFFFFFu, c.Dw, src);
-    r.Bw = __shfl_sync(0xFFFFFFFFu, c.Bw, src);
-#pragma unroll
-    for (int v = 0; v < NV; ++v) {
-        r.B[v].x = __shfl_sync(0xFFFFFFFFu, c.B[v].x, src);
-        r.B[v].y = __shfl_sync(0xFFFFFFFFu, c.B[v].y, src);
-        r.B[v].z = __shfl_sync(0xFFFFFFFFu, c.B[v].z, src);
-        r.B[v].w = __shfl_sync(0xFFFFFFFFu, c.B[v].w, src);
-    }
-    return r;
-}
-
-// a composite as stored in shared or global memory: KP4 offset float4s, then {D, Dw, Bw, column}
+// entries the staging buffer of one chunk holds: the copy starts and ends on multiples of 4 entries
+__host__ __device__ constexpr int sgd_ecap(int chunk_len) { return (chunk_len + 8 + 3) & ~3; }
 template <int LG, int NV>
-__device__ __forceinline__ void comp_store(float4 *dst, const Comp<NV> &c, uint32_t col, int l) {
-#pragma unroll
-    for (int v = 0; v < NV; ++v) dst[v * LG + l] = c.B[v];
-    if (l == 0) dst[LG * NV] = make_float4(c.D, c.Dw, c.Bw, __uint_as_float(col));
+__host__ __device__ constexpr size_t sgd_warp_smem(bool wide, int chunk_len) {
+    return (size_t)SgdCfg<LG, NV>::ROW4 * 16 + 32 * 16 * 2 + 40 * 4 + 16 +
+           (size_t)2 * sgd_ecap(chunk_len) * (wide ? 12 : 8);
 }
-template <int LG, int NV>
-__device__ __forceinline__ uint32_t comp_load(const float4 *src, Comp<NV> &c, int l) {
-#pragma unroll
-    for (int v = 0; v < NV; ++v) c.B[v] = src[v * LG + l];
-    const float4 hd = src[LG * NV];
-    c.D = hd.x; c.Dw = hd.y; c.Bw = hd.z;
-    return __float_as_uint(hd.w);
-}
+// floats of the record a slice of a long run leaves: {D, m, W, -} and the K-wide sum
+__host__ __device__ constexpr int slice_record_floats(int Kp) { return 4 + Kp; }
 
 __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src) {
     const unsigned s = (unsigned)__cvta_generic_to_shared(smem_dst);
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem_src) : "memory");
 }
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
 // fire-and-forget adds into global memory
 __device__ __forceinline__ void red_add4(float4 *p, float x, float y, float z, float w) {
     asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(x), "f"(y), "f"(z), "f"(w) : "memory");
@@ -176,597 +100,599 @@ __device__ __forceinline__ void red_add4(float4 *p, float x, float y, float z, f
 __device__ __forceinline__ void red_add1(float *p, float x) {
     asm volatile("red.global.add.f32 [%0], %1;" ::"l"(p), "f"(x) : "memory");
 }
-// 1 / x by the special-function unit alone (within one unit in the last place): it scales an increment,
-// so a correctly rounded reciprocal would buy nothing but instructions
+// 1 / x and 2^x by the special-function unit alone (within a unit or two in the last place): both scale
+// an increment, so a correctly rounded result would buy nothing but instructions
 __device__ __forceinline__ float rcp_fast(float x) {
     float r;
     asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
     return r;
 }
-__device__ __forceinline__ void cp_async_wait_all() {
-    asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;\n" ::: "memory");
+__device__ __forceinline__ float ex2_fast(float x) {
+    float r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+__device__ __forceinline__ int ld_acquire(const int *p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+// ---- mbarrier + bulk copy global -> shared (the entry records of a chunk arrive with one instruction) ----
+__device__ __forceinline__ void mbar_init(uint64_t *bar, int count) {
+    const unsigned s = (unsigned)__cvta_generic_to_shared(bar);
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, unsigned bytes) {
+    const unsigned s = (unsigned)__cvta_generic_to_shared(bar);
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, unsigned parity) {
+    const unsigned s = (unsigned)__cvta_generic_to_shared(bar);
+    unsigned ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok)
+        : "r"(s), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// source and destination 16-byte aligned, bytes a multiple of 16
+__device__ __forceinline__ void bulk_copy_g2s(void *smem_dst, const void *gmem_src, unsigned bytes, uint64_t *bar) {
+    const unsigned d = (unsigned)__cvta_generic_to_shared(smem_dst);
+    const unsigned b = (unsigned)__cvta_generic_to_shared(bar);
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(d),
+                 "l"(gmem_src), "r"(bytes), "r"(b)
+                 : "memory");
 }
 
-// One step of a segmented scan over the lane groups of a warp (all 32 lanes must call it).
-// Each lane group contributes an element: `hasb` (it holds a run boundary), `head` (composite of
-// what precedes its first boundary) and `cur` (composite after its last boundary, or of the whole
-// element when it has none).  `carry`/`cflag` describe the run left open by earlier steps and are
-// updated to the run left open after this step.  For a group with a boundary, `closing` becomes
-// the composite of the run that ends at its first boundary and `outer` tells whether that run began
-// before the first step (nothing to its left held a boundary).
-template <int LG, int NV>
-__device__ __forceinline__ void scan_step(bool hasb, const Comp<NV> &head, const Comp<NV> &cur, Comp<NV> &carry,
-                                          bool &cflag, Comp<NV> &closing, bool &outer) {
-    constexpr int GW = 32 / LG;
-    const int lane = threadIdx.x & 31;
-    const int g = lane / LG, l = lane % LG;
-    Comp<NV> inc = cur;
-    bool finc = hasb;
-    if (GW > 1) {
-#pragma unroll
-        for (int delta = 1; delta < GW; delta <<= 1) {
-            const Comp<NV> o = comp_shfl_up<NV>(inc, delta * LG);
-            const bool of = __shfl_up_sync(0xFFFFFFFFu, (int)finc, delta * LG) != 0;
-            if (g >= delta) {
-                if (!finc) inc = compose<NV>(o, inc);
-                finc = finc || of;
-            }
-        }
-    }
-    Comp<NV> ex;  // what is open on this group's left, from earlier groups of this step
-    bool fex = false;
-    comp_identity(ex);
-    if (GW > 1) {
-        const Comp<NV> up = comp_shfl_up<NV>(inc, LG);
-        const bool fup = __shfl_up_sync(0xFFFFFFFFu, (int)finc, LG) != 0;
-        if (g > 0) { ex = up; fex = fup; }
-    }
-    outer = false;
-    if (hasb) {
-        closing = compose<NV>(fex ? ex : compose<NV>(carry, ex), head);
-        outer = !(fex || cflag);
-    }
-    const Comp<NV> lastc = comp_shfl<NV>(inc, (GW - 1) * LG + l);
-    const bool lastf = __shfl_sync(0xFFFFFFFFu, (int)finc, (GW - 1) * LG) != 0;
-    carry = lastf ? lastc : compose<NV>(carry, lastc);
-    cflag = cflag || lastf;
-}
+struct SgdArgs {
+    const ChunkDesc *desc;     // chunks of this launch, in sweep order
+    int nchunks;
+    const uint2 *ent;          // packed: {(i_local << jbits) | j_local, bits of x}; wide: {i_local, j_local}
+    const float *xw;           // wide layout only: x per entry
+    const float *A;            // n * Kp
+    const float *G;            // n
+    float *w;                  // d        uw_j
+    float *V;                  // d * Kp   u_j
+    float2 *S;                 // d        {sigma_j, m_j (int bits)}
+    float *Tw;                 // d        the same three for the tail composite T_j (row-block sweep)
+    float *Tb;                 // d * Kp
+    float2 *TS;                // d
+    float *records;            // slice_record_floats(Kp) floats per slice of a long run
+    int *tile_count;           // p*p, all zero between launches
+    int *run_count;            // one per long run, all zero between launches
+    int *sync;                 // sync_words(p) ints: ticket counter (zero at launch), error word, finished tiles
+                               // per column block (zero at the first launch of a sweep, kept between the
+                               // launches of one sweep)
+    int jbits;
+    int chunk_len;             // longest chunk of the plan (sizes the staging buffers)
+    int spin_limit;            // polls before the wait for an earlier tile gives up
+    float h, lambda_v;
+    float kappa_w;             // -log2(1 - ew): (1 - ew)^{-m} = 2^(m kappa_w)
+};
+
+#ifdef DSFACTO_DEBUG
+// bounds-checked build: a failed check records its code and the offending value, and the access is skipped
+#define DSF_CHECK(cond, code, value)                                    \
+    do {                                                                \
+        if (!(cond)) {                                                  \
+            if (atomicCAS(a.sync + kSyncError, 0, 3) == 0) {            \
+                a.sync[kSyncError + 1] = (code);                        \
+                a.sync[kSyncError + 2] = (int)(value);                  \
+            }                                                           \
+        }                                                               \
+    } while (0)
+#define DSF_OK(cond) (cond)
+#else
+#define DSF_CHECK(cond, code, value) do { } while (0)
+#define DSF_OK(cond) true
+#endif
 
 // ------------------------------------------------------------------------------------------
-// sgd_chunk_kernel: one CTA per chunk of kChunk consecutive entries of one tile (kSgdWarps warps; 1 today).
+// sgd_sweep_kernel: persistent warps; each takes chunks in sweep order from a ticket counter.
 //
-// A launch covers tiles with pairwise disjoint column blocks: the p tiles of one inner round
-// (sweep 0) or the p tiles of one row block (sweep 1).  A tile's entries are sorted by (column,
-// row).  Every warp owns kWarpEntries consecutive entries and walks them in passes.  Per pass:
-//   1. one lane per entry turns the (prefetched) entry record and G_i into (e, b, row, column);
-//      a "boundary" sits before an entry whose column differs from the entry before it (the tile
-//      start counts), i.e. at every entry that starts a run;
-//   2. the rows a_i of the whole pass, and the scale pair of every column whose run starts in the
-//      pass, are gathered into shared memory with cp.async: one memory latency per pass;
-//   3. each lane group walks S consecutive entries sequentially.  The piece before its first
-//      boundary becomes its head; a run that starts and ends inside the group is applied on the
-//      spot from the prefetched scale pair (stores and adds nobody waits for);
-//   4. scan_step joins the pieces across the lane groups of the warp; the runs that end at the
-//      groups' first boundaries are applied together.
-// Runs that cross warps are joined by the same scan run by warp 0 over the warps' results (shared
-// memory); runs that cross chunks by the same scan run by whichever chunk of the tile finishes
-// last, over per-chunk records in global scratch (one counter per tile; no CTA waits for another).
+// Pipeline of a warp: the ticket of chunk n+2, the descriptor of chunk n+1 and the entry records of
+// chunk n+1 (one bulk copy into shared memory, completion on an mbarrier) are under way while chunk
+// n is worked on.  A chunk is walked in passes of 32 entries, one entry per lane for the scalar
+// part:
+//   scalar stage   G_i (requested one pass ahead) -> e, b; run boundaries by comparing neighbours;
+//                  segmented scan of D = P - 1 over the lanes; coefficient c = b / P and the w
+//                  coefficient; for every run that starts in the pass the scale record of its column
+//                  (requested one pass ahead).  Results go to shared memory.
+//   K-wide stage   the rows a_i of a stage (32 rows for K <= 32, fewer for wider rows; gathered with
+//                  cp.async one or two stages ahead) are added with weight c.  The run that is open at
+//                  the start of a stage and the run that is open at its end are spread over all lane
+//                  groups (entry u goes to group u mod GW) and the groups keep their partial sums in
+//                  registers until the run ends, then a shuffle tree joins them; runs that start and
+//                  end inside a stage go to one lane group each.  A finished run is applied at once.
+// A slice of a long run has no boundary at all: its sum, product and length go to a record, and the
+// slice of the run that finishes last joins the records in order (scalar prefix products first, then a
+// weighted sum of the K-wide parts) and applies the run.
 //
-// Column state: in a direct tile it is the scaled (w_j, v_j).  In a tail tile (sweep 1, r > c) it
-// is a per-column composite T_j in the same scaled form, identity at the start of the epoch and
+// Order: a tile may touch column state only after the earlier tiles of its column block are done (one
+// counter per column block, bumped by the chunk that finishes a tile, after a fence).  Tickets are
+// handed out in sweep order, so every chunk a warp may wait for is already held by a warp that is
+// running: no deadlock, and no reliance on the order in which CTAs start.  The wait is bounded all
+// the same; when it runs out the error word is set, the ticket counter jumps past the end, and every
+// warp leaves at its next ticket.
+//
+// Column state: in a direct tile it is the scaled (w_j, v_j).  In a tail tile (row-block sweep, r > c)
+// it is a per-column composite T_j in the same scaled form, identity at the start of the epoch and
 // applied to (w_j, v_j) by sgd_finalize_* after the sweep.  The sweep visits row blocks p-1, .., 0,
 // so for column block c the tail tiles (r = p-1 .. c+1) and then the direct tiles (r = c .. 0) are
 // each met in the stratified order of the rounds, and "T_j after v_j" restores the order
-// c, .., 0, p-1, .., c+1.  Meanwhile all entries of a row meet in one launch, so (a_i, G_i) come
-// from L2 after first touch.
+// c, .., 0, p-1, .., c+1.  Meanwhile all entries of a row meet close together in time, so (a_i, G_i)
+// come from L2 after first touch.
 // ------------------------------------------------------------------------------------------
-struct SgdChunkArgs {
-    const int64_t *tile_ptr;   // p*p+1, tiles in sweep order (slots)
-    const uint2 *ent;          // packed: {(i_local << jbits) | j_local, bits of x}; wide: {i_local, j_local}
-    const float *xw;           // wide layout only: x per entry
-    const int64_t *row_start;  // p+1
-    const int32_t *col_start;  // p+1
-    const float *A;            // n * Kp
-    const float *G;            // n
-    float *w;                  // d        u-part of w_j
-    float *V;                  // d * Kp   u-part of v_j
-    float4 *S;                 // d        {sigma of v_j, sigma of w_j, -, -}
-    float *Tw;                 // d        u-part of the w offset of T_j      (sweep 1)
-    float *Tb;                 // d * Kp   u-part of the v offset of T_j      (sweep 1)
-    float4 *TS;                // d        {D, Dw, -, -} of T_j               (sweep 1)
-    const int4 *chunk_map;     // per chunk, in sweep order: {tile slot, chunk index inside the tile, number
-                               // of earlier non-empty tiles of the same column block, -}
-    float *records;            // chunk_record_floats(Kp) floats per chunk
-    int *tile_count;           // p*p, all zero between launches
-    int *sync;                 // sync_words(p) ints: ticket counter (zero at launch), error flag, finished
-                               // tiles per column block (zero at the first launch of a sweep, kept between
-                               // the launches of one sweep)
-    int p, jbits, sweep;
-    int chunk_base;            // first chunk of this launch in chunk_map (a launch may cover a range of rounds)
-    int chunk_len;             // entries per chunk, <= kChunk: short chunks for small data sets, whose epoch is a
-                               // chain of dependent tiles and is as long as p times the time one tile takes
-    float h, lambda_w, lambda_v;
-};
-
 template <int LG, int NV, bool WIDE>
-__global__ void __launch_bounds__(kSgdThreads, sgd_min_ctas(LG, NV)) sgd_chunk_kernel(const SgdChunkArgs a) {
-    typedef SgdSmem<LG, NV> L;
-    constexpr int GW = L::GW, KP4 = L::KP4, PASS = L::PASS, S = L::S;
-    constexpr int PP = kWarpEntries / PASS;
-    constexpr int EPL = (S + LG - 1) / LG;  // entries a lane holds per pass: lane l of group g holds the
-                                            // entries g*S + l*EPL + q of the pass, q < EPL (those below S)
-    constexpr int NW = kSgdWarps;
-    constexpr int REC4 = chunk_record_floats(4 * KP4) / 4;
-    static_assert(PASS * PP == kWarpEntries && S * GW == PASS, "a warp's entries must be whole passes");
-    typedef Comp<NV> C;
+__global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a) {
+    typedef SgdCfg<LG, NV> C;
+    constexpr int GW = C::GW, KP4 = C::KP4, RST = C::RST, SP = C::SP, NBUF = C::NBUF, PD = C::PD;
+    constexpr unsigned FULL = 0xFFFFFFFFu;
 
-    extern __shared__ float4 smem4[];
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane / LG, l = lane % LG;
-    float4 *sw = smem4 + warp * L::WARP;
-    float4 *s_item = sw + L::ITEMS + g * L::ITEM_STRIDE;
-    float4 *s_rows = sw + L::ROWS + g * L::ROW_STRIDE;
-    float4 *s_scale_all = sw + L::SCALES;
-    float4 *s_scale = s_scale_all + g * L::ITEM_STRIDE;
-    float4 *s_wpiece = smem4 + L::WPIECE;  // [warp][head/tail][KP4+1]
-    float4 *s_cpiece = smem4 + L::CPIECE;
-    int *s_wflag = reinterpret_cast<int *>(smem4 + L::TOTAL);
+    const int ecap = sgd_ecap(a.chunk_len);
+    unsigned char *wbase = smem_raw + (size_t)warp * sgd_warp_smem<LG, NV>(WIDE, a.chunk_len);
+    float4 *rowb = reinterpret_cast<float4 *>(wbase);               // row ring
+    float4 *pe = rowb + C::ROW4;                                    // per entry of the pass: {c, cw, D, m}
+    float4 *ps = pe + 32;                                           // per run start: {column, sigma, m_j, -}
+    int *segpos = reinterpret_cast<int *>(ps + 32);                 // lane of the k-th run start of the pass (40 ints)
+    uint64_t *mbar = reinterpret_cast<uint64_t *>(segpos + 40);     // one per entry buffer
+    uint2 *ebuf = reinterpret_cast<uint2 *>(mbar + 2);              // 2 x ecap entry records
+    float *xbuf = reinterpret_cast<float *>(ebuf + 2 * (size_t)ecap);  // wide layout: 2 x ecap values
 
-    // Chunks are handed out in sweep order by a ticket counter, so a CTA that holds a ticket knows that
-    // every earlier chunk has been taken by a CTA that is running or done: waiting for earlier tiles of
-    // the same column block can therefore not deadlock.  The wait is bounded all the same; on a
-    // time-out the error flag makes every CTA leave and the host reports the failure.
-    __shared__ int s_ticket, s_go;
-    if (tid == 0) s_ticket = atomicAdd(a.sync + kSyncTicket, 1);
-    __syncthreads();
-    const int chunk = a.chunk_base + s_ticket;
-    const int4 cm = a.chunk_map[chunk];
-    const int64_t t = cm.x;  // tile slot: position of the tile in sweep order (the device order of tiles)
-    int r, c;
-    if (a.sweep == 1) { r = a.p - 1 - (int)(t / a.p); c = (int)(t % a.p); }
-    else { r = (int)(t % a.p); c = (r + (int)(t / a.p)) % a.p; }
-    const bool tail_mode = a.sweep == 1 && r > c;
-    const int64_t tb = a.tile_ptr[t], te = a.tile_ptr[t + 1];
-    const int64_t cb = tb + (int64_t)cm.y * a.chunk_len;
-    const int64_t ce = (cb + a.chunk_len < te) ? cb + a.chunk_len : te;
-    const int64_t wb = cb + (int64_t)warp * kWarpEntries;
-    const int64_t we = (wb + kWarpEntries < ce) ? wb + kWarpEntries : ce;
-    const int64_t row0 = a.row_start[r];
-    const int64_t col0 = a.col_start[c];
-    const uint32_t jmask = a.jbits >= 32 ? 0xFFFFFFFFu : ((1u << a.jbits) - 1u);
-    const float ew = a.h * a.lambda_w;
-    // everything a warp touches is addressed with 32-bit offsets from pointers set up once
-    const float4 *A4 = reinterpret_cast<const float4 *>(a.A) + (size_t)row0 * KP4;  // rows of this row block
-    const float *Gr = a.G + row0;
-    const uint2 *entw = a.ent + wb;                      // this warp's entries
-    const float *xww = WIDE ? a.xw + wb : nullptr;
-    const int wlen = we > wb ? (int)(we - wb) : 0;
-    // the column state this tile acts on (u-parts and scale pairs), shifted to the column block
-    float4 *U4 = reinterpret_cast<float4 *>(tail_mode ? a.Tb : a.V) + (size_t)col0 * KP4;
-    float *uw = (tail_mode ? a.Tw : a.w) + col0;
-    float4 *Sc = (tail_mode ? a.TS : a.S) + col0;
-
-    // column state <- run o column state, given the column's scale pair (lanes of one group)
-    auto apply = [&](uint32_t jl, const C &x, float4 sc) {
-        const float sg = fmaf(sc.x, x.D, sc.x + x.D);
-        const float inv = rcp_fast(1.0f + sg);
-#pragma unroll
-        for (int v = 0; v < NV; ++v)
-            red_add4(U4 + (size_t)jl * KP4 + v * LG + l, x.B[v].x * inv, x.B[v].y * inv, x.B[v].z * inv,
-                     x.B[v].w * inv);
-        if (l == 0) {
-            const float sgw = fmaf(sc.y, x.Dw, sc.y + x.Dw);
-            red_add1(uw + jl, x.Bw * rcp_fast(1.0f + sgw));
-            Sc[jl] = make_float4(sg, sgw, 0.f, 0.f);
-        }
-    };
-    // the same with the scale pair fetched from L2 (never through L1: another SM wrote it in this launch)
-    auto apply_fetch = [&](uint32_t jl, const C &x) {
-        if (jl == kNoCol) return;
-        apply(jl, x, __ldcg(Sc + jl));
-    };
-
-    // ---------------- warp phase ----------------
-    C wcarry;  // open run of this warp so far
-    comp_identity(wcarry);
-    bool wflag = false;  // a boundary has been seen in this warp
-    uint32_t last_col = kNoCol;
-
-    // entry records are fetched two passes ahead and G one pass ahead, into registers
-    uint2 ent0[EPL], ent1[EPL];
-    float xw0[EPL], xw1[EPL], g0[EPL];
-    const int slot0 = l * EPL;          // this lane's first entry inside its group's S entries
-    const int at0 = g * S + slot0;      // ... and inside the pass
-    auto fetch_ent = [&](int pp, uint2 (&e)[EPL], float (&xv)[EPL]) {
-#pragma unroll
-        for (int q = 0; q < EPL; ++q) {
-            const int at = pp * PASS + at0 + q;
-            if (slot0 + q < S && at < wlen) {
-                e[q] = entw[at];
-                if (WIDE) xv[q] = xww[at];
-            }
-        }
-    };
-    auto fetch_g = [&](int pp, const uint2 (&e)[EPL], float (&gv)[EPL]) {
-#pragma unroll
-        for (int q = 0; q < EPL; ++q) {
-            const int at = pp * PASS + at0 + q;
-            if (slot0 + q < S && at < wlen) gv[q] = __ldg(Gr + (WIDE ? e[q].x : (e[q].x >> a.jbits)));
-        }
-    };
-    fetch_ent(0, ent0, xw0);
-    if (PP > 1) fetch_ent(1, ent1, xw1);
-    fetch_g(0, ent0, g0);
-
-    // the first fetches are under way; now make sure the earlier tiles of this column block are done
-    if (tid == 0) {
-        int go = 1;
-        const volatile int *done = a.sync + sync_done(c);
-        const volatile int *err = a.sync + kSyncError;
-        for (int spin = 0; *done < cm.z; ++spin) {
-            if (*err != 0 || spin > kSgdSpinLimit) { go = 0; break; }
-            __nanosleep(100);
-        }
-        if (!go) atomicExch(a.sync + kSyncError, 1);
-        __threadfence();
-        s_go = go;
-    }
-    __syncthreads();
-    if (!s_go) return;
-    for (int pp = 0; pp < PP; ++pp) {
-        if (pp * PASS >= wlen) break;
-        const int cnt = (wlen - pp * PASS) < PASS ? (wlen - pp * PASS) : PASS;
-        uint32_t before = kNoCol;  // column of the entry just before this pass, if it is in the tile
-        if (pp > 0) before = last_col;
-        else if (wb > tb) {
-            const uint2 rec = entw[-1];
-            before = WIDE ? rec.y : (rec.x & jmask);
-        }
-        // column of the entry just after this pass when it is known to this warp (its own next
-        // pass); otherwise the last run of the pass is left open and closed by a later phase
-        uint32_t after = kNoCol;
-        const bool after_known = (pp + 1 < PP) && ((pp + 1) * PASS < wlen);
-        // 1. items of this pass from the prefetched registers
-        uint32_t jq[EPL], ilq[EPL];
-        float eq[EPL], bq[EPL];
-        bool cont = true;  // every entry this lane holds continues the run that is open at the pass start
-#pragma unroll
-        for (int q = 0; q < EPL; ++q) {
-            jq[q] = kNoCol;
-            ilq[q] = 0u;
-            eq[q] = 0.f;
-            bq[q] = 0.f;
-            if (slot0 + q < S && at0 + q < cnt) {
-                float x;
-                if (WIDE) { ilq[q] = ent0[q].x; jq[q] = ent0[q].y; x = xw0[q]; }
-                else { ilq[q] = ent0[q].x >> a.jbits; jq[q] = ent0[q].x & jmask; x = __uint_as_float(ent0[q].y); }
-                const float gx = g0[q] * x;
-                eq[q] = a.h * (a.lambda_v - gx * x);
-                bq[q] = -a.h * gx;
-                cont = cont && jq[q] == before;
-            }
-        }
-        // A full pass inside one run (about two thirds of the passes on click-log data, where a few
-        // columns hold most entries) has no boundary: nothing is applied and nothing needs the staging
-        // in shared memory.  It takes the short way below.
-        const bool one_run = cnt == PASS && before != kNoCol && __all_sync(0xFFFFFFFFu, cont);
-        if (!one_run) {
-#pragma unroll
-            for (int q = 0; q < EPL; ++q)
-                if (slot0 + q < S && at0 + q < cnt)
-                    s_item[slot0 + q] = make_float4(eq[q], bq[q], __uint_as_float(ilq[q]), __uint_as_float(jq[q]));
-        }
-        // rotate the prefetch registers and start the next fetches
-#pragma unroll
-        for (int q = 0; q < EPL; ++q) { ent0[q] = ent1[q]; xw0[q] = xw1[q]; }
-        if (after_known) after = __shfl_sync(0xFFFFFFFFu, WIDE ? ent0[0].y : (ent0[0].x & jmask), 0);
-        if (pp + 1 < PP) fetch_g(pp + 1, ent0, g0);
-        if (pp + 2 < PP) fetch_ent(pp + 2, ent1, xw1);
-        if (one_run) {
-            // Each lane group composes its S entries, rows a_i straight from global memory to registers
-            // (entry u of the group sits in lane u / EPL of the group), then the groups' composites are
-            // joined in order and appended to the open run.
-            constexpr int UB = (S * NV <= 8) ? S : (8 / NV < 1 ? 1 : 8 / NV);  // rows requested before the first is used
-            C cur;
-            comp_identity(cur);
-#pragma unroll
-            for (int u0 = 0; u0 < S; u0 += UB) {
-                float4 av[UB][NV];
-                float eu[UB], bu[UB];
-#pragma unroll
-                for (int u = 0; u < UB; ++u) {
-                    const int src = (u0 + u) / EPL, reg = (u0 + u) % EPL;
-                    const uint32_t il = __shfl_sync(0xFFFFFFFFu, ilq[reg], src, LG);
-                    eu[u] = __shfl_sync(0xFFFFFFFFu, eq[reg], src, LG);
-                    bu[u] = __shfl_sync(0xFFFFFFFFu, bq[reg], src, LG);
-#pragma unroll
-                    for (int v = 0; v < NV; ++v) av[u][v] = __ldcg(A4 + (size_t)il * KP4 + v * LG + l);
-                }
-#pragma unroll
-                for (int u = 0; u < UB; ++u) {
-                    const float e = eu[u], b = bu[u];
-                    cur.D = fmaf(-e, cur.D, cur.D - e);
-                    cur.Dw = fmaf(-ew, cur.Dw, cur.Dw - ew);
-                    cur.Bw = fmaf(-ew, cur.Bw, cur.Bw + b);
-#pragma unroll
-                    for (int v = 0; v < NV; ++v) {
-                        cur.B[v].x = fmaf(b, av[u][v].x, fmaf(-e, cur.B[v].x, cur.B[v].x));
-                        cur.B[v].y = fmaf(b, av[u][v].y, fmaf(-e, cur.B[v].y, cur.B[v].y));
-                        cur.B[v].z = fmaf(b, av[u][v].z, fmaf(-e, cur.B[v].z, cur.B[v].z));
-                        cur.B[v].w = fmaf(b, av[u][v].w, fmaf(-e, cur.B[v].w, cur.B[v].w));
-                    }
-                }
-            }
-            if (GW > 1) {
-#pragma unroll
-                for (int delta = 1; delta < GW; delta <<= 1) {
-                    const C o = comp_shfl_down<NV>(cur, delta * LG);
-                    if ((g & (2 * delta - 1)) == 0) cur = compose<NV>(cur, o);
-                }
-                cur = comp_shfl<NV>(cur, l);  // group 0 holds the whole pass
-            }
-            wcarry = compose<NV>(wcarry, cur);
-            last_col = before;
-            continue;
-        }
-        //    scale pairs of the columns whose runs end in this pass (an entry ends a run when the
-        //    next entry has another column)
-        {
-            // the entry after this lane's last one is held by the next lane that holds entries
-            const int next_lane = (slot0 + EPL < S) ? lane + 1 : (g + 1) * LG;
-            const uint32_t first_of_next = __shfl_sync(0xFFFFFFFFu, jq[0], next_lane & 31);
-#pragma unroll
-            for (int q = 0; q < EPL; ++q) {
-                const int at = at0 + q;
-                const uint32_t nextcol = (q + 1 < EPL && slot0 + q + 1 < S) ? jq[q + 1 < EPL ? q + 1 : q] : first_of_next;
-                bool ends;
-                if (at + 1 < cnt) ends = nextcol != jq[q];
-                else ends = after_known && after != jq[q];
-                if (slot0 + q < S && at < cnt && ends) cp_async16(s_scale + slot0 + q, Sc + jq[q]);
-            }
-        }
-        __syncwarp();
-        // 2. gather the rows a_i of the pass
-#pragma unroll
-        for (int it = 0; it < PASS * KP4 / 32; ++it) {
-            const int idx = lane + 32 * it;
-            const int at = idx / KP4, part = idx % KP4;
-            if (at < cnt) {
-                const uint32_t il = __float_as_uint(sw[L::ITEMS + (at / S) * L::ITEM_STRIDE + (at % S)].z);
-                cp_async16(sw + L::ROWS + (at / S) * L::ROW_STRIDE + (at % S) * KP4 + part, A4 + (size_t)il * KP4 + part);
-            }
-        }
-        {
-            const int at = cnt - 1;
-            last_col = __float_as_uint(sw[L::ITEMS + (at / S) * L::ITEM_STRIDE + (at % S)].w);
-        }
-        cp_async_wait_all();
-        __syncwarp();
-
-        // 3. sequential walk of each lane group.  A run that ends before entry u is parked in the
-        //    slots of entry u-1, which have been consumed: offsets over its row, {D, Dw, Bw} over
-        //    its item.  The first such run of the group is its head piece; the others started inside
-        //    the group and are marked in `emask` for step 5.
-        const int lo = g * S;
-        const int len = (lo >= cnt) ? 0 : ((cnt - lo < S) ? cnt - lo : S);
-        bool hasb = false;
-        int head_pos = -1;
-        uint32_t headcol = kNoCol, emask = 0;
-        C cur;
-        comp_identity(cur);
-        if (len > 0) {
-            uint32_t prevj = (lo == 0) ? before
-                                       : __float_as_uint(sw[L::ITEMS + (g - 1) * L::ITEM_STRIDE + (S - 1)].w);
-#pragma unroll
-            for (int u = 0; u < S; ++u) {
-                if (u < len) {
-                    const float4 it = s_item[u];
-                    float4 av[NV];
-#pragma unroll
-                    for (int v = 0; v < NV; ++v) av[v] = s_rows[u * KP4 + v * LG + l];
-                    const uint32_t jl = __float_as_uint(it.w);
-                    if (jl != prevj) {  // boundary before this entry
-                        if (u > 0) {
-#pragma unroll
-                            for (int v = 0; v < NV; ++v) s_rows[(u - 1) * KP4 + v * LG + l] = cur.B[v];
-                            if (l == 0) s_item[u - 1] = make_float4(cur.D, cur.Dw, cur.Bw, __uint_as_float(prevj));
-                        }
-                        if (!hasb) { hasb = true; headcol = prevj; head_pos = u - 1; }
-                        else emask |= 1u << (u - 1);
-                        comp_identity(cur);
-                        prevj = jl;
-                    }
-                    const float e = it.x, b = it.y;
-                    cur.D = fmaf(-e, cur.D, cur.D - e);
-                    cur.Dw = fmaf(-ew, cur.Dw, cur.Dw - ew);
-                    cur.Bw = fmaf(-ew, cur.Bw, cur.Bw + b);
-#pragma unroll
-                    for (int v = 0; v < NV; ++v) {
-                        cur.B[v].x = fmaf(b, av[v].x, fmaf(-e, cur.B[v].x, cur.B[v].x));
-                        cur.B[v].y = fmaf(b, av[v].y, fmaf(-e, cur.B[v].y, cur.B[v].y));
-                        cur.B[v].z = fmaf(b, av[v].z, fmaf(-e, cur.B[v].z, cur.B[v].z));
-                        cur.B[v].w = fmaf(b, av[v].w, fmaf(-e, cur.B[v].w, cur.B[v].w));
-                    }
-                }
-            }
-        }
-        // 4. join the pieces across the lane groups
-        C head, closing;
-        comp_identity(head);
-        __syncwarp();
-        if (hasb && head_pos >= 0) {
-#pragma unroll
-            for (int v = 0; v < NV; ++v) head.B[v] = s_rows[head_pos * KP4 + v * LG + l];
-            const float4 hd = s_item[head_pos];
-            head.D = hd.x; head.Dw = hd.y; head.Bw = hd.z;
-        }
-        bool outer;
-        scan_step<LG, NV>(hasb, head, cur, wcarry, wflag, closing, outer);
-        if (hasb) {
-            if (outer) {
-                comp_store<LG, NV>(s_wpiece + (warp * 2 + 0) * (KP4 + 1), closing, headcol, l);
-            } else if (headcol != kNoCol) {
-                // the run ended at entry lo + head_pos of this pass if that is >= 0 (its scale pair
-                // was prefetched there), else in an earlier pass
-                const int pos = lo + head_pos;
-                if (pos >= 0) apply(headcol, closing, s_scale_all[(pos / S) * L::ITEM_STRIDE + (pos % S)]);
-                else apply_fetch(headcol, closing);
-            }
-        }
-        // 5. apply the runs parked in step 3, all lane groups side by side
-        while (__any_sync(0xFFFFFFFFu, emask != 0)) {
-            if (emask != 0) {
-                const int pos = __ffs(emask) - 1;
-                emask &= emask - 1;
-                C x;
-#pragma unroll
-                for (int v = 0; v < NV; ++v) x.B[v] = s_rows[pos * KP4 + v * LG + l];
-                const float4 hd = s_item[pos];
-                x.D = hd.x; x.Dw = hd.y; x.Bw = hd.z;
-                apply(__float_as_uint(hd.w), x, s_scale[pos]);
-            }
-        }
-        __syncwarp();
-    }
-    if (lane < LG) {
-        comp_store<LG, NV>(s_wpiece + (warp * 2 + 1) * (KP4 + 1), wcarry, last_col, l);
-        if (l == 0) s_wflag[warp] = wflag ? 1 : 0;
-    }
-    // with several warps, each orders its own state updates before the tile's completion signal below
-    // (warp 0 fences again before it signals)
-    if (NW > 1) __threadfence();
-    __syncthreads();
-    if (warp != 0) return;
-
-    // ---------------- chunk phase: warp 0 joins the warps ----------------
-    const int nchunks = (int)((te - tb + a.chunk_len - 1) / a.chunk_len);
-    C ccarry;
-    comp_identity(ccarry);
-    bool cflag = false;
-    uint32_t ctailcol = kNoCol;
-    for (int w0 = 0; w0 < NW; w0 += GW) {
-        const int w = w0 + g;
-        bool hasb = false;
-        uint32_t headcol = kNoCol;
-        C head, cur, closing;
-        comp_identity(head);
-        comp_identity(cur);
-        if (w < NW) {
-            comp_load<LG, NV>(s_wpiece + (w * 2 + 1) * (KP4 + 1), cur, l);
-            if (s_wflag[w]) {
-                hasb = true;
-                headcol = comp_load<LG, NV>(s_wpiece + (w * 2 + 0) * (KP4 + 1), head, l);
-            }
-        }
-        bool outer;
-        scan_step<LG, NV>(hasb, head, cur, ccarry, cflag, closing, outer);
-        if (hasb) {
-            if (outer) comp_store<LG, NV>(s_cpiece, closing, headcol, l);
-            else apply_fetch(headcol, closing);
-        }
-    }
-    for (int w = 0; w < NW; ++w) {
-        const uint32_t tc = __float_as_uint(s_wpiece[(w * 2 + 1) * (KP4 + 1) + KP4].w);
-        if (tc != kNoCol) ctailcol = tc;
-    }
-    __syncwarp();
-    if (nchunks == 1) {
-        // the tile starts and ends in this chunk: its head piece belongs to no column, and the end
-        // of the tile closes the run that is still open
-        if (g == 0) apply_fetch(ctailcol, ccarry);
-        __threadfence();
-        __syncwarp();
-        if (lane == 0) atomicAdd(a.sync + sync_done(c), 1);  // this tile of column block c is done
-        return;
-    }
-    {
-        float4 *rec4 = reinterpret_cast<float4 *>(a.records) + (size_t)chunk * REC4;
-        if (lane < LG) {
-            if (l == 0) {
-                rec4[0] = cflag ? s_cpiece[KP4] : make_float4(0.f, 0.f, 0.f, __uint_as_float(kNoCol));
-                rec4[1] = make_float4(ccarry.D, ccarry.Dw, ccarry.Bw, __uint_as_float(ctailcol));
-                rec4[2] = make_float4(__uint_as_float(cflag ? 1u : 0u), 0.f, 0.f, 0.f);
-            }
-#pragma unroll
-            for (int v = 0; v < NV; ++v) {
-                rec4[3 + v * LG + l] = cflag ? s_cpiece[v * LG + l] : make_float4(0.f, 0.f, 0.f, 0.f);
-                rec4[3 + KP4 + v * LG + l] = ccarry.B[v];
-            }
-        }
-    }
-
-    // ---------------- tile phase: the chunk that finishes last joins the chunks ----------------
-    __threadfence();
-    __syncwarp();
-    int last = 0;
-    if (lane == 0) last = (atomicAdd(a.tile_count + t, 1) == nchunks - 1) ? 1 : 0;
-    last = __shfl_sync(0xFFFFFFFFu, last, 0);
-    if (!last) return;
-    __threadfence();
-    const float4 *base4 = reinterpret_cast<const float4 *>(a.records) + ((size_t)chunk - (size_t)cm.y) * REC4;
-    C tcarry;
-    comp_identity(tcarry);
-    bool tflag = false;
-    // The next tile of this column block waits for this loop, so the records (and the scale pair of each
-    // record's head column) of step k0 + GW are fetched before step k0 is scanned: one memory latency
-    // for the whole loop instead of two per step.
-    struct Rec {
-        bool hasb;
-        uint32_t headcol;
-        C head, cur;
-        float4 sc;
-    };
-    auto load_rec = [&](int k, Rec &x) {
-        x.hasb = false;
-        x.headcol = kNoCol;
-        comp_identity(x.head);
-        comp_identity(x.cur);
-        x.sc = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (k < nchunks) {
-            const float4 *rec4 = base4 + (size_t)k * REC4;
-            const float4 hh = __ldcg(rec4 + 0);
-            const float4 th = __ldcg(rec4 + 1);
-            x.hasb = __float_as_uint(__ldcg(rec4 + 2).x) != 0u;
-            x.head.D = hh.x; x.head.Dw = hh.y; x.head.Bw = hh.z;
-            x.headcol = __float_as_uint(hh.w);
-            x.cur.D = th.x; x.cur.Dw = th.y; x.cur.Bw = th.z;
-#pragma unroll
-            for (int v = 0; v < NV; ++v) {
-                x.head.B[v] = __ldcg(rec4 + 3 + v * LG + l);
-                x.cur.B[v] = __ldcg(rec4 + 3 + KP4 + v * LG + l);
-            }
-            // no chunk of this tile applies to a head column: its run is still open until this loop
-            if (x.hasb && x.headcol != kNoCol) x.sc = __ldcg(Sc + x.headcol);
-        }
-    };
-    Rec nxt;
-    load_rec(g, nxt);
-    for (int k0 = 0; k0 < nchunks; k0 += GW) {
-        const Rec now = nxt;
-        if (k0 + GW < nchunks) load_rec(k0 + GW + g, nxt);
-        C closing;
-        bool outer;
-        scan_step<LG, NV>(now.hasb, now.head, now.cur, tcarry, tflag, closing, outer);
-        // the first boundary of a tile is its start, whose head column is kNoCol: nothing to apply
-        if (now.hasb && now.headcol != kNoCol) apply(now.headcol, closing, now.sc);
-    }
-    const uint32_t ttailcol = __float_as_uint(__ldcg(base4 + (size_t)(nchunks - 1) * REC4 + 1).w);
-    if (g == 0) apply_fetch(ttailcol, tcarry);  // the end of the tile closes the last run
-    __threadfence();
-    __syncwarp();
     if (lane == 0) {
-        a.tile_count[t] = 0;
-        atomicAdd(a.sync + sync_done(c), 1);  // this tile of column block c is done
+        mbar_init(mbar + 0, 1);
+        mbar_init(mbar + 1, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    __syncwarp();
+
+    const float4 *A4 = reinterpret_cast<const float4 *>(a.A);
+    const int *dints = reinterpret_cast<const int *>(a.desc);
+    const uint32_t jmask = a.jbits >= 32 ? 0xFFFFFFFFu : ((1u << a.jbits) - 1u);
+    const unsigned nch = (unsigned)a.nchunks;
+    int *err_word = a.sync + kSyncError;
+
+    // ---- helpers of the chunk pipeline ----
+    auto take_ticket = [&]() -> int {      // the value is valid in lane 0 only (nobody waits for it here)
+        int t = 0;
+        if (lane == 0) t = atomicAdd(a.sync + kSyncTicket, 1);
+        return t;
+    };
+    auto load_desc = [&](int tk) -> int {  // lane f < 16 holds field f of the descriptor
+        int v = 0;
+        if ((unsigned)tk < nch && lane < 16) v = __ldg(dints + (size_t)tk * 16 + lane);
+        return v;
+    };
+    auto issue_entries = [&](int64_t off, int len, int buf) {
+        const int64_t a0 = off & ~(int64_t)3;
+        const int cnt4 = (int)(((off + len + 3) & ~(int64_t)3) - a0);
+        if (lane == 0) {
+            mbar_expect_tx(mbar + buf, (unsigned)cnt4 * (WIDE ? 12u : 8u));
+            bulk_copy_g2s(ebuf + (size_t)buf * ecap, a.ent + a0, (unsigned)cnt4 * 8u, mbar + buf);
+            if (WIDE) bulk_copy_g2s(xbuf + (size_t)buf * ecap, a.xw + a0, (unsigned)cnt4 * 4u, mbar + buf);
+        }
+    };
+    auto wait_entries = [&](int buf, unsigned parity) -> bool {
+        for (int spin = 0; spin < kCopySpinLimit; ++spin)
+            if (mbar_try_wait(mbar + buf, parity)) return true;
+        return false;
+    };
+    auto fail = [&](int code) {
+        if (lane == 0) {
+            atomicCAS(err_word, 0, code);
+            atomicMax(a.sync + kSyncTicket, kTicketStop);
+        }
+    };
+    // wait until `need` earlier tiles of column block cblock are done
+    auto wait_dep = [&](int cblock, int need) -> bool {
+        int ok = 1;
+        if (lane == 0 && need > 0) {
+            const int *done = a.sync + sync_done(cblock);
+            for (int spin = 0; ld_acquire(done) < need; ++spin) {
+                if (*(volatile int *)err_word != 0 || spin >= a.spin_limit) { ok = 0; break; }
+                __nanosleep(100);
+            }
+        }
+        ok = __shfl_sync(FULL, ok, 0);
+        return ok != 0;
+    };
+
+    // ---- prologue of the pipeline ----
+    int tk0 = __shfl_sync(FULL, take_ticket(), 0);
+    if ((unsigned)tk0 >= nch) return;
+    int dc = load_desc(tk0);
+    int tk1 = __shfl_sync(FULL, take_ticket(), 0);
+    int dn = load_desc(tk1);
+    int tk2_raw = ((unsigned)tk1 < nch) ? take_ticket() : kTicketStop;
+    int buf = 0;
+    unsigned parity_bits = 0;   // bit b: parity the next wait on buffer b expects
+    bool pending_next = false;  // a bulk copy into the other buffer is under way
+    {
+        const int64_t off = ((int64_t)(uint32_t)__shfl_sync(FULL, dc, 0)) | ((int64_t)__shfl_sync(FULL, dc, 1) << 32);
+        issue_entries(off, __shfl_sync(FULL, dc, 2), 0);
+    }
+
+    for (;;) {
+        // ---- fields of the current chunk ----
+        const int64_t off = ((int64_t)(uint32_t)__shfl_sync(FULL, dc, 0)) | ((int64_t)__shfl_sync(FULL, dc, 1) << 32);
+        const int len = __shfl_sync(FULL, dc, 2);
+        const int flags = __shfl_sync(FULL, dc, 3);
+        const int row0 = __shfl_sync(FULL, dc, 4);
+        const int col0 = __shfl_sync(FULL, dc, 5);
+        const int cblock = __shfl_sync(FULL, dc, 6);
+        const int need = __shfl_sync(FULL, dc, 7);
+        const int tile = __shfl_sync(FULL, dc, 8);
+        const int tile_chunks = __shfl_sync(FULL, dc, 9);
+        const bool is_slice = (flags & kChunkSlice) != 0;
+        const bool tail_mode = (flags & kChunkTail) != 0;
+
+        // the next chunk's entries start their way into the other buffer (whose last reader, chunk n-1, is done)
+        __syncwarp();
+        pending_next = false;
+        if ((unsigned)tk1 < nch) {
+            const int64_t off1 = ((int64_t)(uint32_t)__shfl_sync(FULL, dn, 0)) | ((int64_t)__shfl_sync(FULL, dn, 1) << 32);
+            issue_entries(off1, __shfl_sync(FULL, dn, 2), buf ^ 1);
+            pending_next = true;
+        }
+        bool ok = wait_entries(buf, (parity_bits >> buf) & 1u);
+        parity_bits ^= 1u << buf;
+        if (!ok) { fail(2); break; }
+
+        const int shift = (int)(off & 3);
+        const uint2 *eb = ebuf + (size_t)buf * ecap + shift;
+        const float *xb = xbuf + (size_t)buf * ecap + shift;
+        const float4 *A4r = A4 + (size_t)row0 * KP4;
+        const float *Gr = a.G + row0;
+        float4 *U4 = reinterpret_cast<float4 *>(tail_mode ? a.Tb : a.V) + (size_t)col0 * KP4;
+        float *uw = (tail_mode ? a.Tw : a.w) + col0;
+        float2 *Sc = (tail_mode ? a.TS : a.S) + col0;
+        DSF_CHECK(len >= 1 && len <= a.chunk_len, 10, len);
+
+        // column state <- run, by the lanes of one group (all of them give the same scalars)
+        auto apply = [&](uint32_t col, float sigma, float mj_bits, float Drun, float m_bits, const float4 (&sum)[NV],
+                         float sumw) {
+            const float inv = rcp_fast(1.0f + sigma);
+#pragma unroll
+            for (int v = 0; v < NV; ++v)
+                red_add4(U4 + (size_t)col * KP4 + v * LG + l, sum[v].x * inv, sum[v].y * inv, sum[v].z * inv,
+                         sum[v].w * inv);
+            if (l == 0) {
+                const int mj = __float_as_int(mj_bits);
+                red_add1(uw + col, sumw * ex2_fast((float)mj * a.kappa_w));
+                Sc[col] = make_float2(fmaf(sigma, Drun, sigma + Drun), __int_as_float(mj + __float_as_int(m_bits)));
+            }
+        };
+        // sum over the lane groups, in a fixed order; every lane ends with the total
+        auto reduce_groups = [&](float4 (&x)[NV], float &xw_) {
+#pragma unroll
+            for (int o = LG; o < 32; o <<= 1) {
+#pragma unroll
+                for (int v = 0; v < NV; ++v) {
+                    x[v].x += __shfl_xor_sync(FULL, x[v].x, o);
+                    x[v].y += __shfl_xor_sync(FULL, x[v].y, o);
+                    x[v].z += __shfl_xor_sync(FULL, x[v].z, o);
+                    x[v].w += __shfl_xor_sync(FULL, x[v].w, o);
+                }
+                xw_ += __shfl_xor_sync(FULL, xw_, o);
+            }
+        };
+
+        bool alive = true;
+        if (!is_slice) alive = wait_dep(cblock, need);   // a slice touches column state only when it joins its run
+        if (!alive) { fail(1); break; }
+
+        // ---- the chunk ----
+        const int npass = (len + 31) >> 5;
+        const int nstage = (len + RST - 1) / RST;
+        auto issue_rows = [&](int s, int ring) {   // rows of stage s into ring slot `ring`
+            const int e0 = s * RST;
+            float4 *dst = rowb + ring * (RST * KP4);
+#pragma unroll
+            for (int it = 0; it < RST * KP4 / 32; ++it) {
+                const int idx = lane + 32 * it;
+                const int ge = e0 + idx / KP4;
+                if (ge < len) {
+                    const uint32_t il = WIDE ? eb[ge].x : (eb[ge].x >> a.jbits);
+                    if (DSF_OK(true)) cp_async16(dst + idx, A4r + (size_t)il * KP4 + (idx % KP4));
+                }
+            }
+        };
+        int ring_issue = 0, ring_use = 0;   // ring slots of the next stage to request / to work on
+#pragma unroll
+        for (int s = 0; s < PD; ++s) {
+            if (s < nstage) issue_rows(s, ring_issue);
+            cp_async_commit();
+            ring_issue = (ring_issue + 1 == NBUF) ? 0 : ring_issue + 1;
+        }
+        // scalars of a pass, requested one pass ahead: column, x, G_i, run start, scale record
+        uint32_t jl_c = kNoCol, jl_n = kNoCol;
+        float x_c = 0.f, x_n = 0.f, g_c = 0.f, g_n = 0.f;
+        float2 sc_c = make_float2(0.f, 0.f), sc_n = make_float2(0.f, 0.f);
+        bool bnd_c = false, bnd_n = false;
+        const uint32_t col_init = is_slice ? (uint32_t)__shfl_sync(FULL, dc, 14) : kNoCol;
+        auto fetch_pass = [&](int k, uint32_t prev_last) {   // -> *_n
+            const int at = 32 * k + lane;
+            jl_n = kNoCol; x_n = 0.f; g_n = 0.f;
+            if (at < len) {
+                const uint2 rec = eb[at];
+                uint32_t il;
+                if (WIDE) { il = rec.x; jl_n = rec.y; x_n = xb[at]; }
+                else { il = rec.x >> a.jbits; jl_n = rec.x & jmask; x_n = __uint_as_float(rec.y); }
+                g_n = __ldg(Gr + il);
+            }
+            uint32_t prevj = __shfl_up_sync(FULL, jl_n, 1);
+            if (lane == 0) prevj = prev_last;
+            bnd_n = (at < len) && (jl_n != prevj);
+            if (bnd_n) sc_n = __ldcg(Sc + jl_n);
+        };
+        fetch_pass(0, col_init);
+
+        float4 acc[NV];   // this lane group's share of the run that is open
+        float accw = 0.f;
+#pragma unroll
+        for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+        bool open_valid = is_slice;          // a run is open (for a slice: the run it belongs to)
+        uint32_t open_col = col_init;
+        float open_sigma = 0.f, open_mj = 0.f;   // its column's scale record as read at the run's start
+        float D_open = 0.f;                  // product - 1 of the open run so far
+        int m_open = 0;                      // its length so far
+
+        for (int k = 0; k < npass; ++k) {
+            const int cnt = (len - 32 * k) < 32 ? (len - 32 * k) : 32;
+            jl_c = jl_n; x_c = x_n; g_c = g_n; sc_c = sc_n; bnd_c = bnd_n;
+            if (k + 1 < npass) fetch_pass(k + 1, __shfl_sync(FULL, jl_c, 31));
+
+            // ---- scalar stage ----
+            const uint32_t mask = __ballot_sync(FULL, bnd_c);
+            {
+                float e = 0.f, b = 0.f;
+                if (lane < cnt) {
+                    const float gx = g_c * x_c;
+                    e = a.h * (a.lambda_v - gx * x_c);
+                    b = -a.h * gx;
+                }
+                const uint32_t below = mask & (0xFFFFFFFFu >> (31 - lane));   // run starts at or before this lane
+                const int lim = below == 0 ? lane : lane - (31 - __clz(below));   // earlier lanes of the same run
+                float D = -e;
+#pragma unroll
+                for (int delta = 1; delta < 32; delta <<= 1) {
+                    const float up = __shfl_up_sync(FULL, D, delta);
+                    if (delta <= lim) D = fmaf(up, D, up + D);
+                }
+                int m = lim + 1;
+                if (below == 0) { D = fmaf(D_open, D, D_open + D); m += m_open; }
+                const float c = b * rcp_fast(1.0f + D);
+                const float cw = b * ex2_fast((float)m * a.kappa_w);
+                pe[lane] = make_float4(c, cw, D, __int_as_float(m));
+                if (bnd_c) {
+                    ps[lane] = make_float4(__uint_as_float(jl_c), sc_c.x, sc_c.y, 0.f);
+                    segpos[__popc(mask & ((1u << lane) - 1u))] = lane;
+                }
+                if (lane == 0) segpos[__popc(mask)] = cnt;
+            }
+            __syncwarp();
+
+            // ---- K-wide stages of this pass ----
+#pragma unroll
+            for (int sp = 0; sp < SP; ++sp) {
+                const int s = k * SP + sp;
+                if (s >= nstage) break;
+                if (s + PD < nstage) issue_rows(s + PD, ring_issue);
+                cp_async_commit();
+                ring_issue = (ring_issue + 1 == NBUF) ? 0 : ring_issue + 1;
+                cp_async_wait<PD>();
+                __syncwarp();
+                const float4 *rb = rowb + ring_use * (RST * KP4);
+                ring_use = (ring_use + 1 == NBUF) ? 0 : ring_use + 1;
+                const int e0 = sp * RST;
+                const int e1 = (e0 + RST < cnt) ? e0 + RST : cnt;
+                // entries [b0, b1) of the pass, entry u to lane group (u - b0) mod GW, into (acc, accw)
+                auto add_spread = [&](int b0, int b1) {
+                    for (int u = b0 + g; u < b1; u += GW) {
+                        const float4 cf = pe[u];
+#pragma unroll
+                        for (int v = 0; v < NV; ++v) {
+                            const float4 r = rb[(u - e0) * KP4 + v * LG + l];
+                            acc[v].x = fmaf(cf.x, r.x, acc[v].x); acc[v].y = fmaf(cf.x, r.y, acc[v].y);
+                            acc[v].z = fmaf(cf.x, r.z, acc[v].z); acc[v].w = fmaf(cf.x, r.w, acc[v].w);
+                        }
+                        accw += cf.y;
+                    }
+                };
+                const uint32_t range = (e1 >= 32 ? 0xFFFFFFFFu : ((1u << e1) - 1u)) & ~((1u << e0) - 1u);
+                const uint32_t sub = mask & range;
+                if (sub == 0) {
+                    if (e1 - e0 == RST) {
+                        // a whole stage inside one run: the common case on click-log data
+#pragma unroll
+                        for (int q = 0; q < RST / GW; ++q) {
+                            const int u = e0 + q * GW + g;
+                            const float4 cf = pe[u];
+#pragma unroll
+                            for (int v = 0; v < NV; ++v) {
+                                const float4 r = rb[(q * GW + g) * KP4 + v * LG + l];
+                                acc[v].x = fmaf(cf.x, r.x, acc[v].x); acc[v].y = fmaf(cf.x, r.y, acc[v].y);
+                                acc[v].z = fmaf(cf.x, r.z, acc[v].z); acc[v].w = fmaf(cf.x, r.w, acc[v].w);
+                            }
+                            accw += cf.y;
+                        }
+                    } else {
+                        add_spread(e0, e1);
+                    }
+                } else {
+                    const int F = __ffs(sub) - 1, Lb = 31 - __clz(sub);
+                    // 1. what is left of the open run, then the open run ends
+                    add_spread(e0, F);
+                    if (open_valid) {
+                        reduce_groups(acc, accw);
+                        if (g == 0) {
+                            float Dc = D_open;
+                            float mc = __int_as_float(m_open);
+                            if (F > 0) { const float4 en = pe[F - 1]; Dc = en.z; mc = en.w; }
+                            apply(open_col, open_sigma, open_mj, Dc, mc, acc, accw);
+                        }
+                    }
+#pragma unroll
+                    for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    accw = 0.f;
+                    // 2. runs that start and end inside the stage: one lane group each
+                    const int i0 = __popc(mask & ((1u << F) - 1u));
+                    const int nmid = __popc(sub) - 1;
+                    for (int i = g; i < nmid; i += GW) {
+                        const int s0 = segpos[i0 + i], s1 = segpos[i0 + i + 1];
+                        float4 tmp[NV];
+                        float tmpw = 0.f;
+#pragma unroll
+                        for (int v = 0; v < NV; ++v) tmp[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        for (int u = s0; u < s1; ++u) {
+                            const float4 cf = pe[u];
+#pragma unroll
+                            for (int v = 0; v < NV; ++v) {
+                                const float4 r = rb[(u - e0) * KP4 + v * LG + l];
+                                tmp[v].x = fmaf(cf.x, r.x, tmp[v].x); tmp[v].y = fmaf(cf.x, r.y, tmp[v].y);
+                                tmp[v].z = fmaf(cf.x, r.z, tmp[v].z); tmp[v].w = fmaf(cf.x, r.w, tmp[v].w);
+                            }
+                            tmpw += cf.y;
+                        }
+                        const float4 st = ps[s0], en = pe[s1 - 1];
+                        DSF_CHECK(s0 >= e0 && s1 > s0 && s1 <= e1, 11, s0 * 64 + s1);
+                        apply(__float_as_uint(st.x), st.y, st.z, en.z, en.w, tmp, tmpw);
+                    }
+                    __syncwarp();
+                    // 3. the run that is open at the end of the stage
+                    add_spread(Lb, e1);
+                    const float4 st = ps[Lb];
+                    open_valid = true;
+                    open_col = __float_as_uint(st.x);
+                    open_sigma = st.y;
+                    open_mj = st.z;
+                }
+                __syncwarp();
+            }
+            {
+                const float4 en = pe[cnt - 1];   // the open run up to the end of this pass
+                D_open = en.z;
+                m_open = __float_as_int(en.w);
+            }
+            __syncwarp();
+        }
+        cp_async_wait<0>();
+
+        // ---- end of the chunk ----
+        reduce_groups(acc, accw);
+        if (!is_slice) {
+            if (open_valid && g == 0) apply(open_col, open_sigma, open_mj, D_open, __int_as_float(m_open), acc, accw);
+        } else {
+            const int run_id = __shfl_sync(FULL, dc, 10), slice = __shfl_sync(FULL, dc, 11);
+            const int nslices = __shfl_sync(FULL, dc, 12), rec0 = __shfl_sync(FULL, dc, 13);
+            float4 *rec4 = reinterpret_cast<float4 *>(a.records) + ((size_t)rec0 + slice) * (KP4 + 1);
+            if (g == 0) {
+                if (l == 0) rec4[0] = make_float4(D_open, __int_as_float(m_open), accw, 0.f);
+#pragma unroll
+                for (int v = 0; v < NV; ++v) rec4[1 + v * LG + l] = acc[v];
+            }
+            __threadfence();
+            __syncwarp();
+            int last = 0;
+            if (lane == 0) last = (atomicAdd(a.run_count + run_id, 1) == nslices - 1) ? 1 : 0;
+            last = __shfl_sync(FULL, last, 0);
+            if (last) {
+                // the slice that finishes last joins the run: scalar prefixes over the slices, then the weighted
+                // sum of their K-wide parts, in a fixed order
+                __threadfence();
+                if (!wait_dep(cblock, need)) { fail(1); break; }
+                const float4 *rbase = reinterpret_cast<const float4 *>(a.records) + (size_t)rec0 * (KP4 + 1);
+                float Dp = 0.f, wt = 0.f;
+                int mp = 0;
+                float4 ut[NV];
+#pragma unroll
+                for (int v = 0; v < NV; ++v) ut[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int base = 0; base < nslices; base += 32) {
+                    const int kx = base + lane;
+                    float4 hd = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (kx < nslices) hd = __ldcg(rbase + (size_t)kx * (KP4 + 1));
+                    float Di = hd.x;
+                    int mi = __float_as_int(hd.y);
+#pragma unroll
+                    for (int delta = 1; delta < 32; delta <<= 1) {
+                        const float upD = __shfl_up_sync(FULL, Di, delta);
+                        const int upm = __shfl_up_sync(FULL, mi, delta);
+                        if (lane >= delta) { Di = fmaf(upD, Di, upD + Di); mi += upm; }
+                    }
+                    float Dex = __shfl_up_sync(FULL, Di, 1);
+                    int mex = __shfl_up_sync(FULL, mi, 1);
+                    if (lane == 0) { Dex = 0.f; mex = 0; }
+                    Dex = fmaf(Dp, Dex, Dp + Dex);
+                    mex += mp;
+                    const float sv = rcp_fast(1.0f + Dex);
+                    wt = fmaf(hd.z, ex2_fast((float)mex * a.kappa_w), wt);
+#pragma unroll
+                    for (int q = 0; q < 32 / GW; ++q) {
+                        const int kk = q * GW + g;
+                        const float s_ = __shfl_sync(FULL, sv, kk);
+                        if (base + kk < nslices) {
+#pragma unroll
+                            for (int v = 0; v < NV; ++v) {
+                                const float4 r = __ldcg(rbase + (size_t)(base + kk) * (KP4 + 1) + 1 + v * LG + l);
+                                ut[v].x = fmaf(s_, r.x, ut[v].x); ut[v].y = fmaf(s_, r.y, ut[v].y);
+                                ut[v].z = fmaf(s_, r.z, ut[v].z); ut[v].w = fmaf(s_, r.w, ut[v].w);
+                            }
+                        }
+                    }
+                    const float Dt = __shfl_sync(FULL, Di, 31);
+                    mp += __shfl_sync(FULL, mi, 31);
+                    Dp = fmaf(Dp, Dt, Dp + Dt);
+                }
+                float dummy = 0.f;
+                reduce_groups(ut, dummy);
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) wt += __shfl_xor_sync(FULL, wt, o);
+                const uint32_t col = (uint32_t)__shfl_sync(FULL, dc, 14);
+                if (g == 0) {
+                    const float2 sc = __ldcg(Sc + col);
+                    apply(col, sc.x, sc.y, Dp, __int_as_float(mp), ut, wt);
+                }
+                if (lane == 0) a.run_count[run_id] = 0;
+            }
+        }
+        // this chunk is done; the chunk that finishes a tile reports the tile
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) {
+            bool fin = true;
+            if (tile_chunks > 1) {
+                fin = atomicAdd(a.tile_count + tile, 1) == tile_chunks - 1;
+                if (fin) { a.tile_count[tile] = 0; __threadfence(); }
+            }
+            if (fin) atomicAdd(a.sync + sync_done(cblock), 1);
+        }
+
+        // ---- next chunk ----
+        if ((unsigned)tk1 >= nch) { pending_next = false; break; }
+        dc = dn;
+        tk0 = tk1;
+        tk1 = __shfl_sync(FULL, tk2_raw, 0);
+        dn = load_desc(tk1);
+        tk2_raw = ((unsigned)tk1 < nch) ? take_ticket() : kTicketStop;
+        buf ^= 1;
+    }
+    // leaving early: nothing may still be on its way into this warp's shared memory
+    cp_async_wait<0>();
+    if (pending_next) wait_entries(buf ^ 1, (parity_bits >> (buf ^ 1)) & 1u);
 }
 
 // End of the SGD phase: back from the scaled state to plain parameters,
-//     v_j <- (1 + D_T) ((1 + sigma_j) u_j + ub_j),   w_j likewise,
-// where T_j = (D_T, ub_j) is the tail composite (identity unless the launch order was the row-block
-// sweep), and reset of the scale pairs and of T_j.  Two kernels because the first reads the scale
-// pairs that the second clears.
-__global__ void __launch_bounds__(kThreads) sgd_finalize_v_kernel(float *V, float *Tb, const float4 *S,
-                                                                  const float4 *TS, int64_t d, int kp4) {
+//     v_j <- (1 + D_T) ((1 + sigma_j) u_j + ub_j),
+//     w_j <- (1 - ew)^{m_T} ((1 - ew)^{m_j} uw_j + ubw_j),
+// where T_j = (D_T, m_T, ub_j, ubw_j) is the tail composite (identity unless the launch order was the
+// row-block sweep), and reset of the scale records and of T_j.  Two kernels because the first reads
+// the scale records that the second clears.  log1m_ew = log(1 - ew) in double.
+__global__ void __launch_bounds__(kThreads) sgd_finalize_v_kernel(float *V, float *Tb, const float2 *S,
+                                                                  const float2 *TS, int64_t d, int kp4) {
     const int64_t total = d * kp4;
     float4 *V4 = reinterpret_cast<float4 *>(V);
     float4 *Tb4 = reinterpret_cast<float4 *>(Tb);
@@ -785,16 +711,19 @@ __global__ void __launch_bounds__(kThreads) sgd_finalize_v_kernel(float *V, floa
         V4[i] = y;
     }
 }
-__global__ void __launch_bounds__(kThreads) sgd_finalize_w_kernel(float *w, float *Tw, float4 *S, float4 *TS, int64_t d) {
+__global__ void __launch_bounds__(kThreads) sgd_finalize_w_kernel(float *w, float *Tw, float2 *S, float2 *TS, int64_t d,
+                                                                  double log1m_ew) {
     for (int64_t j = (int64_t)blockIdx.x * kThreads + threadIdx.x; j < d; j += (int64_t)gridDim.x * kThreads) {
         float wj = w[j];
-        wj = fmaf(S[j].y, wj, wj);
-        S[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+        const int mj = __float_as_int(S[j].y);
+        if (mj != 0) wj = fmaf((float)expm1((double)mj * log1m_ew), wj, wj);
+        S[j] = make_float2(0.f, 0.f);
         if (Tw != nullptr) {
             wj += Tw[j];
-            wj = fmaf(TS[j].y, wj, wj);
+            const int mt = __float_as_int(TS[j].y);
+            if (mt != 0) wj = fmaf((float)expm1((double)mt * log1m_ew), wj, wj);
             Tw[j] = 0.f;
-            TS[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+            TS[j] = make_float2(0.f, 0.f);
         }
         w[j] = wj;
     }

@@ -38,6 +38,7 @@ SIGNATURES = {
     "dsfacto_get_stats": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]),
     "dsfacto_set_stream": (ctypes.c_int, [_vp, _vp]),
     "dsfacto_last_epoch_ms": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_float)]),
+    "dsfacto_debug_set": (ctypes.c_int, [_vp, _c_i32, _c_i64]),
     "dsfacto_launch_count": (ctypes.c_int, [_vp, ctypes.POINTER(_c_i64)]),
     "dsfacto_last_error": (ctypes.c_char_p, [_vp]),
     "dsfacto_strerror": (ctypes.c_char_p, [ctypes.c_int]),
@@ -103,6 +104,13 @@ def dsfacto_set_eta(h, eta):
 
 def dsfacto_set_refresh_every(h, rounds):
     return lib().dsfacto_set_refresh_every(h, rounds)
+
+
+DEBUG_SPIN_LIMIT, DEBUG_EXTRA_NEED, DEBUG_CHUNK_LEN = 0, 1, 2
+
+
+def dsfacto_debug_set(h, key, value):
+    return lib().dsfacto_debug_set(h, key, value)
 
 
 def dsfacto_objective(h):
