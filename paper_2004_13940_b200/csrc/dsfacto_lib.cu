@@ -474,7 +474,7 @@ void run_sgd_phase(dsfacto *h, int64_t L0, int64_t L1) {
     a.ent = h->d_ent; a.xw = h->d_xw; a.A = h->d_A; a.G = h->d_G; a.w = h->d_w; a.V = h->d_V;
     a.S = h->d_S; a.Tb = h->d_Tb; a.Tw = h->d_Tw; a.TS = h->d_TS; a.records = h->d_records;
     a.tile_count = h->d_tile_count; a.run_count = h->d_run_count;
-    a.jbits = h->jbits; a.chunk_len = h->chunk_len; a.spin_limit = h->spin_limit;
+    a.n = h->n; a.d = h->d; a.jbits = h->jbits; a.chunk_len = h->chunk_len; a.spin_limit = h->spin_limit;
     a.h = h->h; a.lambda_v = h->lambda_v;
     const double ew = (double)h->h * (double)h->lambda_w;
     const double log1m_ew = std::log1p(-ew);           // log(1 - ew); -inf / NaN for absurd steps, which then diverge

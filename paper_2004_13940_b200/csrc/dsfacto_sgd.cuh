@@ -80,7 +80,7 @@ struct SgdCfg {
 __host__ __device__ constexpr int sgd_ecap(int chunk_len) { return (chunk_len + 8 + 3) & ~3; }
 template <int LG, int NV>
 __host__ __device__ constexpr size_t sgd_warp_smem(bool wide, int chunk_len) {
-    return (size_t)SgdCfg<LG, NV>::ROW4 * 16 + 32 * 16 * 2 + 40 * 4 + 16 +
+    return (size_t)SgdCfg<LG, NV>::ROW4 * 16 + 32 * 8 + 32 * 4 + 40 * 4 + 16 +
            (size_t)2 * sgd_ecap(chunk_len) * (wide ? 12 : 8);
 }
 // floats of the record a slice of a long run leaves: {D, m, W, -} and the K-wide sum
@@ -164,6 +164,7 @@ struct SgdArgs {
     int *sync;                 // sync_words(p) ints: ticket counter (zero at launch), error word, finished tiles
                                // per column block (zero at the first launch of a sweep, kept between the
                                // launches of one sweep)
+    int64_t n, d;              // rows and columns of the data set (checks of the debug build)
     int jbits;
     int chunk_len;             // longest chunk of the plan (sizes the staging buffers)
     int spin_limit;            // polls before the wait for an earlier tile gives up
@@ -236,9 +237,9 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
     const int ecap = sgd_ecap(a.chunk_len);
     unsigned char *wbase = smem_raw + (size_t)warp * sgd_warp_smem<LG, NV>(WIDE, a.chunk_len);
     float4 *rowb = reinterpret_cast<float4 *>(wbase);               // row ring
-    float4 *pe = rowb + C::ROW4;                                    // per entry of the pass: {c, cw, D, m}
-    float4 *ps = pe + 32;                                           // per run start: {column, sigma, m_j, -}
-    int *segpos = reinterpret_cast<int *>(ps + 32);                 // lane of the k-th run start of the pass (40 ints)
+    float2 *pc = reinterpret_cast<float2 *>(rowb + C::ROW4);        // per entry of the pass: {c, cw}
+    uint32_t *pcol = reinterpret_cast<uint32_t *>(pc + 32);         // per entry of the pass: local column
+    int *segpos = reinterpret_cast<int *>(pcol + 32);               // lane of the k-th run start of the pass (40 ints)
     uint64_t *mbar = reinterpret_cast<uint64_t *>(segpos + 40);     // one per entry buffer
     uint2 *ebuf = reinterpret_cast<uint2 *>(mbar + 2);              // 2 x ecap entry records
     float *xbuf = reinterpret_cast<float *>(ebuf + 2 * (size_t)ecap);  // wide layout: 2 x ecap values
@@ -287,17 +288,19 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
             atomicMax(a.sync + kSyncTicket, kTicketStop);
         }
     };
-    // wait until `need` earlier tiles of column block cblock are done
-    auto wait_dep = [&](int cblock, int need) -> bool {
+    // Wait until `need` earlier tiles of column block cblock are done.  `seen` is an earlier reading of the
+    // counter (lane 0; it only grows), so that a tile that was ready long ago costs no round trip to L2.
+    auto wait_dep = [&](int cblock, int need, int seen) -> bool {
         int ok = 1;
-        if (lane == 0 && need > 0) {
+        if (lane == 0 && seen < need) {
             const int *done = a.sync + sync_done(cblock);
             for (int spin = 0; ld_acquire(done) < need; ++spin) {
-                if (*(volatile int *)err_word != 0 || spin >= a.spin_limit) { ok = 0; break; }
-                __nanosleep(100);
+                if (spin >= a.spin_limit || ((spin & 7) == 7 && *(volatile int *)err_word != 0)) { ok = 0; break; }
+                __nanosleep(200);
             }
         }
         ok = __shfl_sync(FULL, ok, 0);
+        __syncwarp();   // lane 0's acquire comes before the other lanes' reads of the column state
         return ok != 0;
     };
 
@@ -305,12 +308,11 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
     int tk0 = __shfl_sync(FULL, take_ticket(), 0);
     if ((unsigned)tk0 >= nch) return;
     int dc = load_desc(tk0);
-    int tk1 = __shfl_sync(FULL, take_ticket(), 0);
-    int dn = load_desc(tk1);
-    int tk2_raw = ((unsigned)tk1 < nch) ? take_ticket() : kTicketStop;
+    int tk1 = kTicketStop, dn = 0, tk1_raw = 0, dep_seen_next = 0;
     int buf = 0;
     unsigned parity_bits = 0;   // bit b: parity the next wait on buffer b expects
     bool pending_next = false;  // a bulk copy into the other buffer is under way
+    int dep_seen = 0;           // lane 0: the progress counter of the chunk's column block, read ahead
     {
         const int64_t off = ((int64_t)(uint32_t)__shfl_sync(FULL, dc, 0)) | ((int64_t)__shfl_sync(FULL, dc, 1) << 32);
         issue_entries(off, __shfl_sync(FULL, dc, 2), 0);
@@ -330,14 +332,9 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
         const bool is_slice = (flags & kChunkSlice) != 0;
         const bool tail_mode = (flags & kChunkTail) != 0;
 
-        // the next chunk's entries start their way into the other buffer (whose last reader, chunk n-1, is done)
-        __syncwarp();
+        // the ticket of the next chunk is asked for now; its descriptor and entries follow during the passes
+        tk1_raw = take_ticket();
         pending_next = false;
-        if ((unsigned)tk1 < nch) {
-            const int64_t off1 = ((int64_t)(uint32_t)__shfl_sync(FULL, dn, 0)) | ((int64_t)__shfl_sync(FULL, dn, 1) << 32);
-            issue_entries(off1, __shfl_sync(FULL, dn, 2), buf ^ 1);
-            pending_next = true;
-        }
         bool ok = wait_entries(buf, (parity_bits >> buf) & 1u);
         parity_bits ^= 1u << buf;
         if (!ok) { fail(2); break; }
@@ -352,19 +349,13 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
         float2 *Sc = (tail_mode ? a.TS : a.S) + col0;
         DSF_CHECK(len >= 1 && len <= a.chunk_len, 10, len);
 
-        // column state <- run, by the lanes of one group (all of them give the same scalars)
-        auto apply = [&](uint32_t col, float sigma, float mj_bits, float Drun, float m_bits, const float4 (&sum)[NV],
-                         float sumw) {
-            const float inv = rcp_fast(1.0f + sigma);
+        // adds a finished run's sums to its column (the lanes of one group; sums already carry the column's scale)
+        auto flush = [&](uint32_t col, const float4 (&sum)[NV], float sumw) {
+            DSF_CHECK((int64_t)col0 + col < a.d, 12, col);
 #pragma unroll
             for (int v = 0; v < NV; ++v)
-                red_add4(U4 + (size_t)col * KP4 + v * LG + l, sum[v].x * inv, sum[v].y * inv, sum[v].z * inv,
-                         sum[v].w * inv);
-            if (l == 0) {
-                const int mj = __float_as_int(mj_bits);
-                red_add1(uw + col, sumw * ex2_fast((float)mj * a.kappa_w));
-                Sc[col] = make_float2(fmaf(sigma, Drun, sigma + Drun), __int_as_float(mj + __float_as_int(m_bits)));
-            }
+                red_add4(U4 + (size_t)col * KP4 + v * LG + l, sum[v].x, sum[v].y, sum[v].z, sum[v].w);
+            if (l == 0) red_add1(uw + col, sumw);
         };
         // sum over the lane groups, in a fixed order; every lane ends with the total
         auto reduce_groups = [&](float4 (&x)[NV], float &xw_) {
@@ -382,54 +373,58 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
         };
 
         bool alive = true;
-        if (!is_slice) alive = wait_dep(cblock, need);   // a slice touches column state only when it joins its run
+        if (!is_slice) alive = wait_dep(cblock, need, dep_seen);   // a slice touches column state only when it joins its run
         if (!alive) { fail(1); break; }
 
         // ---- the chunk ----
         const int npass = (len + 31) >> 5;
         const int nstage = (len + RST - 1) / RST;
-        auto issue_rows = [&](int s, int ring) {   // rows of stage s into ring slot `ring`
-            const int e0 = s * RST;
-            float4 *dst = rowb + ring * (RST * KP4);
-#pragma unroll
-            for (int it = 0; it < RST * KP4 / 32; ++it) {
-                const int idx = lane + 32 * it;
-                const int ge = e0 + idx / KP4;
-                if (ge < len) {
-                    const uint32_t il = WIDE ? eb[ge].x : (eb[ge].x >> a.jbits);
-                    if (DSF_OK(true)) cp_async16(dst + idx, A4r + (size_t)il * KP4 + (idx % KP4));
-                }
-            }
-        };
-        int ring_issue = 0, ring_use = 0;   // ring slots of the next stage to request / to work on
-#pragma unroll
-        for (int s = 0; s < PD; ++s) {
-            if (s < nstage) issue_rows(s, ring_issue);
-            cp_async_commit();
-            ring_issue = (ring_issue + 1 == NBUF) ? 0 : ring_issue + 1;
-        }
-        // scalars of a pass, requested one pass ahead: column, x, G_i, run start, scale record
-        uint32_t jl_c = kNoCol, jl_n = kNoCol;
+        // scalars of a pass, requested one pass ahead: row, column, x, G_i, run start, scale record
+        uint32_t il_c = 0, il_n = 0, jl_c = kNoCol, jl_n = kNoCol;
         float x_c = 0.f, x_n = 0.f, g_c = 0.f, g_n = 0.f;
         float2 sc_c = make_float2(0.f, 0.f), sc_n = make_float2(0.f, 0.f);
         bool bnd_c = false, bnd_n = false;
         const uint32_t col_init = is_slice ? (uint32_t)__shfl_sync(FULL, dc, 14) : kNoCol;
         auto fetch_pass = [&](int k, uint32_t prev_last) {   // -> *_n
             const int at = 32 * k + lane;
-            jl_n = kNoCol; x_n = 0.f; g_n = 0.f;
+            jl_n = kNoCol; x_n = 0.f; g_n = 0.f; il_n = 0;
             if (at < len) {
                 const uint2 rec = eb[at];
-                uint32_t il;
-                if (WIDE) { il = rec.x; jl_n = rec.y; x_n = xb[at]; }
-                else { il = rec.x >> a.jbits; jl_n = rec.x & jmask; x_n = __uint_as_float(rec.y); }
-                g_n = __ldg(Gr + il);
+                if (WIDE) { il_n = rec.x; jl_n = rec.y; x_n = xb[at]; }
+                else { il_n = rec.x >> a.jbits; jl_n = rec.x & jmask; x_n = __uint_as_float(rec.y); }
+                DSF_CHECK((int64_t)row0 + il_n < a.n, 13, il_n);
+                g_n = __ldg(Gr + il_n);
             }
             uint32_t prevj = __shfl_up_sync(FULL, jl_n, 1);
             if (lane == 0) prevj = prev_last;
             bnd_n = (at < len) && (jl_n != prevj);
             if (bnd_n) sc_n = __ldcg(Sc + jl_n);
         };
+        // rows of stage sp of a pass whose local rows are `il` (one per lane) into ring slot `ring`: lane group
+        // q of the warp fetches the row of entry sp*RST + it*GW + q, 16 bytes per lane (rows past the end of
+        // the chunk repeat row 0 of the block)
+        auto issue_rows = [&](uint32_t il, int sp, int ring) {
+            float4 *dst = rowb + ring * (RST * KP4) + g * KP4 + l;
+#pragma unroll
+            for (int it = 0; it < RST / GW; ++it) {
+                const uint32_t ir = __shfl_sync(FULL, il, sp * RST + it * GW + g);
+#pragma unroll
+                for (int v = 0; v < NV; ++v)
+                    cp_async16(dst + it * GW * KP4 + v * LG, A4r + (size_t)ir * KP4 + v * LG + l);
+            }
+        };
         fetch_pass(0, col_init);
+        il_c = il_n;
+        int ring_issue = 0, ring_use = 0;   // ring slots of the next stage to request / to work on
+        // stage s of the chunk = stage s % SP of pass s / SP; the first PD stages are requested here
+#pragma unroll
+        for (int s = 0; s < PD; ++s) {
+            if (s < SP) {   // (PD <= SP except for one-stage passes, where PD = 1 = SP)
+                if (s < nstage) issue_rows(il_n, s, ring_issue);
+            }
+            cp_async_commit();
+            ring_issue = (ring_issue + 1 == NBUF) ? 0 : ring_issue + 1;
+        }
 
         float4 acc[NV];   // this lane group's share of the run that is open
         float accw = 0.f;
@@ -437,17 +432,18 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
         for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
         bool open_valid = is_slice;          // a run is open (for a slice: the run it belongs to)
         uint32_t open_col = col_init;
-        float open_sigma = 0.f, open_mj = 0.f;   // its column's scale record as read at the run's start
-        float D_open = 0.f;                  // product - 1 of the open run so far
-        int m_open = 0;                      // its length so far
+        float D_open = 0.f;                  // (scale of the column) x (product of the open run so far) - 1
+        int m_open = 0;                      // entries of the column so far, the open run included
 
         for (int k = 0; k < npass; ++k) {
             const int cnt = (len - 32 * k) < 32 ? (len - 32 * k) : 32;
-            jl_c = jl_n; x_c = x_n; g_c = g_n; sc_c = sc_n; bnd_c = bnd_n;
+            il_c = il_n; jl_c = jl_n; x_c = x_n; g_c = g_n; sc_c = sc_n; bnd_c = bnd_n;
             if (k + 1 < npass) fetch_pass(k + 1, __shfl_sync(FULL, jl_c, 31));
 
             // ---- scalar stage ----
             const uint32_t mask = __ballot_sync(FULL, bnd_c);
+            float D;
+            int m;
             {
                 float e = 0.f, b = 0.f;
                 if (lane < cnt) {
@@ -456,23 +452,26 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
                     b = -a.h * gx;
                 }
                 const uint32_t below = mask & (0xFFFFFFFFu >> (31 - lane));   // run starts at or before this lane
-                const int lim = below == 0 ? lane : lane - (31 - __clz(below));   // earlier lanes of the same run
-                float D = -e;
+                const int start = 31 - __clz(below);                              // -1: the run was open before the pass
+                const int lim = below == 0 ? lane : lane - start;                 // earlier lanes of the same run
+                // a run starts from its column's scale, so that the sums need no scaling when they are applied
+                D = bnd_c ? fmaf(sc_c.x, -e, sc_c.x - e) : -e;
 #pragma unroll
                 for (int delta = 1; delta < 32; delta <<= 1) {
                     const float up = __shfl_up_sync(FULL, D, delta);
                     if (delta <= lim) D = fmaf(up, D, up + D);
                 }
-                int m = lim + 1;
-                if (below == 0) { D = fmaf(D_open, D, D_open + D); m += m_open; }
+                const int mj = __shfl_sync(FULL, bnd_c ? __float_as_int(sc_c.y) : 0, start < 0 ? 0 : start);
+                m = lim + 1 + mj;
+                if (below == 0) { D = fmaf(D_open, D, D_open + D); m = lane + 1 + m_open; }
                 const float c = b * rcp_fast(1.0f + D);
                 const float cw = b * ex2_fast((float)m * a.kappa_w);
-                pe[lane] = make_float4(c, cw, D, __int_as_float(m));
-                if (bnd_c) {
-                    ps[lane] = make_float4(__uint_as_float(jl_c), sc_c.x, sc_c.y, 0.f);
-                    segpos[__popc(mask & ((1u << lane) - 1u))] = lane;
-                }
+                pc[lane] = make_float2(c, cw);
+                pcol[lane] = jl_c;
+                if (bnd_c) segpos[__popc(mask & ((1u << lane) - 1u))] = lane;
                 if (lane == 0) segpos[__popc(mask)] = cnt;
+                // a run that ends inside the pass leaves its column's new scale record right here
+                if (lane + 1 < cnt && ((mask >> (lane + 1)) & 1u)) Sc[jl_c] = make_float2(D, __int_as_float(m));
             }
             __syncwarp();
 
@@ -481,7 +480,10 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
             for (int sp = 0; sp < SP; ++sp) {
                 const int s = k * SP + sp;
                 if (s >= nstage) break;
-                if (s + PD < nstage) issue_rows(s + PD, ring_issue);
+                if (s + PD < nstage) {
+                    if (sp + PD < SP) issue_rows(il_c, sp + PD, ring_issue);
+                    else issue_rows(il_n, sp + PD - SP, ring_issue);
+                }
                 cp_async_commit();
                 ring_issue = (ring_issue + 1 == NBUF) ? 0 : ring_issue + 1;
                 cp_async_wait<PD>();
@@ -493,7 +495,7 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
                 // entries [b0, b1) of the pass, entry u to lane group (u - b0) mod GW, into (acc, accw)
                 auto add_spread = [&](int b0, int b1) {
                     for (int u = b0 + g; u < b1; u += GW) {
-                        const float4 cf = pe[u];
+                        const float2 cf = pc[u];
 #pragma unroll
                         for (int v = 0; v < NV; ++v) {
                             const float4 r = rb[(u - e0) * KP4 + v * LG + l];
@@ -510,8 +512,7 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
                         // a whole stage inside one run: the common case on click-log data
 #pragma unroll
                         for (int q = 0; q < RST / GW; ++q) {
-                            const int u = e0 + q * GW + g;
-                            const float4 cf = pe[u];
+                            const float2 cf = pc[e0 + q * GW + g];
 #pragma unroll
                             for (int v = 0; v < NV; ++v) {
                                 const float4 r = rb[(q * GW + g) * KP4 + v * LG + l];
@@ -530,10 +531,9 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
                     if (open_valid) {
                         reduce_groups(acc, accw);
                         if (g == 0) {
-                            float Dc = D_open;
-                            float mc = __int_as_float(m_open);
-                            if (F > 0) { const float4 en = pe[F - 1]; Dc = en.z; mc = en.w; }
-                            apply(open_col, open_sigma, open_mj, Dc, mc, acc, accw);
+                            flush(open_col, acc, accw);
+                            // (a run that ends inside the pass has left its scale record in the scalar stage)
+                            if (F == 0 && l == 0) Sc[open_col] = make_float2(D_open, __int_as_float(m_open));
                         }
                     }
 #pragma unroll
@@ -544,12 +544,13 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
                     const int nmid = __popc(sub) - 1;
                     for (int i = g; i < nmid; i += GW) {
                         const int s0 = segpos[i0 + i], s1 = segpos[i0 + i + 1];
+                        DSF_CHECK(s0 >= e0 && s1 > s0 && s1 <= e1, 11, s0 * 64 + s1);
                         float4 tmp[NV];
                         float tmpw = 0.f;
 #pragma unroll
                         for (int v = 0; v < NV; ++v) tmp[v] = make_float4(0.f, 0.f, 0.f, 0.f);
                         for (int u = s0; u < s1; ++u) {
-                            const float4 cf = pe[u];
+                            const float2 cf = pc[u];
 #pragma unroll
                             for (int v = 0; v < NV; ++v) {
                                 const float4 r = rb[(u - e0) * KP4 + v * LG + l];
@@ -558,34 +559,44 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
                             }
                             tmpw += cf.y;
                         }
-                        const float4 st = ps[s0], en = pe[s1 - 1];
-                        DSF_CHECK(s0 >= e0 && s1 > s0 && s1 <= e1, 11, s0 * 64 + s1);
-                        apply(__float_as_uint(st.x), st.y, st.z, en.z, en.w, tmp, tmpw);
+                        flush(pcol[s0], tmp, tmpw);
                     }
                     __syncwarp();
                     // 3. the run that is open at the end of the stage
                     add_spread(Lb, e1);
-                    const float4 st = ps[Lb];
                     open_valid = true;
-                    open_col = __float_as_uint(st.x);
-                    open_sigma = st.y;
-                    open_mj = st.z;
+                    open_col = pcol[Lb];
                 }
                 __syncwarp();
             }
-            {
-                const float4 en = pe[cnt - 1];   // the open run up to the end of this pass
-                D_open = en.z;
-                m_open = __float_as_int(en.w);
+            // the open run up to the end of this pass
+            D_open = __shfl_sync(FULL, D, cnt - 1);
+            m_open = __shfl_sync(FULL, m, cnt - 1);
+
+            // the next chunk: its descriptor after the first pass, its entries (and a first look at the progress
+            // of its column block) a little later, so that neither request is waited for
+            if (k == 0) {
+                tk1 = __shfl_sync(FULL, tk1_raw, 0);
+                dn = load_desc(tk1);
             }
-            __syncwarp();
+            if (k == (npass > 2 ? 2 : npass - 1) && (unsigned)tk1 < nch) {
+                const int64_t off1 = ((int64_t)(uint32_t)__shfl_sync(FULL, dn, 0)) | ((int64_t)__shfl_sync(FULL, dn, 1) << 32);
+                const int len1 = __shfl_sync(FULL, dn, 2), cb1 = __shfl_sync(FULL, dn, 6);
+                __syncwarp();
+                issue_entries(off1, len1, buf ^ 1);   // the other buffer's last reader was the chunk before this one
+                pending_next = true;
+                if (lane == 0) dep_seen_next = ld_acquire(a.sync + sync_done(cb1));
+            }
         }
         cp_async_wait<0>();
 
         // ---- end of the chunk ----
         reduce_groups(acc, accw);
         if (!is_slice) {
-            if (open_valid && g == 0) apply(open_col, open_sigma, open_mj, D_open, __int_as_float(m_open), acc, accw);
+            if (open_valid && g == 0) {
+                flush(open_col, acc, accw);
+                if (l == 0) Sc[open_col] = make_float2(D_open, __int_as_float(m_open));
+            }
         } else {
             const int run_id = __shfl_sync(FULL, dc, 10), slice = __shfl_sync(FULL, dc, 11);
             const int nslices = __shfl_sync(FULL, dc, 12), rec0 = __shfl_sync(FULL, dc, 13);
@@ -602,9 +613,9 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
             last = __shfl_sync(FULL, last, 0);
             if (last) {
                 // the slice that finishes last joins the run: scalar prefixes over the slices, then the weighted
-                // sum of their K-wide parts, in a fixed order
+                // sum of their K-wide parts, in a fixed order; the column's own scale comes last
                 __threadfence();
-                if (!wait_dep(cblock, need)) { fail(1); break; }
+                if (!wait_dep(cblock, need, dep_seen)) { fail(1); break; }
                 const float4 *rbase = reinterpret_cast<const float4 *>(a.records) + (size_t)rec0 * (KP4 + 1);
                 float Dp = 0.f, wt = 0.f;
                 int mp = 0;
@@ -654,7 +665,14 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
                 const uint32_t col = (uint32_t)__shfl_sync(FULL, dc, 14);
                 if (g == 0) {
                     const float2 sc = __ldcg(Sc + col);
-                    apply(col, sc.x, sc.y, Dp, __int_as_float(mp), ut, wt);
+                    const float inv = rcp_fast(1.0f + sc.x);
+                    const int mj = __float_as_int(sc.y);
+#pragma unroll
+                    for (int v = 0; v < NV; ++v) {
+                        ut[v].x *= inv; ut[v].y *= inv; ut[v].z *= inv; ut[v].w *= inv;
+                    }
+                    flush(col, ut, wt * ex2_fast((float)mj * a.kappa_w));
+                    if (l == 0) Sc[col] = make_float2(fmaf(sc.x, Dp, sc.x + Dp), __int_as_float(mj + mp));
                 }
                 if (lane == 0) a.run_count[run_id] = 0;
             }
@@ -675,9 +693,7 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
         if ((unsigned)tk1 >= nch) { pending_next = false; break; }
         dc = dn;
         tk0 = tk1;
-        tk1 = __shfl_sync(FULL, tk2_raw, 0);
-        dn = load_desc(tk1);
-        tk2_raw = ((unsigned)tk1 < nch) ? take_ticket() : kTicketStop;
+        dep_seen = dep_seen_next;
         buf ^= 1;
     }
     // leaving early: nothing may still be on its way into this warp's shared memory
