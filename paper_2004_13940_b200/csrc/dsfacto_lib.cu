@@ -64,8 +64,8 @@ struct dsfacto {
     int debug_extra_need = 0;   // tests: added to the `need` of the first chunk, so that its wait runs out
     bool failed = false;        // an SGD launch gave up; the parameters are unusable until they are set again
     float *d_records = nullptr, *d_Tb = nullptr, *d_Tw = nullptr;
-    float2 *d_S = nullptr, *d_TS = nullptr;  // scale records of the scaled column state (zero outside the SGD phase)
-    int *d_tile_count = nullptr, *d_run_count = nullptr;
+    float4 *d_S = nullptr, *d_TS = nullptr;  // scale records of the scaled column state (zero outside the SGD phase)
+    int *d_run_count = nullptr;
     int refresh_grid = 0, norm_grid = 0;
 
     double loss_sum = 0, g_sum = 0, w2 = 0, v2 = 0, objective = 0;
@@ -232,7 +232,7 @@ void unpack_tiles(const dsfacto *h, const std::vector<int64_t> &canon_ptr, const
 void free_data(dsfacto *h) {
     dev_free(h->d_A); dev_free(h->d_G); dev_free(h->d_y); dev_free(h->d_val); dev_free(h->d_xw);
     dev_free(h->d_indptr); dev_free(h->d_tile_ptr); dev_free(h->d_idx); dev_free(h->d_ent);
-    dev_free(h->d_partials); dev_free(h->d_desc); dev_free(h->d_records); dev_free(h->d_tile_count); dev_free(h->d_run_count);
+    dev_free(h->d_partials); dev_free(h->d_desc); dev_free(h->d_records); dev_free(h->d_run_count);
     dev_free(h->d_sync);
     h->launch_ptr.clear();
     h->loaded = false;
@@ -416,7 +416,7 @@ int finish_sgd_plan(dsfacto *h, SgdPlanBuild &pb) {
     for (int64_t t = 0; t < nt; ++t) total += pb.refs[(size_t)t].count;
     if (total >= (int64_t)kTicketStop / 2) return DSFACTO_ERR_INVALID_ARG;
     HostBuf<ChunkDesc> all;
-    std::vector<int> seen;   // non-empty tiles met so far per column block
+    std::vector<int> seen;   // chunks met so far per column block
     if (!all.alloc((size_t)total)) return DSFACTO_ERR_OOM;
     try {
         h->launch_ptr.assign((size_t)p + 1, 0);
@@ -444,7 +444,7 @@ int finish_sgd_plan(dsfacto *h, SgdPlanBuild &pb) {
             }
             all[(size_t)pos++] = d;
         }
-        if (ref.count > 0) seen[(size_t)c] += 1;
+        seen[(size_t)c] += ref.count;
         if ((slot + 1) % p == 0) h->launch_ptr[(size_t)((slot + 1) / p)] = pos;
     }
     if (recs >= ((int64_t)1 << 31)) return DSFACTO_ERR_INVALID_ARG;
@@ -455,10 +455,8 @@ int finish_sgd_plan(dsfacto *h, SgdPlanBuild &pb) {
     int rc;
     if ((rc = dev_alloc(h, &h->d_desc, (size_t)total)) ||
         (rc = dev_alloc(h, &h->d_records, (size_t)recs * slice_record_floats(h->Kp))) ||
-        (rc = dev_alloc(h, &h->d_run_count, (size_t)runs)) || (rc = dev_alloc(h, &h->d_tile_count, (size_t)nt)) ||
-        (rc = dev_alloc(h, &h->d_sync, sync_words((int)p))))
+        (rc = dev_alloc(h, &h->d_run_count, (size_t)runs)) || (rc = dev_alloc(h, &h->d_sync, sync_words((int)p))))
         return rc;
-    CU_TRY(h, cudaMemsetAsync(h->d_tile_count, 0, sizeof(int) * (size_t)nt, h->stream));
     CU_TRY(h, cudaMemsetAsync(h->d_run_count, 0, sizeof(int) * (size_t)std::max<int64_t>(runs, 1), h->stream));
     CU_TRY(h, cudaMemsetAsync(h->d_sync, 0, sizeof(int) * sync_words((int)p), h->stream));
     if (total > 0)
@@ -473,7 +471,7 @@ void run_sgd_phase(dsfacto *h, int64_t L0, int64_t L1) {
     SgdArgs a{};
     a.ent = h->d_ent; a.xw = h->d_xw; a.A = h->d_A; a.G = h->d_G; a.w = h->d_w; a.V = h->d_V;
     a.S = h->d_S; a.Tb = h->d_Tb; a.Tw = h->d_Tw; a.TS = h->d_TS; a.records = h->d_records;
-    a.tile_count = h->d_tile_count; a.run_count = h->d_run_count;
+    a.run_count = h->d_run_count;
     a.n = h->n; a.d = h->d; a.jbits = h->jbits; a.chunk_len = h->chunk_len; a.spin_limit = h->spin_limit;
     a.h = h->h; a.lambda_v = h->lambda_v;
     const double ew = (double)h->h * (double)h->lambda_w;
@@ -1006,14 +1004,14 @@ int dsfacto_create(dsfacto_t **out, int64_t n, int32_t d, int32_t K, int32_t p, 
     h->norm_grid = h->sm_count * 8;
     if (const char *env = std::getenv("DSFACTO_SWEEP")) h->sweep = (std::strcmp(env, "round") == 0) ? 0 : 1;
     if ((rc = dev_alloc(h, &h->d_S, (size_t)d))) return fail(rc);
-    if (cudaMemset(h->d_S, 0, sizeof(float2) * (size_t)d) != cudaSuccess) return fail(DSFACTO_ERR_CUDA);
+    if (cudaMemset(h->d_S, 0, sizeof(float4) * (size_t)d) != cudaSuccess) return fail(DSFACTO_ERR_CUDA);
     if (h->sweep == 1) {
         if ((rc = dev_alloc(h, &h->d_Tb, (size_t)d * h->Kp)) || (rc = dev_alloc(h, &h->d_Tw, (size_t)d)) ||
             (rc = dev_alloc(h, &h->d_TS, (size_t)d)))
             return fail(rc);
         if (cudaMemset(h->d_Tb, 0, sizeof(float) * (size_t)d * h->Kp) != cudaSuccess ||
             cudaMemset(h->d_Tw, 0, sizeof(float) * (size_t)d) != cudaSuccess ||
-            cudaMemset(h->d_TS, 0, sizeof(float2) * (size_t)d) != cudaSuccess)
+            cudaMemset(h->d_TS, 0, sizeof(float4) * (size_t)d) != cudaSuccess)
             return fail(DSFACTO_ERR_CUDA);
     }
     *out = h;
@@ -1142,12 +1140,11 @@ static int sgd_gave_up(dsfacto *h, const int code[3]) {
     else std::snprintf(buf, sizeof buf, "stratum SGD: debug check %d failed (value %d)", code[1], code[2]);
     h->err = buf;
     const size_t d = (size_t)h->d;
-    cudaMemsetAsync(h->d_tile_count, 0, sizeof(int) * (size_t)h->p * h->p, h->stream);
     cudaMemsetAsync(h->d_run_count, 0, sizeof(int) * (size_t)std::max<int64_t>(h->long_runs, 1), h->stream);
     cudaMemsetAsync(h->d_sync, 0, sizeof(int) * sync_words(h->p), h->stream);
-    cudaMemsetAsync(h->d_S, 0, sizeof(float2) * d, h->stream);
+    cudaMemsetAsync(h->d_S, 0, sizeof(float4) * d, h->stream);
     if (h->d_TS) {
-        cudaMemsetAsync(h->d_TS, 0, sizeof(float2) * d, h->stream);
+        cudaMemsetAsync(h->d_TS, 0, sizeof(float4) * d, h->stream);
         cudaMemsetAsync(h->d_Tw, 0, sizeof(float) * d, h->stream);
         cudaMemsetAsync(h->d_Tb, 0, sizeof(float) * d * h->Kp, h->stream);
     }

@@ -38,7 +38,7 @@ constexpr int kTicketStop = 0x40000000;           // ticket counter value that m
 constexpr int kSyncStride = 32;                   // ints between two words
 constexpr int kSyncTicket = 0;                    // next chunk to hand out
 constexpr int kSyncError = kSyncStride;           // set when a wait ran out (1: earlier tile, 2: bulk copy, 3: debug check)
-__host__ __device__ constexpr size_t sync_done(int c) { return (size_t)(2 + c) * kSyncStride; }  // finished tiles of column block c
+__host__ __device__ constexpr size_t sync_done(int c) { return (size_t)(2 + c) * kSyncStride; }  // finished chunks of column block c
 __host__ __device__ constexpr size_t sync_words(int p) { return (size_t)(2 + p) * kSyncStride; }
 
 // One unit of work of the sweep: a range of consecutive entries of one tile (entries of a tile are
@@ -51,8 +51,8 @@ struct ChunkDesc {
     int32_t row0;      // first row of the tile's row block
     int32_t col0;      // first column of the tile's column block
     int32_t cblock;    // column block (index of its progress counter)
-    int32_t need;      // earlier non-empty tiles of that column block, in sweep order
-    int32_t tile;      // tile slot (index of its chunk counter)
+    int32_t need;      // chunks of the earlier tiles of that column block, in sweep order
+    int32_t tile;      // tile slot
     int32_t nchunks;   // chunks of the tile
     int32_t run_id;    // slice: index of the long run (its join counter)
     int32_t slice;     // slice: number of this slice inside the run
@@ -69,12 +69,13 @@ template <int LG, int NV>
 struct SgdCfg {
     static constexpr int GW = 32 / LG;               // lane groups per warp = rows worked on side by side
     static constexpr int KP4 = LG * NV;              // float4s per factor row
-    // rows of A gathered per stage: at most 4 KB a stage
+    // rows of A gathered per stage: a whole pass for rows up to 128 bytes, at most 4 KB for wider rows
     static constexpr int RST = KP4 <= 8 ? 32 : (KP4 <= 16 ? 16 : (KP4 <= 32 ? 8 : 4));
     static constexpr int SP = 32 / RST;              // stages per 32-entry pass
-    static constexpr int NBUF = KP4 <= 8 ? 2 : 3;    // stages in the ring
+    static constexpr int NBUF = 2;                   // stages in the ring (three were no faster on any workload)
     static constexpr int PD = NBUF - 1;              // stages requested ahead
     static constexpr int ROW4 = NBUF * RST * KP4;    // float4s of the row ring
+    static constexpr int DG = SP == 1 ? PD : 1;      // passes ahead at which G_i and the scale records are requested
 };
 // entries the staging buffer of one chunk holds: the copy starts and ends on multiples of 4 entries
 __host__ __device__ constexpr int sgd_ecap(int chunk_len) { return (chunk_len + 8 + 3) & ~3; }
@@ -89,6 +90,10 @@ __host__ __device__ constexpr int slice_record_floats(int Kp) { return 4 + Kp; }
 __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src) {
     const unsigned s = (unsigned)__cvta_generic_to_shared(smem_dst);
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async4(void *smem_dst, const void *gmem_src) {
+    const unsigned s = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"(s), "l"(gmem_src) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N>
@@ -154,14 +159,13 @@ struct SgdArgs {
     const float *G;            // n
     float *w;                  // d        uw_j
     float *V;                  // d * Kp   u_j
-    float2 *S;                 // d        {sigma_j, m_j (int bits)}
+    float4 *S;                 // d        {sigma_j, m_j (int bits), -, -} (16 bytes: fetched with one cp.async.cg)
     float *Tw;                 // d        the same three for the tail composite T_j (row-block sweep)
     float *Tb;                 // d * Kp
-    float2 *TS;                // d
+    float4 *TS;                // d
     float *records;            // slice_record_floats(Kp) floats per slice of a long run
-    int *tile_count;           // p*p, all zero between launches
     int *run_count;            // one per long run, all zero between launches
-    int *sync;                 // sync_words(p) ints: ticket counter (zero at launch), error word, finished tiles
+    int *sync;                 // sync_words(p) ints: ticket counter (zero at launch), error word, finished chunks
                                // per column block (zero at the first launch of a sweep, kept between the
                                // launches of one sweep)
     int64_t n, d;              // rows and columns of the data set (checks of the debug build)
@@ -228,7 +232,7 @@ struct SgdArgs {
 template <int LG, int NV, bool WIDE>
 __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a) {
     typedef SgdCfg<LG, NV> C;
-    constexpr int GW = C::GW, KP4 = C::KP4, RST = C::RST, SP = C::SP, NBUF = C::NBUF, PD = C::PD;
+    constexpr int GW = C::GW, KP4 = C::KP4, RST = C::RST, SP = C::SP, NBUF = C::NBUF, PD = C::PD, DG = C::DG;
     constexpr unsigned FULL = 0xFFFFFFFFu;
 
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -236,10 +240,10 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
     const int g = lane / LG, l = lane % LG;
     const int ecap = sgd_ecap(a.chunk_len);
     unsigned char *wbase = smem_raw + (size_t)warp * sgd_warp_smem<LG, NV>(WIDE, a.chunk_len);
-    float4 *rowb = reinterpret_cast<float4 *>(wbase);               // row ring
+    float4 *rowb = reinterpret_cast<float4 *>(wbase);               // ring of row stages
     float2 *pc = reinterpret_cast<float2 *>(rowb + C::ROW4);        // per entry of the pass: {c, cw}
     uint32_t *pcol = reinterpret_cast<uint32_t *>(pc + 32);         // per entry of the pass: local column
-    int *segpos = reinterpret_cast<int *>(pcol + 32);               // lane of the k-th run start of the pass (40 ints)
+    int *segpos = reinterpret_cast<int *>(pcol + 32);               // lane of the k-th run start of the pass (33 used)
     uint64_t *mbar = reinterpret_cast<uint64_t *>(segpos + 40);     // one per entry buffer
     uint2 *ebuf = reinterpret_cast<uint2 *>(mbar + 2);              // 2 x ecap entry records
     float *xbuf = reinterpret_cast<float *>(ebuf + 2 * (size_t)ecap);  // wide layout: 2 x ecap values
@@ -288,8 +292,9 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
             atomicMax(a.sync + kSyncTicket, kTicketStop);
         }
     };
-    // Wait until `need` earlier tiles of column block cblock are done.  `seen` is an earlier reading of the
-    // counter (lane 0; it only grows), so that a tile that was ready long ago costs no round trip to L2.
+    // Wait until the `need` chunks of the earlier tiles of column block cblock are done.  `seen` is an earlier
+    // reading of the counter (lane 0; it only grows), so that a tile that was ready long ago costs no round
+    // trip to L2.
     auto wait_dep = [&](int cblock, int need, int seen) -> bool {
         int ok = 1;
         if (lane == 0 && seen < need) {
@@ -308,7 +313,7 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
     int tk0 = __shfl_sync(FULL, take_ticket(), 0);
     if ((unsigned)tk0 >= nch) return;
     int dc = load_desc(tk0);
-    int tk1 = kTicketStop, dn = 0, tk1_raw = 0, dep_seen_next = 0;
+    int tk1 = kTicketStop, dn = 0, tk1_raw = 0, dep_seen_next = 0, cb1 = 0;
     int buf = 0;
     unsigned parity_bits = 0;   // bit b: parity the next wait on buffer b expects
     bool pending_next = false;  // a bulk copy into the other buffer is under way
@@ -327,8 +332,6 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
         const int col0 = __shfl_sync(FULL, dc, 5);
         const int cblock = __shfl_sync(FULL, dc, 6);
         const int need = __shfl_sync(FULL, dc, 7);
-        const int tile = __shfl_sync(FULL, dc, 8);
-        const int tile_chunks = __shfl_sync(FULL, dc, 9);
         const bool is_slice = (flags & kChunkSlice) != 0;
         const bool tail_mode = (flags & kChunkTail) != 0;
 
@@ -346,7 +349,7 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
         const float *Gr = a.G + row0;
         float4 *U4 = reinterpret_cast<float4 *>(tail_mode ? a.Tb : a.V) + (size_t)col0 * KP4;
         float *uw = (tail_mode ? a.Tw : a.w) + col0;
-        float2 *Sc = (tail_mode ? a.TS : a.S) + col0;
+        float4 *Sc = (tail_mode ? a.TS : a.S) + col0;
         DSF_CHECK(len >= 1 && len <= a.chunk_len, 10, len);
 
         // adds a finished run's sums to its column (the lanes of one group; sums already carry the column's scale)
@@ -379,32 +382,39 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
         // ---- the chunk ----
         const int npass = (len + 31) >> 5;
         const int nstage = (len + RST - 1) / RST;
-        // scalars of a pass, requested one pass ahead: row, column, x, G_i, run start, scale record
-        uint32_t il_c = 0, il_n = 0, jl_c = kNoCol, jl_n = kNoCol;
-        float x_c = 0.f, x_n = 0.f, g_c = 0.f, g_n = 0.f;
-        float2 sc_c = make_float2(0.f, 0.f), sc_n = make_float2(0.f, 0.f);
-        bool bnd_c = false, bnd_n = false;
         const uint32_t col_init = is_slice ? (uint32_t)__shfl_sync(FULL, dc, 14) : kNoCol;
-        auto fetch_pass = [&](int k, uint32_t prev_last) {   // -> *_n
+        // What a pass needs from global memory is requested ahead of time.  Scalars (G_i of every entry, the scale
+        // record of every column whose run starts in the pass) come DG passes ahead into a queue of registers;
+        // the rows a_i come PD stages ahead with cp.async into the row ring, one commit group per stage.
+        float gq[DG], xq[DG];
+        uint32_t jq[DG];
+        float4 scq[DG];
+        uint32_t mq[DG];                     // run starts of the pass as a lane mask
+        uint32_t il_c = 0, il_n = 0;         // local rows (one per lane) of the pass at work and of the next one
+        auto fetch_pass = [&](int k, float &g_out, float4 &sc_out, uint32_t &mask_out, uint32_t &jl, float &x_out) -> uint32_t {
             const int at = 32 * k + lane;
-            jl_n = kNoCol; x_n = 0.f; g_n = 0.f; il_n = 0;
+            bool bnd = false;
+            uint32_t il = 0;
+            g_out = 0.f; x_out = 0.f; jl = kNoCol;
             if (at < len) {
                 const uint2 rec = eb[at];
-                if (WIDE) { il_n = rec.x; jl_n = rec.y; x_n = xb[at]; }
-                else { il_n = rec.x >> a.jbits; jl_n = rec.x & jmask; x_n = __uint_as_float(rec.y); }
-                DSF_CHECK((int64_t)row0 + il_n < a.n, 13, il_n);
-                g_n = __ldg(Gr + il_n);
+                uint32_t prevj = col_init;
+                if (WIDE) { il = rec.x; jl = rec.y; x_out = xb[at]; }
+                else { il = rec.x >> a.jbits; jl = rec.x & jmask; x_out = __uint_as_float(rec.y); }
+                if (at > 0) prevj = WIDE ? eb[at - 1].y : (eb[at - 1].x & jmask);
+                bnd = jl != prevj;
+                DSF_CHECK((int64_t)row0 + il < a.n, 13, il);
+                g_out = __ldg(Gr + il);
+                if (bnd) sc_out = __ldcg(Sc + jl);
             }
-            uint32_t prevj = __shfl_up_sync(FULL, jl_n, 1);
-            if (lane == 0) prevj = prev_last;
-            bnd_n = (at < len) && (jl_n != prevj);
-            if (bnd_n) sc_n = __ldcg(Sc + jl_n);
+            mask_out = __ballot_sync(FULL, bnd);
+            return il;
         };
-        // rows of stage sp of a pass whose local rows are `il` (one per lane) into ring slot `ring`: lane group
-        // q of the warp fetches the row of entry sp*RST + it*GW + q, 16 bytes per lane (rows past the end of
-        // the chunk repeat row 0 of the block)
-        auto issue_rows = [&](uint32_t il, int sp, int ring) {
-            float4 *dst = rowb + ring * (RST * KP4) + g * KP4 + l;
+        // rows of stage sp of a pass whose local rows are `il`: lane group q fetches the row of entry
+        // sp*RST + it*GW + q, 16 bytes per lane (rows past the end of the chunk repeat row 0 of the block)
+        int ring_issue = 0, ring_use = 0;     // row ring: slot of the next stage to request / to work on
+        auto issue_rows = [&](uint32_t il, int sp) {
+            float4 *dst = rowb + ring_issue * (RST * KP4) + g * KP4 + l;
 #pragma unroll
             for (int it = 0; it < RST / GW; ++it) {
                 const uint32_t ir = __shfl_sync(FULL, il, sp * RST + it * GW + g);
@@ -412,18 +422,25 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
                 for (int v = 0; v < NV; ++v)
                     cp_async16(dst + it * GW * KP4 + v * LG, A4r + (size_t)ir * KP4 + v * LG + l);
             }
-        };
-        fetch_pass(0, col_init);
-        il_c = il_n;
-        int ring_issue = 0, ring_use = 0;   // ring slots of the next stage to request / to work on
-        // stage s of the chunk = stage s % SP of pass s / SP; the first PD stages are requested here
-#pragma unroll
-        for (int s = 0; s < PD; ++s) {
-            if (s < SP) {   // (PD <= SP except for one-stage passes, where PD = 1 = SP)
-                if (s < nstage) issue_rows(il_n, s, ring_issue);
-            }
-            cp_async_commit();
             ring_issue = (ring_issue + 1 == NBUF) ? 0 : ring_issue + 1;
+        };
+#pragma unroll
+        for (int q = 0; q < DG; ++q) {
+            gq[q] = 0.f; xq[q] = 0.f; jq[q] = kNoCol; mq[q] = 0u; scq[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+            uint32_t il = 0;
+            if (q < npass) il = fetch_pass(q, gq[q], scq[q], mq[q], jq[q], xq[q]);
+            if (q == 0) il_n = il;
+            if (SP == 1) {   // a stage is a pass: its rows are requested together with its scalars
+                if (q < nstage) issue_rows(il, 0);
+                cp_async_commit();
+            }
+        }
+        if (SP > 1) {
+#pragma unroll
+            for (int s = 0; s < PD; ++s) {   // PD <= SP: the first PD stages belong to the first pass
+                if (s < nstage) issue_rows(il_n, s);
+                cp_async_commit();
+            }
         }
 
         float4 acc[NV];   // this lane group's share of the run that is open
@@ -437,15 +454,25 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
 
         for (int k = 0; k < npass; ++k) {
             const int cnt = (len - 32 * k) < 32 ? (len - 32 * k) : 32;
-            il_c = il_n; jl_c = jl_n; x_c = x_n; g_c = g_n; sc_c = sc_n; bnd_c = bnd_n;
-            if (k + 1 < npass) fetch_pass(k + 1, __shfl_sync(FULL, jl_c, 31));
+            // this pass's scalars leave the queue; those of pass k + DG are requested
+            const float g_c = gq[0], x_c = xq[0];
+            const uint32_t jl_c = jq[0];
+            const float4 sc_q0 = scq[0];
+            const uint32_t mask = mq[0];
+#pragma unroll
+            for (int q = 0; q + 1 < DG; ++q) { gq[q] = gq[q + 1]; xq[q] = xq[q + 1]; jq[q] = jq[q + 1]; scq[q] = scq[q + 1]; mq[q] = mq[q + 1]; }
+            il_c = il_n;
+            uint32_t il_f = 0;
+            if (k + DG < npass) il_f = fetch_pass(k + DG, gq[DG - 1], scq[DG - 1], mq[DG - 1], jq[DG - 1], xq[DG - 1]);
+            if (SP > 1) il_n = il_f;
 
             // ---- scalar stage ----
-            const uint32_t mask = __ballot_sync(FULL, bnd_c);
             float D;
             int m;
             {
+                const bool bnd_c = (mask >> lane) & 1u;
                 float e = 0.f, b = 0.f;
+                const float4 sc_c = sc_q0;
                 if (lane < cnt) {
                     const float gx = g_c * x_c;
                     e = a.h * (a.lambda_v - gx * x_c);
@@ -467,11 +494,13 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
                 const float c = b * rcp_fast(1.0f + D);
                 const float cw = b * ex2_fast((float)m * a.kappa_w);
                 pc[lane] = make_float2(c, cw);
-                pcol[lane] = jl_c;
-                if (bnd_c) segpos[__popc(mask & ((1u << lane) - 1u))] = lane;
-                if (lane == 0) segpos[__popc(mask)] = cnt;
-                // a run that ends inside the pass leaves its column's new scale record right here
-                if (lane + 1 < cnt && ((mask >> (lane + 1)) & 1u)) Sc[jl_c] = make_float2(D, __int_as_float(m));
+                if (mask != 0u) {   // only passes with a run start need the rest
+                    pcol[lane] = jl_c;
+                    if (bnd_c) segpos[__popc(mask & ((1u << lane) - 1u))] = lane;
+                    if (lane == 0) segpos[__popc(mask)] = cnt;
+                    // a run that ends inside the pass leaves its column's new scale record right here
+                    if (lane + 1 < cnt && ((mask >> (lane + 1)) & 1u)) Sc[jl_c] = make_float4(D, __int_as_float(m), 0.f, 0.f);
+                }
             }
             __syncwarp();
 
@@ -481,11 +510,11 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
                 const int s = k * SP + sp;
                 if (s >= nstage) break;
                 if (s + PD < nstage) {
-                    if (sp + PD < SP) issue_rows(il_c, sp + PD, ring_issue);
-                    else issue_rows(il_n, sp + PD - SP, ring_issue);
+                    if (SP == 1) issue_rows(il_f, 0);
+                    else if (sp + PD < SP) issue_rows(il_c, sp + PD);
+                    else issue_rows(il_n, sp + PD - SP);
                 }
                 cp_async_commit();
-                ring_issue = (ring_issue + 1 == NBUF) ? 0 : ring_issue + 1;
                 cp_async_wait<PD>();
                 __syncwarp();
                 const float4 *rb = rowb + ring_use * (RST * KP4);
@@ -533,33 +562,61 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
                         if (g == 0) {
                             flush(open_col, acc, accw);
                             // (a run that ends inside the pass has left its scale record in the scalar stage)
-                            if (F == 0 && l == 0) Sc[open_col] = make_float2(D_open, __int_as_float(m_open));
+                            if (F == 0 && l == 0) Sc[open_col] = make_float4(D_open, __int_as_float(m_open), 0.f, 0.f);
                         }
                     }
 #pragma unroll
                     for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
                     accw = 0.f;
-                    // 2. runs that start and end inside the stage: one lane group each
+                    // 2. runs that start and end inside the stage
                     const int i0 = __popc(mask & ((1u << F) - 1u));
                     const int nmid = __popc(sub) - 1;
-                    for (int i = g; i < nmid; i += GW) {
-                        const int s0 = segpos[i0 + i], s1 = segpos[i0 + i + 1];
-                        DSF_CHECK(s0 >= e0 && s1 > s0 && s1 <= e1, 11, s0 * 64 + s1);
-                        float4 tmp[NV];
-                        float tmpw = 0.f;
+                    if (KP4 <= 8 && nmid >= GW) {
+                        // many short runs (rows of up to 128 bytes): one lane each, the lane holds the whole row sum
+                        constexpr int Q = KP4 <= 8 ? KP4 : 1;
+                        if (lane < nmid) {
+                            const int s0 = segpos[i0 + lane], s1 = segpos[i0 + lane + 1];
+                            DSF_CHECK(s0 >= e0 && s1 > s0 && s1 <= e1, 11, s0 * 64 + s1);
+                            float4 t[Q];
+                            float tw = 0.f;
 #pragma unroll
-                        for (int v = 0; v < NV; ++v) tmp[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        for (int u = s0; u < s1; ++u) {
-                            const float2 cf = pc[u];
+                            for (int q = 0; q < Q; ++q) t[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                            for (int u = s0; u < s1; ++u) {
+                                const float2 cf = pc[u];
 #pragma unroll
-                            for (int v = 0; v < NV; ++v) {
-                                const float4 r = rb[(u - e0) * KP4 + v * LG + l];
-                                tmp[v].x = fmaf(cf.x, r.x, tmp[v].x); tmp[v].y = fmaf(cf.x, r.y, tmp[v].y);
-                                tmp[v].z = fmaf(cf.x, r.z, tmp[v].z); tmp[v].w = fmaf(cf.x, r.w, tmp[v].w);
+                                for (int q = 0; q < Q; ++q) {
+                                    const float4 r = rb[(u - e0) * KP4 + q];
+                                    t[q].x = fmaf(cf.x, r.x, t[q].x); t[q].y = fmaf(cf.x, r.y, t[q].y);
+                                    t[q].z = fmaf(cf.x, r.z, t[q].z); t[q].w = fmaf(cf.x, r.w, t[q].w);
+                                }
+                                tw += cf.y;
                             }
-                            tmpw += cf.y;
+                            const uint32_t col = pcol[s0];
+                            DSF_CHECK((int64_t)col0 + col < a.d, 12, col);
+#pragma unroll
+                            for (int q = 0; q < Q; ++q) red_add4(U4 + (size_t)col * KP4 + q, t[q].x, t[q].y, t[q].z, t[q].w);
+                            red_add1(uw + col, tw);
                         }
-                        flush(pcol[s0], tmp, tmpw);
+                    } else {
+                    for (int i = g; i < nmid; i += GW) {
+                            const int s0 = segpos[i0 + i], s1 = segpos[i0 + i + 1];
+                            DSF_CHECK(s0 >= e0 && s1 > s0 && s1 <= e1, 11, s0 * 64 + s1);
+                            float4 tmp[NV];
+                            float tmpw = 0.f;
+#pragma unroll
+                            for (int v = 0; v < NV; ++v) tmp[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+                            for (int u = s0; u < s1; ++u) {
+                                const float2 cf = pc[u];
+#pragma unroll
+                                for (int v = 0; v < NV; ++v) {
+                                    const float4 r = rb[(u - e0) * KP4 + v * LG + l];
+                                    tmp[v].x = fmaf(cf.x, r.x, tmp[v].x); tmp[v].y = fmaf(cf.x, r.y, tmp[v].y);
+                                    tmp[v].z = fmaf(cf.x, r.z, tmp[v].z); tmp[v].w = fmaf(cf.x, r.w, tmp[v].w);
+                                }
+                                tmpw += cf.y;
+                            }
+                            flush(pcol[s0], tmp, tmpw);
+                        }
                     }
                     __syncwarp();
                     // 3. the run that is open at the end of the stage
@@ -573,29 +630,30 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
             D_open = __shfl_sync(FULL, D, cnt - 1);
             m_open = __shfl_sync(FULL, m, cnt - 1);
 
-            // the next chunk: its descriptor after the first pass, its entries (and a first look at the progress
-            // of its column block) a little later, so that neither request is waited for
+            // the next chunk: its descriptor after the first pass, its entries a little later, so that neither
+            // request is waited for
             if (k == 0) {
                 tk1 = __shfl_sync(FULL, tk1_raw, 0);
                 dn = load_desc(tk1);
             }
             if (k == (npass > 2 ? 2 : npass - 1) && (unsigned)tk1 < nch) {
                 const int64_t off1 = ((int64_t)(uint32_t)__shfl_sync(FULL, dn, 0)) | ((int64_t)__shfl_sync(FULL, dn, 1) << 32);
-                const int len1 = __shfl_sync(FULL, dn, 2), cb1 = __shfl_sync(FULL, dn, 6);
+                const int len1 = __shfl_sync(FULL, dn, 2);
+                cb1 = __shfl_sync(FULL, dn, 6);
                 __syncwarp();
                 issue_entries(off1, len1, buf ^ 1);   // the other buffer's last reader was the chunk before this one
                 pending_next = true;
-                if (lane == 0) dep_seen_next = ld_acquire(a.sync + sync_done(cb1));
             }
         }
         cp_async_wait<0>();
 
         // ---- end of the chunk ----
         reduce_groups(acc, accw);
+        int done_add = 1;   // what this chunk adds to the progress counter of its column block
         if (!is_slice) {
             if (open_valid && g == 0) {
                 flush(open_col, acc, accw);
-                if (l == 0) Sc[open_col] = make_float2(D_open, __int_as_float(m_open));
+                if (l == 0) Sc[open_col] = make_float4(D_open, __int_as_float(m_open), 0.f, 0.f);
             }
         } else {
             const int run_id = __shfl_sync(FULL, dc, 10), slice = __shfl_sync(FULL, dc, 11);
@@ -608,6 +666,9 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
             }
             __threadfence();
             __syncwarp();
+            // Slices do not wait for earlier tiles, so they must not count as progress before their run has been
+            // applied: the slice that joins the run reports all of them.
+            done_add = 0;
             int last = 0;
             if (lane == 0) last = (atomicAdd(a.run_count + run_id, 1) == nslices - 1) ? 1 : 0;
             last = __shfl_sync(FULL, last, 0);
@@ -664,7 +725,7 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
                 for (int o = 16; o > 0; o >>= 1) wt += __shfl_xor_sync(FULL, wt, o);
                 const uint32_t col = (uint32_t)__shfl_sync(FULL, dc, 14);
                 if (g == 0) {
-                    const float2 sc = __ldcg(Sc + col);
+                    const float4 sc = __ldcg(Sc + col);
                     const float inv = rcp_fast(1.0f + sc.x);
                     const int mj = __float_as_int(sc.y);
 #pragma unroll
@@ -672,21 +733,20 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
                         ut[v].x *= inv; ut[v].y *= inv; ut[v].z *= inv; ut[v].w *= inv;
                     }
                     flush(col, ut, wt * ex2_fast((float)mj * a.kappa_w));
-                    if (l == 0) Sc[col] = make_float2(fmaf(sc.x, Dp, sc.x + Dp), __int_as_float(mj + mp));
+                    if (l == 0) Sc[col] = make_float4(fmaf(sc.x, Dp, sc.x + Dp), __int_as_float(mj + mp), 0.f, 0.f);
                 }
                 if (lane == 0) a.run_count[run_id] = 0;
+                done_add = nslices;
             }
         }
-        // this chunk is done; the chunk that finishes a tile reports the tile
-        __threadfence();
-        __syncwarp();
-        if (lane == 0) {
-            bool fin = true;
-            if (tile_chunks > 1) {
-                fin = atomicAdd(a.tile_count + tile, 1) == tile_chunks - 1;
-                if (fin) { a.tile_count[tile] = 0; __threadfence(); }
-            }
-            if (fin) atomicAdd(a.sync + sync_done(cblock), 1);
+        // This chunk is done: what it wrote becomes visible, then the progress counter of its column block goes
+        // up by one (nobody waits for the add).  The first look at the counter of the next chunk's column block
+        // is taken just before, so that its round trip overlaps the fence.
+        if (lane == 0 && (unsigned)tk1 < nch) dep_seen_next = ld_acquire(a.sync + sync_done(cb1));
+        if (done_add > 0) {
+            __threadfence();
+            __syncwarp();
+            if (lane == 0) atomicAdd(a.sync + sync_done(cblock), done_add);
         }
 
         // ---- next chunk ----
@@ -707,8 +767,8 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
 // where T_j = (D_T, m_T, ub_j, ubw_j) is the tail composite (identity unless the launch order was the
 // row-block sweep), and reset of the scale records and of T_j.  Two kernels because the first reads
 // the scale records that the second clears.  log1m_ew = log(1 - ew) in double.
-__global__ void __launch_bounds__(kThreads) sgd_finalize_v_kernel(float *V, float *Tb, const float2 *S,
-                                                                  const float2 *TS, int64_t d, int kp4) {
+__global__ void __launch_bounds__(kThreads) sgd_finalize_v_kernel(float *V, float *Tb, const float4 *S,
+                                                                  const float4 *TS, int64_t d, int kp4) {
     const int64_t total = d * kp4;
     float4 *V4 = reinterpret_cast<float4 *>(V);
     float4 *Tb4 = reinterpret_cast<float4 *>(Tb);
@@ -727,19 +787,19 @@ __global__ void __launch_bounds__(kThreads) sgd_finalize_v_kernel(float *V, floa
         V4[i] = y;
     }
 }
-__global__ void __launch_bounds__(kThreads) sgd_finalize_w_kernel(float *w, float *Tw, float2 *S, float2 *TS, int64_t d,
+__global__ void __launch_bounds__(kThreads) sgd_finalize_w_kernel(float *w, float *Tw, float4 *S, float4 *TS, int64_t d,
                                                                   double log1m_ew) {
     for (int64_t j = (int64_t)blockIdx.x * kThreads + threadIdx.x; j < d; j += (int64_t)gridDim.x * kThreads) {
         float wj = w[j];
         const int mj = __float_as_int(S[j].y);
         if (mj != 0) wj = fmaf((float)expm1((double)mj * log1m_ew), wj, wj);
-        S[j] = make_float2(0.f, 0.f);
+        S[j] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (Tw != nullptr) {
             wj += Tw[j];
             const int mt = __float_as_int(TS[j].y);
             if (mt != 0) wj = fmaf((float)expm1((double)mt * log1m_ew), wj, wj);
             Tw[j] = 0.f;
-            TS[j] = make_float2(0.f, 0.f);
+            TS[j] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
         w[j] = wj;
     }
