@@ -27,7 +27,7 @@
 
 namespace dsf {
 
-constexpr int kSgdWarps = 2;                      // warps per CTA; every warp works on its own chunks
+constexpr int kSgdWarps = 1;                      // warps per CTA; every warp works on its own chunks
 constexpr int kSgdThreads = 32 * kSgdWarps;
 constexpr int kChunkMax = 512;                    // most entries a chunk may hold
 constexpr int kSgdSpinLimit = 1 << 22;            // polls (about 100 ns each) before a dependency wait gives up
@@ -568,55 +568,27 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
 #pragma unroll
                     for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
                     accw = 0.f;
-                    // 2. runs that start and end inside the stage
+                    // 2. runs that start and end inside the stage: one lane group each
                     const int i0 = __popc(mask & ((1u << F) - 1u));
                     const int nmid = __popc(sub) - 1;
-                    if (KP4 <= 8 && nmid >= GW) {
-                        // many short runs (rows of up to 128 bytes): one lane each, the lane holds the whole row sum
-                        constexpr int Q = KP4 <= 8 ? KP4 : 1;
-                        if (lane < nmid) {
-                            const int s0 = segpos[i0 + lane], s1 = segpos[i0 + lane + 1];
-                            DSF_CHECK(s0 >= e0 && s1 > s0 && s1 <= e1, 11, s0 * 64 + s1);
-                            float4 t[Q];
-                            float tw = 0.f;
-#pragma unroll
-                            for (int q = 0; q < Q; ++q) t[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-                            for (int u = s0; u < s1; ++u) {
-                                const float2 cf = pc[u];
-#pragma unroll
-                                for (int q = 0; q < Q; ++q) {
-                                    const float4 r = rb[(u - e0) * KP4 + q];
-                                    t[q].x = fmaf(cf.x, r.x, t[q].x); t[q].y = fmaf(cf.x, r.y, t[q].y);
-                                    t[q].z = fmaf(cf.x, r.z, t[q].z); t[q].w = fmaf(cf.x, r.w, t[q].w);
-                                }
-                                tw += cf.y;
-                            }
-                            const uint32_t col = pcol[s0];
-                            DSF_CHECK((int64_t)col0 + col < a.d, 12, col);
-#pragma unroll
-                            for (int q = 0; q < Q; ++q) red_add4(U4 + (size_t)col * KP4 + q, t[q].x, t[q].y, t[q].z, t[q].w);
-                            red_add1(uw + col, tw);
-                        }
-                    } else {
                     for (int i = g; i < nmid; i += GW) {
-                            const int s0 = segpos[i0 + i], s1 = segpos[i0 + i + 1];
-                            DSF_CHECK(s0 >= e0 && s1 > s0 && s1 <= e1, 11, s0 * 64 + s1);
-                            float4 tmp[NV];
-                            float tmpw = 0.f;
+                        const int s0 = segpos[i0 + i], s1 = segpos[i0 + i + 1];
+                        DSF_CHECK(s0 >= e0 && s1 > s0 && s1 <= e1, 11, s0 * 64 + s1);
+                        float4 tmp[NV];
+                        float tmpw = 0.f;
 #pragma unroll
-                            for (int v = 0; v < NV; ++v) tmp[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-                            for (int u = s0; u < s1; ++u) {
-                                const float2 cf = pc[u];
+                        for (int v = 0; v < NV; ++v) tmp[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        for (int u = s0; u < s1; ++u) {
+                            const float2 cf = pc[u];
 #pragma unroll
-                                for (int v = 0; v < NV; ++v) {
-                                    const float4 r = rb[(u - e0) * KP4 + v * LG + l];
-                                    tmp[v].x = fmaf(cf.x, r.x, tmp[v].x); tmp[v].y = fmaf(cf.x, r.y, tmp[v].y);
-                                    tmp[v].z = fmaf(cf.x, r.z, tmp[v].z); tmp[v].w = fmaf(cf.x, r.w, tmp[v].w);
-                                }
-                                tmpw += cf.y;
+                            for (int v = 0; v < NV; ++v) {
+                                const float4 r = rb[(u - e0) * KP4 + v * LG + l];
+                                tmp[v].x = fmaf(cf.x, r.x, tmp[v].x); tmp[v].y = fmaf(cf.x, r.y, tmp[v].y);
+                                tmp[v].z = fmaf(cf.x, r.z, tmp[v].z); tmp[v].w = fmaf(cf.x, r.w, tmp[v].w);
                             }
-                            flush(pcol[s0], tmp, tmpw);
+                            tmpw += cf.y;
                         }
+                        flush(pcol[s0], tmp, tmpw);
                     }
                     __syncwarp();
                     // 3. the run that is open at the end of the stage
