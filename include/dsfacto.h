@@ -170,11 +170,12 @@ int dsfacto_last_epoch_ms(dsfacto_t *h, float ms[4]);
  *                             earlier tile of the same column block gives up; dsfacto_epoch then returns
  *                             DSFACTO_ERR_CUDA and the handle refuses further epochs until dsfacto_set_params
  *                             replaces w and V or dsfacto_load_csr loads a data set.
- *   DSFACTO_DEBUG_EXTRA_NEED  (before dsfacto_load_csr) the first chunk of the sweep is made to wait for that
- *                             many tiles more than exist, so that its wait runs out: the failure path above
- *                             can be exercised without a fault or a hang.
- *   DSFACTO_DEBUG_CHUNK_LEN   (before dsfacto_load_csr) entries per chunk, 16 .. 512, 0 = chosen by the load;
- *                             the environment variable DSFACTO_CHUNK does the same for every handle.
+ *   DSFACTO_DEBUG_EXTRA_NEED  (takes effect at the next dsfacto_load_csr) the first chunk of the sweep is made to
+ *                             wait for that many finished chunks more than its column block really has before
+ *                             it; with a value larger than the number of chunks its wait runs out, so the
+ *                             failure path above can be exercised without a fault or a hang.  0 = off.
+ *   DSFACTO_DEBUG_CHUNK_LEN   (takes effect at the next dsfacto_load_csr) entries per chunk, 16 .. 512, 0 = chosen
+ *                             by the load; the environment variable DSFACTO_CHUNK does the same for every handle.
  * The environment variable DSFACTO_SWEEP=round (read by dsfacto_create) stores and sweeps the tiles round by
  * round, exactly Algorithm 1's order, instead of row block by row block. */
 enum { DSFACTO_DEBUG_SPIN_LIMIT = 0, DSFACTO_DEBUG_EXTRA_NEED = 1, DSFACTO_DEBUG_CHUNK_LEN = 2 };

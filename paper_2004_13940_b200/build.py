@@ -15,6 +15,7 @@ CSRC = PKG / "csrc"
 INCLUDE = ROOT / "include"
 
 LIB_CUDA = PKG / "libdsfacto.so"
+LIB_CUDA_DEBUG = PKG / "libdsfacto_debug.so"
 LIB_WORKLOADS = PKG / "_workloads_gen.so"
 
 NVCC_ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
@@ -40,18 +41,24 @@ def _nvcc() -> str:
     return exe
 
 
-def build_cuda(force: bool = False, verbose_ptxas: bool = False) -> Path:
+def build_cuda(force: bool = False, verbose_ptxas: bool = False, debug: bool = False) -> Path:
+    """The C-ABI library.  debug=True builds libdsfacto_debug.so with -DDSFACTO_DEBUG: the stratum SGD kernel
+    then checks every index it forms (rows, columns, chunk and run bounds); a failed check is recorded in
+    the launch's error word and reported by dsfacto_epoch, nothing traps."""
     srcs = sorted(CSRC.glob("*.cu"))
     deps = srcs + sorted(CSRC.glob("*.cuh")) + sorted(CSRC.glob("*.h")) + sorted(INCLUDE.glob("*.h"))
-    if force or _stale(LIB_CUDA, deps):
-        tmp = LIB_CUDA.with_suffix(".so.tmp%d" % os.getpid())
+    target = LIB_CUDA_DEBUG if debug else LIB_CUDA
+    if force or _stale(target, deps):
+        tmp = target.with_suffix(".so.tmp%d" % os.getpid())
         cmd = [_nvcc(), "-O3", "-std=c++17", "-lineinfo", *NVCC_ARCH, "-shared", "-Xcompiler",
                "-fPIC,-O3,-fopenmp,-Wall", "-I", INCLUDE, "-I", CSRC, "-o", tmp, *srcs, "-lgomp"]
+        if debug:
+            cmd[1:1] = ["-DDSFACTO_DEBUG"]
         if verbose_ptxas:
             cmd[1:1] = ["-Xptxas", "-v"]
         _run(cmd)
-        os.replace(tmp, LIB_CUDA)
-    return LIB_CUDA
+        os.replace(tmp, target)
+    return target
 
 
 def build_workloads(force: bool = False) -> Path:
@@ -66,3 +73,4 @@ def build_workloads(force: bool = False) -> Path:
 def build_all(force: bool = False) -> None:
     build_workloads(force)
     build_cuda(force)
+    build_cuda(force, debug=True)

@@ -61,7 +61,7 @@ struct dsfacto {
     int chunk_override = 0;     // > 0: chunk length forced by dsfacto_debug_set (tests)
     int sgd_grid = 0;           // CTAs of the persistent stratum SGD launch
     int spin_limit = kSgdSpinLimit;  // polls before a wait for an earlier tile gives up
-    int debug_extra_need = 0;   // tests: added to the `need` of the first chunk, so that its wait runs out
+    int debug_extra_need = 0;   // tests: added to the `need` of the first chunk at the next load, so that its wait runs out
     bool failed = false;        // an SGD launch gave up; the parameters are unusable until they are set again
     float *d_records = nullptr, *d_Tb = nullptr, *d_Tw = nullptr;
     float4 *d_S = nullptr, *d_TS = nullptr;  // scale records of the scaled column state (zero outside the SGD phase)
@@ -1396,11 +1396,11 @@ int dsfacto_debug_set(dsfacto_t *h, int32_t key, int64_t value) {
         h->spin_limit = (int)value;
         return DSFACTO_OK;
     case DSFACTO_DEBUG_EXTRA_NEED:
-        if (value < 0 || value > 1000 || h->loaded) return DSFACTO_ERR_INVALID_ARG;
+        if (value < 0 || value > kTicketStop) return DSFACTO_ERR_INVALID_ARG;
         h->debug_extra_need = (int)value;
         return DSFACTO_OK;
     case DSFACTO_DEBUG_CHUNK_LEN:
-        if ((value != 0 && (value < 16 || value > kChunkMax)) || h->loaded) return DSFACTO_ERR_INVALID_ARG;
+        if (value != 0 && (value < 16 || value > kChunkMax)) return DSFACTO_ERR_INVALID_ARG;
         h->chunk_override = (int)value;
         return DSFACTO_OK;
     default:

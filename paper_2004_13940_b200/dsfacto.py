@@ -49,16 +49,35 @@ SIGNATURES = {
 _lib = None
 
 
+def _load(path) -> ctypes.CDLL:
+    L = ctypes.CDLL(str(path))
+    for name, (res, args) in SIGNATURES.items():
+        fn = getattr(L, name)
+        fn.restype, fn.argtypes = res, args
+    return L
+
+
 def lib() -> ctypes.CDLL:
     """Loads (building first if the sources are newer) libdsfacto.so; raises if that fails."""
     global _lib
     if _lib is None:
-        L = ctypes.CDLL(str(_build.build_cuda()))
-        for name, (res, args) in SIGNATURES.items():
-            fn = getattr(L, name)
-            fn.restype, fn.argtypes = res, args
-        _lib = L
+        _lib = _load(_build.build_cuda())
     return _lib
+
+
+class use_debug_library:
+    """Context manager: inside it every call of this module goes to libdsfacto_debug.so, the same sources
+    built with -DDSFACTO_DEBUG (index checks in the stratum SGD kernel that report instead of trapping)."""
+
+    def __enter__(self):
+        global _lib
+        self._saved = lib()
+        _lib = _load(_build.build_cuda(debug=True))
+        return _lib
+
+    def __exit__(self, *exc):
+        global _lib
+        _lib = self._saved
 
 
 class DSFactoError(RuntimeError):
@@ -279,6 +298,9 @@ class DSFacto:
         ms = (ctypes.c_float * 4)()
         self._check(lib().dsfacto_last_epoch_ms(self._h, ms), "dsfacto_last_epoch_ms")
         return [float(x) for x in ms]
+
+    def debug_set(self, key: int, value: int):
+        self._check(dsfacto_debug_set(self._h, int(key), int(value)), "dsfacto_debug_set")
 
     def launch_count(self) -> int:
         v = _c_i64()
