@@ -32,9 +32,10 @@ sys.path.insert(0, str(ROOT))
 METRIC = "nonzero-updates/sec"
 UNIT = "updates/s"
 ORACLE_SAMPLE_ROWS = 1_000_000
-# dram__bytes_read.sum + dram__bytes_write.sum of sgd_chunk_kernel per stored entry, from the ncu capture
-# summarised in profiles/ (None once the kernel has changed since the counters were taken)
-SGD_DRAM_BYTES_PER_ENTRY = None
+# dram__bytes_read.sum + dram__bytes_write.sum of sgd_sweep_kernel per stored entry, by factor width K, from
+# the ncu captures summarised in profiles/ (scaled cases; DRAM traffic of the sweep grows with the entries).
+# A width without a capture of the current kernel reports traffic = null.
+SGD_DRAM_BYTES_PER_ENTRY = {}
 
 
 def peaks():
@@ -252,12 +253,22 @@ def run_ours(args):
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     phase = np.zeros(4)
     ev0.record(stream)
-    for _ in range(args.steps):
+    epoch_log = []
+    for step in range(args.steps):
         g.epoch()
-        phase += np.asarray(g.last_epoch_ms())
+        ph = np.asarray(g.last_epoch_ms())
+        phase += ph
+        if args.log and rank == 0:
+            epoch_log.append({"epoch": args.warmup + step + 1, "objective": g.objective(), "loss": g.stats()[0],
+                              "seconds": ph[0] * 1e-3, "nnz_updates_per_s": nnz / (ph[0] * 1e-3),
+                              "ms": {"sgd_strata": float(ph[1]), "refresh": float(ph[2]), "norms": float(ph[3])}})
     ev1.record(stream)
     torch.cuda.synchronize(); barrier()
     clocks = sampler.stop(t_begin, datetime.datetime.now()) if rank == 0 else None
+    if args.log and rank == 0:
+        with open(args.log, "a") as fh:
+            for rec in epoch_log:
+                fh.write(json.dumps(rec) + "\n")
     ms = ev0.elapsed_time(ev1)
     launches = g.launch_count() - launches0
     objective = g.objective()
@@ -265,19 +276,23 @@ def run_ours(args):
 
     # ---- e2e: host buffers -> load_csr -> epoch -> objective, through the C ABI ----
     def e2e_leg():
-        torch.cuda.synchronize()
-        t0 = time.perf_counter()
+        per_step = []
         for _ in range(args.e2e_steps):
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
             hh = new_handle()
             hh.load_csr(wl.indptr, wl.indices, wl.values, wl.y)
             hh.epoch()
             _ = hh.objective()
             hh.close()
-        torch.cuda.synchronize()
-        return 1e3 * (time.perf_counter() - t0)
+            torch.cuda.synchronize()
+            per_step.append(1e3 * (time.perf_counter() - t0))
+        return per_step
 
-    e2e_ms = take_turns(rank, world, barrier, e2e_leg)
-    ms, e2e_ms = max_over_ranks([ms, e2e_ms], world, "cuda")
+    e2e_steps_ms = take_turns(rank, world, barrier, e2e_leg) or [0.0]
+    e2e_ms = float(sum(e2e_steps_ms))
+    e2e_min, e2e_med = float(min(e2e_steps_ms)), float(statistics.median(e2e_steps_ms))
+    ms, e2e_ms, e2e_min, e2e_med = max_over_ranks([ms, e2e_ms, e2e_min, e2e_med], world, "cuda")
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -297,21 +312,24 @@ def run_ours(args):
     ref_bytes = 8 * nnz + 8 * (n + 1) + 4 * d * (K + 2) + 4 * n * K + 8 * n
     sgd_s, ref_s = phase[1] * 1e-3, phase[2] * 1e-3
     # the counters were taken on the default schedule (row-block sweep, one launch per sweep)
-    traffic = None if (SGD_DRAM_BYTES_PER_ENTRY is None or sweep != "rowblock") else SGD_DRAM_BYTES_PER_ENTRY * nnz
+    per_entry = SGD_DRAM_BYTES_PER_ENTRY.get(K)
+    traffic = None if (per_entry is None or sweep != "rowblock" or segments != 1) else per_entry * nnz
     roof = {"bound": "hbm", "kernel": "sgd_sweep_kernel", "launches_per_step": segments, "sweep": sweep,
             "achieved": sgd_bytes / sgd_s / 1e9, "peak": peak, "unit": "GB/s", "frac": sgd_bytes / sgd_s / 1e9 / peak,
             "peak_kind": "of " + peak_kind, "traffic": traffic,
             "algorithmic_bytes_per_launch": sgd_bytes / segments, "avg_launch_us": 1e6 * sgd_s / segments,
             "model": ("gather: nnz*(8+4K+4) + 8d(K+1)" if sweep == "round" else "stream floor: 8nnz + 4n(K+1) + 8d(K+1)")
                      + "; one launch covers the whole sweep",
-            "gather_model": {"bytes_per_step": sgd_gather, "achieved": sgd_gather / sgd_s / 1e9,
-                             "frac": sgd_gather / sgd_s / 1e9 / peak},
+            # bytes the sweep asks its caches for when nothing is reused in registers; most of them are served
+            # by L2, so this rate is NOT a fraction of the HBM peak and is given for context only
+            "cache_request_model": {"bytes_per_step": sgd_gather, "rate_GBps": sgd_gather / sgd_s / 1e9},
             "refresh_kernel": {"algorithmic_bytes_per_step": ref_bytes, "ms": phase[2],
                                "achieved": ref_bytes / ref_s / 1e9, "frac": ref_bytes / ref_s / 1e9 / peak}}
     value = whole_job_rate(world, nnz, args.steps, ms)
     h2d = (wl.indptr.nbytes + wl.indices.nbytes + wl.values.nbytes + wl.y.nbytes + 8 * nnz + 8 * (p * p + 1))
     e2e = {"value": whole_job_rate(world, nnz, args.e2e_steps, e2e_ms) if args.e2e_steps > 0 else None, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
            "d2h_bytes_per_step": 32, "steps": args.e2e_steps, "ms_per_step": e2e_ms / max(args.e2e_steps, 1),
+           "ms_per_step_min": e2e_min, "ms_per_step_median": e2e_med,
            "what": "dsfacto_create + dsfacto_load_csr (host bucketing streamed to the device, H2D) + dsfacto_epoch + dsfacto_objective"}
     cfg = workload_config(args.workload)
     if args.refresh_every > 0:
@@ -343,7 +361,9 @@ def main():
     ap.add_argument("--p", type=int, default=None, help="override the tile grid (profiling)")
     ap.add_argument("--refresh-every", type=int, default=0,
                     help="second schedule: recompute G, A after every R inner rounds (0: once per epoch)")
-    ap.add_argument("--e2e-steps", type=int, default=1)
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--log", default=None, help="append one JSON line per timed epoch to this file: epoch, objective, "
+                                                "mean loss, seconds, updates/s, per-phase ms")
     ap.add_argument("--oracle-rows", type=int, default=ORACLE_SAMPLE_ROWS)
     ap.add_argument("--oracle-seconds", type=float, default=10.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")

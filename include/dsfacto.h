@@ -117,8 +117,8 @@ int dsfacto_set_eta(dsfacto_t *h, float eta);
  * shorter) and runs the recompute pass after every segment; before a segment of m rounds w0 takes the
  * share m/p of its step, w0 <- w0 - (eta/n) (m/p) sum_i G_i, with the multipliers frozen for that
  * segment.  R >= p is the default schedule.  An epoch then costs ceil(p/R) recompute passes.
- * Must be called before dsfacto_load_csr (DSFACTO_ERR_INVALID_ARG afterwards): a value > 0 makes the
- * load store the tiles round by round, and the handle keeps that order even if 0 is set later. */
+ * Must be called before dsfacto_load_csr (DSFACTO_ERR_INVALID_ARG afterwards): the load cuts its launch
+ * plan into the segments. */
 int dsfacto_set_refresh_every(dsfacto_t *h, int32_t rounds);
 
 /* Objective eq. (fm_obj) as of the last recompute pass (after load_csr, epoch or set_params). */
@@ -209,8 +209,9 @@ const char *dsfacto_strerror(int status);
  * 1 <= m <= 67,108,864 rows, because the per-CTA partial sums of the reduction live in a fixed
  * 1 MiB array inside the library image (every GPU that loads the library holds it until the
  * process exits).  Anything outside these limits returns DSFACTO_ERR_INVALID_ARG.
- * The first call on each device looks up that array's device address; make this first call
- * outside any stream capture.  All calls on a device share the array: it keeps the last call's
+ * V_dev must be 16-byte aligned and none of the pointers may be NULL (DSFACTO_ERR_INVALID_ARG otherwise).
+ * The first call on each device looks up that array's device address (a host-side query, once per
+ * device).  All calls on a device share the array: it keeps the last call's
  * contents, every call overwrites the slots it uses before reading them (nothing needs clearing),
  * and two calls that overlap on the GPU (different streams or threads) race on it - serialise them.
  * The call performs no cudaMalloc/cudaFree and returns after its work on the stream has finished. */

@@ -52,7 +52,8 @@ struct dsfacto {
     double *d_partials = nullptr, *d_scal = nullptr;
     // stratum SGD launch plan: launch L covers chunks [launch_ptr[L], launch_ptr[L+1]) of chunk_map
     int sweep = 1;  // 1: a launch is a row block (p-1 .. 0); 0: a launch is an inner round (0 .. p-1)
-    int refresh_every = 0;  // > 0: G, A recomputed after every that many inner rounds (needs the round sweep)
+    int refresh_every = 0;  // > 0: G, A recomputed after every that many inner rounds
+    int64_t plan_segments = 0;  // > 0: the launch plan is cut into that many segments of refresh_every rounds (row-block sweep)
     std::vector<int64_t> launch_ptr;
     ChunkDesc *d_desc = nullptr;   // chunk descriptors in sweep order
     int *d_sync = nullptr;     // ticket, error word, per-column-block progress of the fused SGD launch
@@ -424,30 +425,58 @@ int finish_sgd_plan(dsfacto *h, SgdPlanBuild &pb) {
         h->launch_ptr.assign((size_t)p + 1, 0);
         seen.assign((size_t)p, 0);
     } catch (const std::bad_alloc &) { return DSFACTO_ERR_OOM; }
+    // Segments: with the second schedule (recompute after every R inner rounds) on the row-block sweep, a
+    // launch covers the tiles of R consecutive rounds, still visited row block by row block.  For column
+    // block c a segment that starts at round s0 begins at row block (c - s0) mod p and descends cyclically,
+    // so inside a segment the tiles above that row block are the ones that act on the tail composite.
+    const bool segmented = h->sweep == 1 && h->refresh_every > 0 && h->refresh_every < p;
+    const int64_t every = segmented ? h->refresh_every : p;
+    const int64_t nseg = segmented ? (p + every - 1) / every : 1;
+    try {
+        if (segmented) h->launch_ptr.assign((size_t)nseg + 1, 0);
+    } catch (const std::bad_alloc &) { return DSFACTO_ERR_OOM; }
+    h->plan_segments = segmented ? nseg : 0;
     int64_t pos = 0, runs = 0, recs = 0, cur_run = 0, cur_rec0 = 0;
-    for (int64_t slot = 0; slot < nt; ++slot) {
-        int64_t r, c;
-        slot_tile(h, slot, r, c);
-        const TileDescRef &ref = pb.refs[(size_t)slot];
-        const bool tail = h->sweep == 1 && r > c;
-        for (int32_t q = 0; q < ref.count; ++q) {
-            ChunkDesc d = pb.planners[(size_t)ref.owner].descs[(size_t)(ref.first + q)];
-            d.row0 = (int32_t)h->row_start[(size_t)r];
-            d.col0 = h->col_start[(size_t)c];
-            d.cblock = (int32_t)c;
-            d.need = seen[(size_t)c];
-            d.tile = (int32_t)slot;
-            d.nchunks = ref.count;
-            if (tail) d.flags |= kChunkTail;
-            if (d.flags & kChunkSlice) {
-                if (d.slice == 0) { cur_run = runs++; cur_rec0 = recs; recs += d.nslices; }
-                d.run_id = (int32_t)cur_run;
-                d.rec0 = (int32_t)cur_rec0;
+    for (int64_t seg = 0; seg < nseg; ++seg) {
+        const int64_t s0 = seg * every, s1 = std::min(s0 + every, p);
+        if (segmented) std::fill(seen.begin(), seen.end(), 0);
+        // plain plan: every slot in order; segmented plan: row block by row block, the tiles of rounds [s0, s1)
+        const int64_t visits = segmented ? p * (s1 - s0) : nt;
+        for (int64_t vis = 0; vis < visits; ++vis) {
+            int64_t slot = vis, r, c;
+            bool tail;
+            if (segmented) {
+                r = p - 1 - vis / (s1 - s0);
+                c = (r + s0 + vis % (s1 - s0)) % p;
+                slot = tile_slot(h, r, c);
+                int64_t r_first = c - s0;
+                if (r_first < 0) r_first += p;
+                tail = r > r_first;
+            } else {
+                slot_tile(h, slot, r, c);
+                tail = h->sweep == 1 && r > c;
             }
-            all[(size_t)pos++] = d;
+            const TileDescRef &ref = pb.refs[(size_t)slot];
+            for (int32_t q = 0; q < ref.count; ++q) {
+                ChunkDesc d = pb.planners[(size_t)ref.owner].descs[(size_t)(ref.first + q)];
+                d.row0 = (int32_t)h->row_start[(size_t)r];
+                d.col0 = h->col_start[(size_t)c];
+                d.cblock = (int32_t)c;
+                d.need = seen[(size_t)c];
+                d.tile = (int32_t)slot;
+                d.nchunks = ref.count;
+                if (tail) d.flags |= kChunkTail;
+                if (d.flags & kChunkSlice) {
+                    if (d.slice == 0) { cur_run = runs++; cur_rec0 = recs; recs += d.nslices; }
+                    d.run_id = (int32_t)cur_run;
+                    d.rec0 = (int32_t)cur_rec0;
+                }
+                all[(size_t)pos++] = d;
+            }
+            seen[(size_t)c] += ref.count;
+            if (!segmented && (slot + 1) % p == 0) h->launch_ptr[(size_t)((slot + 1) / p)] = pos;
         }
-        seen[(size_t)c] += ref.count;
-        if ((slot + 1) % p == 0) h->launch_ptr[(size_t)((slot + 1) / p)] = pos;
+        if (segmented) h->launch_ptr[(size_t)seg + 1] = pos;
     }
     if (recs >= ((int64_t)1 << 31)) return DSFACTO_ERR_INVALID_ARG;
     h->total_chunks = total;
@@ -483,11 +512,15 @@ void run_sgd_phase(dsfacto *h, int64_t L0, int64_t L1) {
     // by round) and a tile waits only for the earlier tiles of its own column block.  The counters of
     // finished tiles are cumulative over the sweep, so they are cleared at its first launch only; the
     // ticket counter restarts with every launch.
-    if (L0 == 0) cudaMemsetAsync(h->d_sync, 0, sizeof(int) * sync_words(h->p), h->stream);
+    // With a segmented plan (second schedule on the row-block sweep) a launch is one segment, whose chunks count
+    // their earlier tiles from the segment's start: all words are cleared every time.
+    int64_t first = L0, last = L1;
+    if (h->plan_segments > 0) { first = L0 / h->refresh_every; last = first + 1; }
+    if (L0 == 0 || h->plan_segments > 0) cudaMemsetAsync(h->d_sync, 0, sizeof(int) * sync_words(h->p), h->stream);
     else cudaMemsetAsync(h->d_sync + kSyncTicket, 0, sizeof(int), h->stream);
     a.sync = h->d_sync;
-    const int64_t chunks = h->launch_ptr[(size_t)L1] - h->launch_ptr[(size_t)L0];
-    a.desc = h->d_desc + h->launch_ptr[(size_t)L0];
+    const int64_t chunks = h->launch_ptr[(size_t)last] - h->launch_ptr[(size_t)first];
+    a.desc = h->d_desc + h->launch_ptr[(size_t)first];
     a.nchunks = (int)chunks;
     if (chunks > 0) {
         DSF_DISPATCH(h, launch_sgd, h, a, chunks);
@@ -572,6 +605,8 @@ int validate_csr(int64_t m, int32_t d, const int64_t *indptr, const int32_t *ind
 // ascending inside a tile because threads own ascending row ranges), then a stable counting sort
 // by local column inside every tile.
 // ---------------------------------------------------------------------------------------------
+void column_blocks(const dsfacto *h, std::vector<int32_t> &cb);
+
 int bucket_tiles(dsfacto *h, const int64_t *indptr, const int32_t *indices, const float *values,
                  HostBuf<uint2> &ent, HostBuf<float> &xw, SgdPlanBuild *pb) {
     const int64_t n = h->n, nnz = indptr[n];
@@ -583,12 +618,12 @@ int bucket_tiles(dsfacto *h, const int64_t *indptr, const int32_t *indices, cons
     if (T > 64) T = 64;
     if ((int64_t)T > n) T = (int)std::max<int64_t>(1, n);
 
-    std::vector<int32_t> cb(d);  // column block of every column
-    for (int32_t c = 0; c < p; ++c)
-        for (int32_t j = h->col_start[c]; j < h->col_start[c + 1]; ++j) cb[j] = c;
-
-    // thread k owns rows [rs[k], rs[k+1]) chosen to balance stored entries
-    std::vector<int64_t> rs(T + 1);
+    std::vector<int32_t> cb;  // column block of every column
+    std::vector<int64_t> rs;  // thread k owns rows [rs[k], rs[k+1]) chosen to balance stored entries
+    try {
+        column_blocks(h, cb);
+        rs.resize((size_t)T + 1);
+    } catch (const std::bad_alloc &) { return DSFACTO_ERR_OOM; }
     rs[0] = 0;
     for (int k = 1; k < T; ++k) {
         const int64_t target = (int64_t)((__int128)nnz * k / T);
@@ -609,7 +644,7 @@ int bucket_tiles(dsfacto *h, const int64_t *indptr, const int32_t *indices, cons
     } catch (const std::bad_alloc &) {
         return DSFACTO_ERR_OOM;
     }
-    h->tile_ptr.assign((size_t)nt + 1, 0);
+    try { h->tile_ptr.assign((size_t)nt + 1, 0); } catch (const std::bad_alloc &) { return DSFACTO_ERR_OOM; }
 
 #pragma omp parallel num_threads(T)
     {
@@ -626,7 +661,6 @@ int bucket_tiles(dsfacto *h, const int64_t *indptr, const int32_t *indices, cons
     // offsets: tile-major, thread-minor
     {
         int64_t run = 0;
-        std::vector<int64_t> off((size_t)T);
         for (int64_t t = 0; t < nt; ++t) {
             h->tile_ptr[t] = run;
             for (int k = 0; k < T; ++k) run += counts[(size_t)k * nt + t];
@@ -664,18 +698,31 @@ int bucket_tiles(dsfacto *h, const int64_t *indptr, const int32_t *indices, cons
     }
     // stable counting sort by local column inside each tile
     const uint32_t jmask = jbits >= 32 ? 0xFFFFFFFFu : ((1u << jbits) - 1u);
+    int64_t widest = 0;
+    for (int32_t c = 0; c < p; ++c) widest = std::max<int64_t>(widest, h->col_start[c + 1] - h->col_start[c]);
+    int sort_failed = 0;
 #pragma omp parallel
     {
         std::vector<int64_t> hist;
+        bool have = true;
+        try { hist.resize((size_t)widest + 1); } catch (const std::bad_alloc &) { have = false; }
+        if (!have) {
+#pragma omp atomic write
+            sort_failed = 1;
+        }
+#pragma omp barrier
+        int stop;
+#pragma omp atomic read
+        stop = sort_failed;
 #pragma omp for schedule(dynamic, 8)
         for (int64_t t = 0; t < nt; ++t) {
             const int64_t b = h->tile_ptr[t], e = h->tile_ptr[t + 1];
-            if (b == e) continue;
+            if (b == e || stop) continue;
             int64_t r, c;
             slot_tile(h, t, r, c);
             (void)r;
             const int64_t width = h->col_start[c + 1] - h->col_start[c];
-            hist.assign((size_t)width + 1, 0);
+            std::fill(hist.begin(), hist.begin() + width + 1, (int64_t)0);
             for (int64_t q = b; q < e; ++q) {
                 const uint32_t jl = wide ? tmp_e[q].y : (tmp_e[q].x & jmask);
                 hist[jl + 1] += 1;
@@ -690,7 +737,7 @@ int bucket_tiles(dsfacto *h, const int64_t *indptr, const int32_t *indices, cons
             plan_tile(h, pb, omp_get_thread_num(), t, b, hist.data(), width);   // hist[j] is now the end of column j
         }
     }
-    return DSFACTO_OK;
+    return sort_failed ? DSFACTO_ERR_OOM : DSFACTO_OK;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -723,7 +770,7 @@ void column_blocks(const dsfacto *h, std::vector<int32_t> &cb) {
 // counts per tile (slot order) -> h->tile_ptr; returns the largest number of entries of a row block
 int64_t count_tiles_by_row_block(dsfacto *h, const std::vector<int32_t> &cb, const int64_t *indptr, const int32_t *indices) {
     const int64_t p = h->p, nt = p * p;
-    h->tile_ptr.assign((size_t)nt + 1, 0);
+    try { h->tile_ptr.assign((size_t)nt + 1, 0); } catch (const std::bad_alloc &) { return -1; }
 #pragma omp parallel for schedule(dynamic, 1)
     for (int64_t r = 0; r < p; ++r) {
         int64_t *cnt = h->tile_ptr.data() + 1 + (p - 1 - r) * p;   // slot (p-1-r)*p + c
@@ -768,7 +815,7 @@ void bucket_row_block(const dsfacto *h, int64_t r, const std::vector<int32_t> &c
         const int64_t b = tp[c] - base, e = tp[c + 1] - base;
         if (b == e) continue;
         const int64_t width = h->col_start[c + 1] - h->col_start[c];
-        sc.hist.assign((size_t)width + 1, 0);
+        std::fill(sc.hist.begin(), sc.hist.begin() + width + 1, (int64_t)0);   // (sized for the widest column block)
         for (int64_t q = b; q < e; ++q) sc.hist[(wide ? tmp_e[q].y : (tmp_e[q].x & jmask)) + 1] += 1;
         for (int64_t j = 0; j < width; ++j) sc.hist[(size_t)j + 1] += sc.hist[(size_t)j];
         for (int64_t q = b; q < e; ++q) {
@@ -782,7 +829,12 @@ void bucket_row_block(const dsfacto *h, int64_t r, const std::vector<int32_t> &c
 }
 
 bool alloc_row_block_scratch(const dsfacto *h, RowBlockScratch &sc, int64_t longest) {
-    try { sc.fill.assign((size_t)h->p, 0); } catch (const std::bad_alloc &) { return false; }
+    int64_t widest = 0;
+    for (int32_t c = 0; c < h->p; ++c) widest = std::max<int64_t>(widest, h->col_start[(size_t)c + 1] - h->col_start[(size_t)c]);
+    try {
+        sc.fill.assign((size_t)h->p, 0);
+        sc.hist.assign((size_t)widest + 1, 0);
+    } catch (const std::bad_alloc &) { return false; }
     return sc.tmp_e.alloc((size_t)longest) && (!h->wide || sc.tmp_x.alloc((size_t)longest));
 }
 
@@ -793,6 +845,7 @@ int bucket_tiles_by_row_block(dsfacto *h, const int64_t *indptr, const int32_t *
     std::vector<int32_t> cb;
     try { column_blocks(h, cb); } catch (const std::bad_alloc &) { return DSFACTO_ERR_OOM; }
     const int64_t longest = count_tiles_by_row_block(h, cb, indptr, indices);
+    if (longest < 0) return DSFACTO_ERR_OOM;
     if (!ent.alloc((size_t)nnz) || (h->wide && !xw.alloc((size_t)nnz))) return DSFACTO_ERR_OOM;
     int failed = 0;
 #pragma omp parallel
@@ -1091,6 +1144,7 @@ int dsfacto_load_csr(dsfacto_t *h, const int64_t *indptr, const int32_t *indices
     if (streamed) {
         try { column_blocks(h, cb); } catch (const std::bad_alloc &) { cudaStreamSynchronize(st); free_data(h); return DSFACTO_ERR_OOM; }
         longest = count_tiles_by_row_block(h, cb, indptr, indices);
+        if (longest < 0) { cudaStreamSynchronize(st); free_data(h); return DSFACTO_ERR_OOM; }
     } else {
         rc = by_row_block ? bucket_tiles_by_row_block(h, indptr, indices, values, ent, xw, &pb)
                           : bucket_tiles(h, indptr, indices, values, ent, xw, &pb);
@@ -1189,12 +1243,7 @@ int dsfacto_epoch(dsfacto_t *h) {
 int dsfacto_set_refresh_every(dsfacto_t *h, int32_t rounds) {
     if (!h || rounds < 0) return DSFACTO_ERR_INVALID_ARG;
     if (h->loaded) return DSFACTO_ERR_INVALID_ARG;   // the tile order on the device is fixed by dsfacto_load_csr
-    h->refresh_every = rounds;
-    if (rounds > 0 && h->sweep != 0) {
-        // inner rounds must be launches of their own: switch to the round sweep (no tail composites)
-        h->sweep = 0;
-        dev_free(h->d_Tb); dev_free(h->d_Tw); dev_free(h->d_TS);
-    }
+    h->refresh_every = rounds;   // the launch plan built by dsfacto_load_csr is cut into segments of that many rounds
     return DSFACTO_OK;
 }
 
@@ -1256,7 +1305,8 @@ int dsfacto_get_tiles(dsfacto_t *h, int64_t *tile_ptr, int32_t *rows, int32_t *c
     if (!h) return DSFACTO_ERR_INVALID_ARG;
     if (!h->loaded) return DSFACTO_ERR_NO_DATA;
     const int64_t nt = (int64_t)h->p * h->p;
-    const std::vector<int64_t> canon = canonical_tile_ptr(h);
+    std::vector<int64_t> canon;
+    try { canon = canonical_tile_ptr(h); } catch (const std::bad_alloc &) { return DSFACTO_ERR_OOM; }
     if (tile_ptr) std::memcpy(tile_ptr, canon.data(), sizeof(int64_t) * ((size_t)nt + 1));
     if (!rows && !cols && !vals) return DSFACTO_OK;
     HostBuf<uint2> ent;
@@ -1288,7 +1338,8 @@ int dsfacto_bucket_host(int64_t n, int32_t d, int32_t p, const int64_t *indptr, 
     rc = tmp.sweep == 1 ? bucket_tiles_by_row_block(&tmp, indptr, indices, values, ent, xw, nullptr)
                         : bucket_tiles(&tmp, indptr, indices, values, ent, xw, nullptr);
     if (rc) return rc;
-    const std::vector<int64_t> canon = canonical_tile_ptr(&tmp);
+    std::vector<int64_t> canon;
+    try { canon = canonical_tile_ptr(&tmp); } catch (const std::bad_alloc &) { return DSFACTO_ERR_OOM; }
     std::memcpy(tile_ptr, canon.data(), sizeof(int64_t) * canon.size());
     unpack_tiles(&tmp, canon, ent.data(), xw.data(), rows, cols, vals);
     return DSFACTO_OK;

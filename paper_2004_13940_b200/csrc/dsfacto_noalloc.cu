@@ -12,6 +12,7 @@
 #include "dsfacto_common.cuh"
 
 #include <cmath>
+#include <cstdint>
 
 namespace {
 
@@ -130,7 +131,11 @@ extern "C" int dsfacto_score_loss_noalloc(int64_t m, int32_t d, int32_t K, int32
                                           const int32_t *indices_dev, const float *values_dev, const float *y_dev,
                                           float w0, const float *w_dev, const float *V_dev, float *scores_dev,
                                           double *sums_dev, void *cuda_stream) {
-    if (m < 1 || d < 1 || !indptr_dev || !y_dev || !w_dev || !V_dev || !scores_dev || !sums_dev) return DSFACTO_ERR_INVALID_ARG;
+    if (m < 1 || d < 1 || !indptr_dev || !indices_dev || !values_dev || !y_dev || !w_dev || !V_dev || !scores_dev || !sums_dev)
+        return DSFACTO_ERR_INVALID_ARG;
+    // rows of V are read 16 bytes at a time: a pointer that is not 16-byte aligned would fault on the device,
+    // so it is refused here instead
+    if ((reinterpret_cast<uintptr_t>(V_dev) & 15u) != 0) return DSFACTO_ERR_INVALID_ARG;
     if (loss != DSFACTO_SQUARED && loss != DSFACTO_LOGISTIC) return DSFACTO_ERR_INVALID_ARG;
     if (!std::isfinite(w0)) return DSFACTO_ERR_INVALID_ARG;
     // rows of V are read as float4 lane groups: K must be 4, 8, 16, 32, 64, 128 or 256

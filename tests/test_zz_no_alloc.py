@@ -63,6 +63,16 @@ def test_two_calls_in_a_row_match_the_handle_based_path():
     _check(W.make("C1"), seed=2)          # 2,000 rows, K = 8, squared
 
 
+@pytest.mark.parametrize("K", [4, 256])
+def test_narrowest_and_widest_factor_rows(K):
+    # K = 4 is one lane per row, K = 256 two 16-byte pieces per lane of a whole warp: the two ends of the
+    # lane layouts the entry point is built for
+    wl = W.make("C2", n=3000)
+    wl.K = K
+    _check(wl, seed=K)
+    _check(wl, seed=K + 1)
+
+
 def test_limits_are_rejected_with_a_clear_status():
     import torch
 
@@ -79,5 +89,7 @@ def test_limits_are_rejected_with_a_clear_status():
     assert call(m=67_108_865) == D.ERR_INVALID_ARG            # beyond the fixed scratch array
     assert call(m=0) == D.ERR_INVALID_ARG
     assert call(loss=3) == D.ERR_INVALID_ARG
+    # V not 16-byte aligned: refused on the host, never handed to the kernel
+    assert D.dsfacto_score_loss_noalloc(4, 4, 8, 0, p, p, p, p, 0.0, p, p + 4, p, p, 0) == D.ERR_INVALID_ARG
     assert D.lib().dsfacto_score_loss_noalloc(4, 4, 8, 0, None, None, None, None, 0.0, None, None, None, None,
                                               None) == D.ERR_INVALID_ARG
