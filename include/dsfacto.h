@@ -189,6 +189,48 @@ const char *dsfacto_last_error(dsfacto_t *h);
 
 const char *dsfacto_strerror(int status);
 
+/* ---- column shards: the partition of Section 4.2 across several GPUs ----
+ *
+ * Section 4.2 spreads the column blocks of w and V over the workers and lets every worker see the rows.
+ * With G and A frozen the columns never interact during the update loop, so a shard that owns a contiguous
+ * range of column blocks runs the strata of its own tiles without any exchange; only the recompute pass needs
+ * the other shards: a_ik, lin_i = sum_j w_j x_ij and q_i = sum_j sum_k v_jk^2 x_ij^2 are sums over columns.
+ * Each shard computes them over its own columns, the partial results are added up across the shards (one
+ * all-reduce of n (Kp + 2) floats, outside this library: NCCL through torch.distributed in the Python
+ * package), and every shard finishes the pass (f_i, l_i, G_i) from the totals.  The paper's own way of moving
+ * column blocks between workers round by round is the distributed-memory form of the same partition.
+ *
+ * dsfacto_create_shard: like dsfacto_create for shard `shard` of `nshards` (1 <= nshards <= p); the handle
+ *   owns column blocks [floor(shard p / nshards), floor((shard+1) p / nshards)).  w, V of other columns are
+ *   held but never touched.  dsfacto_shard_columns returns the owned column range [col_lo, col_hi).
+ * dsfacto_load_csr on a shard takes the WHOLE data set, keeps the stored entries of its own columns, builds
+ *   their tile lists (the canonical lists restricted to those columns) and computes the partial auxiliaries of
+ *   the initial parameters; the caller then adds the shards' partial buffers up and calls
+ *   dsfacto_shard_epoch_end once before the first epoch.
+ * One epoch of a shard:
+ *   dsfacto_shard_epoch_begin   w0 step (identical on every shard), the p strata over the shard's tiles, the
+ *                               partial recompute pass
+ *   dsfacto_shard_partial       copies the partial buffer [A (n x Kp, Kp = K rounded up to the lane layout) |
+ *                               lin (n) | q (n)], dsfacto_shard_partial_count floats, to DEVICE memory of the caller
+ *   (the caller sums the buffers of all shards)
+ *   dsfacto_shard_epoch_end     takes the summed buffer (DEVICE memory), finishes the recompute pass and returns
+ *                               sums[4] = { sum_i l_i, sum_i G_i, sum of w_j^2 and sum of v_jk^2 over the shard's
+ *                               OWN columns }; the objective eq. (fm_obj) is sums[0]/n + lambda_w/2 (sum of the
+ *                               shards' sums[2]) + lambda_v/2 (sum of the shards' sums[3]).
+ * dsfacto_epoch and dsfacto_set_refresh_every(> 0) are refused on a shard (DSFACTO_ERR_INVALID_ARG).
+ * dsfacto_bucket_host_shard is dsfacto_bucket_host for one shard: the tile lists of the entries whose column
+ * the shard owns (*kept = their number); it touches no GPU. */
+int dsfacto_create_shard(dsfacto_t **out, int64_t n, int32_t d, int32_t K, int32_t p, int32_t loss,
+                         float lambda_w, float lambda_v, float eta, uint64_t seed, int32_t shard, int32_t nshards);
+int dsfacto_shard_columns(dsfacto_t *h, int32_t *col_lo, int32_t *col_hi);
+int dsfacto_shard_partial_count(dsfacto_t *h, int64_t *count);
+int dsfacto_shard_epoch_begin(dsfacto_t *h);
+int dsfacto_shard_partial(dsfacto_t *h, float *dst_dev, int64_t count);
+int dsfacto_shard_epoch_end(dsfacto_t *h, const float *summed_dev, int64_t count, double sums[4]);
+int dsfacto_bucket_host_shard(int64_t n, int32_t d, int32_t p, int32_t shard, int32_t nshards, const int64_t *indptr,
+                              const int32_t *indices, const float *values, int64_t *kept, int64_t *tile_ptr,
+                              int32_t *rows, int32_t *cols, float *vals);
+
 /* ---- for callers that cannot allocate ---- */
 
 /* Scores, loss sum and multiplier sum of m rows, without any allocation.  (The paper has no

@@ -32,6 +32,11 @@ struct dsfacto {
     uint64_t seed = 0;
     float w0 = 0.f;
     bool loaded = false, wide = false;
+    // column shard (Section 4.2: the column blocks of w and V spread over workers): this handle owns column
+    // blocks [cb_lo, cb_hi), i.e. columns [col_lo, col_hi); nshards == 1 is the ordinary handle
+    int32_t shard = 0, nshards = 1, cb_lo = 0, cb_hi = 0, col_lo = 0, col_hi = 0;
+    bool awaiting_sum = false;   // shard: partial auxiliaries computed, totals not yet handed in
+    float *d_lin = nullptr, *d_q = nullptr;   // shard: per-row partial sums, stored right behind A
     int ibits = 0, jbits = 0;
     cudaStream_t stream = nullptr;
     cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
@@ -236,6 +241,8 @@ void free_data(dsfacto *h) {
     dev_free(h->d_partials); dev_free(h->d_desc); dev_free(h->d_records); dev_free(h->d_run_count);
     dev_free(h->d_sync);
     h->launch_ptr.clear();
+    h->d_lin = h->d_q = nullptr;
+    h->awaiting_sum = false;
     h->loaded = false;
     h->nnz = 0;
 }
@@ -270,6 +277,7 @@ template <int LG, int NV>
 void launch_refresh(dsfacto *h, const RefreshArgs &a, int mode, int grid) {
     if (mode == kTrain) refresh_kernel<LG, NV, kTrain><<<grid, kThreads, 0, h->stream>>>(a);
     else if (mode == kEvaluate) refresh_kernel<LG, NV, kEvaluate><<<grid, kThreads, 0, h->stream>>>(a);
+    else if (mode == kPartial) refresh_kernel<LG, NV, kPartial><<<grid, kThreads, 0, h->stream>>>(a);
     else refresh_kernel<LG, NV, kScore><<<grid, kThreads, 0, h->stream>>>(a);
 }
 
@@ -534,8 +542,54 @@ void run_sgd_phase(dsfacto *h, int64_t L0, int64_t L1) {
     }
 }
 
+template <int LG, int NV>
+void launch_finish(dsfacto *h, int grid) {
+    finish_kernel<LG, NV><<<grid, kThreads, 0, h->stream>>>(h->n, h->d_A, h->d_lin, h->d_q, h->d_y, h->d_G, h->d_partials,
+                                                            h->w0, h->loss);
+}
+
+// Column shard, first half of the recompute pass: a_i, lin_i, q_i over the shard's own columns.
+int run_partial_refresh(dsfacto *h) {
+    RefreshArgs a{};
+    a.n = h->n; a.indptr = h->d_indptr; a.idx = h->d_idx; a.val = h->d_val; a.y = h->d_y;
+    a.w = h->d_w; a.V = h->d_V; a.A = h->d_A; a.G = h->d_G; a.f_out = nullptr;
+    a.lin_out = h->d_lin; a.q_out = h->d_q;
+    a.partials = h->d_partials; a.w0 = h->w0; a.loss = h->loss;
+    DSF_DISPATCH_REFRESH(h, h, a, kPartial, h->refresh_grid);
+    h->launches += 1;
+    cudaEventRecord(h->ev[2], h->stream);   // (the epoch's phase timers expect both marks)
+    cudaEventRecord(h->ev[3], h->stream);
+    CU_TRY(h, cudaStreamSynchronize(h->stream));
+    CU_TRY(h, cudaGetLastError());
+    h->awaiting_sum = true;
+    return DSFACTO_OK;
+}
+
+// Column shard, second half: the totals [A | lin | q] are in place; f, loss, G, the two sums, and the squared
+// norms of the shard's own columns.
+int run_finish(dsfacto *h) {
+    DSF_DISPATCH(h, launch_finish, h, h->refresh_grid);
+    reduce2_kernel<<<1, kThreads, 0, h->stream>>>(h->d_partials, h->refresh_grid, h->d_scal);
+    double *np = h->d_partials + 2 * (size_t)h->refresh_grid;
+    const int64_t cols = h->col_hi - h->col_lo;
+    sqnorm_kernel<<<h->norm_grid, kThreads, 0, h->stream>>>(h->d_w + h->col_lo, cols, h->d_V + (size_t)h->col_lo * h->Kp,
+                                                            cols * h->Kp, np);
+    reduce2_kernel<<<1, kThreads, 0, h->stream>>>(np, h->norm_grid, h->d_scal + 2);
+    h->launches += 4;
+    double s[4];
+    CU_TRY(h, cudaMemcpyAsync(s, h->d_scal, sizeof s, cudaMemcpyDeviceToHost, h->stream));
+    CU_TRY(h, cudaStreamSynchronize(h->stream));
+    CU_TRY(h, cudaGetLastError());
+    h->loss_sum = s[0]; h->g_sum = s[1]; h->w2 = s[2]; h->v2 = s[3];
+    // the regulariser share of the other shards is missing here: the caller adds the shares up
+    h->objective = s[0] / (double)h->n + 0.5 * (double)h->lambda_w * s[2] + 0.5 * (double)h->lambda_v * s[3];
+    h->awaiting_sum = false;
+    return DSFACTO_OK;
+}
+
 // recompute pass + norms + objective; ends with a stream sync and the four sums on the host
 int run_refresh(dsfacto *h, bool timed) {
+    if (h->nshards > 1) return run_partial_refresh(h);
     RefreshArgs a{};
     a.n = h->n; a.indptr = h->d_indptr; a.idx = h->d_idx; a.val = h->d_val; a.y = h->d_y;
     a.w = h->d_w; a.V = h->d_V; a.A = h->d_A; a.G = h->d_G; a.f_out = nullptr;
@@ -998,10 +1052,11 @@ const char *dsfacto_strerror(int status) {
 
 const char *dsfacto_last_error(dsfacto_t *h) { return h ? h->err.c_str() : ""; }
 
-int dsfacto_create(dsfacto_t **out, int64_t n, int32_t d, int32_t K, int32_t p, int32_t loss, float lambda_w,
-                   float lambda_v, float eta, uint64_t seed) {
+static int create_handle(dsfacto_t **out, int64_t n, int32_t d, int32_t K, int32_t p, int32_t loss, float lambda_w,
+                         float lambda_v, float eta, uint64_t seed, int32_t shard, int32_t nshards) {
     if (!out) return DSFACTO_ERR_INVALID_ARG;
     *out = nullptr;
+    if (nshards < 1 || shard < 0 || shard >= nshards || nshards > p) return DSFACTO_ERR_INVALID_ARG;
     if (n < 1 || n >= ((int64_t)1 << 31) || d < 1 || K < 1 || K > 256 || p < 1 || p > 4096) return DSFACTO_ERR_INVALID_ARG;
     if (loss != DSFACTO_SQUARED && loss != DSFACTO_LOGISTIC) return DSFACTO_ERR_INVALID_ARG;
     if (!(lambda_w >= 0.f) || !(lambda_v >= 0.f) || !(eta > 0.f) || !std::isfinite(lambda_w) ||
@@ -1037,6 +1092,11 @@ int dsfacto_create(dsfacto_t **out, int64_t n, int32_t d, int32_t K, int32_t p, 
 
     auto fail = [&](int rc) { dsfacto_destroy(h); return rc; };
     if (setup_partition(h)) return fail(DSFACTO_ERR_OOM);
+    h->shard = shard; h->nshards = nshards;
+    h->cb_lo = (int32_t)(((int64_t)shard * p) / nshards);
+    h->cb_hi = (int32_t)(((int64_t)(shard + 1) * p) / nshards);
+    h->col_lo = h->col_start[(size_t)h->cb_lo];
+    h->col_hi = h->col_start[(size_t)h->cb_hi];
 
     for (auto &e : h->ev)
         if (cudaEventCreate(&e) != cudaSuccess) return fail(DSFACTO_ERR_CUDA);
@@ -1073,6 +1133,23 @@ int dsfacto_create(dsfacto_t **out, int64_t n, int32_t d, int32_t K, int32_t p, 
     return DSFACTO_OK;
 }
 
+int dsfacto_create(dsfacto_t **out, int64_t n, int32_t d, int32_t K, int32_t p, int32_t loss, float lambda_w,
+                   float lambda_v, float eta, uint64_t seed) {
+    return create_handle(out, n, d, K, p, loss, lambda_w, lambda_v, eta, seed, 0, 1);
+}
+
+int dsfacto_create_shard(dsfacto_t **out, int64_t n, int32_t d, int32_t K, int32_t p, int32_t loss, float lambda_w,
+                         float lambda_v, float eta, uint64_t seed, int32_t shard, int32_t nshards) {
+    return create_handle(out, n, d, K, p, loss, lambda_w, lambda_v, eta, seed, shard, nshards);
+}
+
+int dsfacto_shard_columns(dsfacto_t *h, int32_t *col_lo, int32_t *col_hi) {
+    if (!h) return DSFACTO_ERR_INVALID_ARG;
+    if (col_lo) *col_lo = h->col_lo;
+    if (col_hi) *col_hi = h->col_hi;
+    return DSFACTO_OK;
+}
+
 void dsfacto_destroy(dsfacto_t *h) {
     if (!h) return;
     cudaStreamSynchronize(h->stream);
@@ -1090,6 +1167,34 @@ int dsfacto_set_stream(dsfacto_t *h, void *cuda_stream) {
     return DSFACTO_OK;
 }
 
+// entries of columns [lo, hi) only, as a CSR over the same rows
+static int filter_columns(int64_t n, const int64_t *indptr, const int32_t *indices, const float *values, int32_t lo, int32_t hi,
+                          HostBuf<int64_t> &f_indptr, HostBuf<int32_t> &f_indices, HostBuf<float> &f_values) {
+    if (!f_indptr.alloc((size_t)n + 1)) return DSFACTO_ERR_OOM;
+    int64_t *fp = f_indptr.data();
+    fp[0] = 0;
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < n; ++i) {
+        int64_t cnt = 0;
+        for (int64_t t = indptr[i]; t < indptr[i + 1]; ++t) cnt += (indices[t] >= lo && indices[t] < hi) ? 1 : 0;
+        fp[i + 1] = cnt;
+    }
+    for (int64_t i = 0; i < n; ++i) fp[i + 1] += fp[i];
+    const int64_t kept = fp[n];
+    if (!f_indices.alloc((size_t)std::max<int64_t>(kept, 1)) || !f_values.alloc((size_t)std::max<int64_t>(kept, 1))) return DSFACTO_ERR_OOM;
+    int32_t *fi = f_indices.data();
+    float *fv = f_values.data();
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < n; ++i) {
+        int64_t at = fp[i];
+        for (int64_t t = indptr[i]; t < indptr[i + 1]; ++t)
+            if (indices[t] >= lo && indices[t] < hi) { fi[at] = indices[t]; fv[at] = values[t]; ++at; }
+    }
+    return DSFACTO_OK;
+}
+
+static int load_validated(dsfacto_t *h, const int64_t *indptr, const int32_t *indices, const float *values, const float *y);
+
 int dsfacto_load_csr(dsfacto_t *h, const int64_t *indptr, const int32_t *indices, const float *values, const float *y) {
     if (!h || !indptr || !y) return DSFACTO_ERR_INVALID_ARG;
     const int64_t n = h->n;
@@ -1104,6 +1209,21 @@ int dsfacto_load_csr(dsfacto_t *h, const int64_t *indptr, const int32_t *indices
         if (!std::isfinite(y[i])) bad |= 1;
     if (bad) return DSFACTO_ERR_INVALID_CSR;
 
+    // a column shard keeps only the stored entries of its own columns (all rows stay, some become empty)
+    HostBuf<int64_t> f_indptr;
+    HostBuf<int32_t> f_indices;
+    HostBuf<float> f_values;
+    if (h->nshards > 1) {
+        rc = filter_columns(n, indptr, indices, values, h->col_lo, h->col_hi, f_indptr, f_indices, f_values);
+        if (rc) return rc;
+        indptr = f_indptr.data(); indices = f_indices.data(); values = f_values.data();
+    }
+    return load_validated(h, indptr, indices, values, y);
+}
+
+static int load_validated(dsfacto_t *h, const int64_t *indptr, const int32_t *indices, const float *values, const float *y) {
+    const int64_t n = h->n, nnz = indptr[n];
+    int rc = DSFACTO_OK;
     CU_TRY(h, cudaStreamSynchronize(h->stream));
     free_data(h);
     h->nnz = nnz;
@@ -1151,7 +1271,7 @@ int dsfacto_load_csr(dsfacto_t *h, const int64_t *indptr, const int32_t *indices
         if (rc) { cudaStreamSynchronize(st); free_data(h); return rc; }
     }
     h->nnz = nnz;   // (free_data on an error path above resets it)
-    if ((rc = dev_alloc(h, &h->d_A, (size_t)n * h->Kp)) || (rc = dev_alloc(h, &h->d_G, (size_t)n)) ||
+    if ((rc = dev_alloc(h, &h->d_A, (size_t)n * h->Kp + (h->nshards > 1 ? 2 * (size_t)n : 0))) || (rc = dev_alloc(h, &h->d_G, (size_t)n)) ||
         (rc = dev_alloc(h, &h->d_tile_ptr, h->tile_ptr.size())) || (rc = dev_alloc(h, &h->d_ent, cnt + 4)) ||
         (rc = dev_alloc(h, &h->d_partials, 2 * ((size_t)h->refresh_grid + (size_t)h->norm_grid))) ||
         (h->wide && (rc = dev_alloc(h, &h->d_xw, cnt + 4)))) {
@@ -1179,8 +1299,13 @@ int dsfacto_load_csr(dsfacto_t *h, const int64_t *indptr, const int32_t *indices
     if ((rc = finish_sgd_plan(h, pb))) { free_data(h); return rc; }
     h->failed = false;
     h->loaded = true;
+    if (h->nshards > 1) {   // the partial sums sit right behind A, so that one buffer holds what the shards exchange
+        h->d_lin = h->d_A + (size_t)n * h->Kp;
+        h->d_q = h->d_lin + n;
+    }
     rc = run_refresh(h, false);
     if (rc) return rc;
+    if (h->nshards > 1) return DSFACTO_OK;   // no objective before the shards' partial sums have been added up
     return std::isfinite(h->objective) ? DSFACTO_OK : DSFACTO_ERR_DIVERGED;
 }
 
@@ -1208,10 +1333,17 @@ static int sgd_gave_up(dsfacto *h, const int code[3]) {
     return DSFACTO_ERR_CUDA;
 }
 
+static int epoch_impl(dsfacto_t *h);
+
 int dsfacto_epoch(dsfacto_t *h) {
     if (!h) return DSFACTO_ERR_INVALID_ARG;
     if (!h->loaded) return DSFACTO_ERR_NO_DATA;
     if (h->failed) { h->err = "the last stratum SGD launch gave up: set the parameters again (dsfacto_set_params) first"; return DSFACTO_ERR_CUDA; }
+    if (h->nshards > 1) return DSFACTO_ERR_INVALID_ARG;   // a column shard advances with dsfacto_shard_epoch_begin / _end
+    return epoch_impl(h);
+}
+
+static int epoch_impl(dsfacto_t *h) {
     cudaStream_t st = h->stream;
     CU_TRY(h, cudaEventRecord(h->ev[0], st));
     const int64_t p = h->p;
@@ -1237,12 +1369,68 @@ int dsfacto_epoch(dsfacto_t *h) {
     CU_TRY(h, cudaMemcpy(sgd_error, h->d_sync + kSyncError, sizeof sgd_error, cudaMemcpyDeviceToHost));
     if (sgd_error[0]) return sgd_gave_up(h, sgd_error);
     h->ms[0] = t01 + t12 + t23; h->ms[1] = t01; h->ms[2] = t12; h->ms[3] = t23;
+    if (h->nshards > 1) return DSFACTO_OK;   // the objective exists only after the shards' sums have been added up
     return std::isfinite(h->objective) ? DSFACTO_OK : DSFACTO_ERR_DIVERGED;
+}
+
+// ---- column shards ----
+int dsfacto_shard_partial_count(dsfacto_t *h, int64_t *count) {
+    if (!h || !count) return DSFACTO_ERR_INVALID_ARG;
+    *count = h->n * ((int64_t)h->Kp + 2);
+    return DSFACTO_OK;
+}
+
+int dsfacto_shard_epoch_begin(dsfacto_t *h) {
+    if (!h) return DSFACTO_ERR_INVALID_ARG;
+    if (h->nshards < 2) return DSFACTO_ERR_INVALID_ARG;
+    if (!h->loaded) return DSFACTO_ERR_NO_DATA;
+    if (h->awaiting_sum) { h->err = "the summed auxiliaries of the last step have not been handed in (dsfacto_shard_epoch_end)"; return DSFACTO_ERR_INVALID_ARG; }
+    return epoch_impl(h);   // w0 step, the strata over the shard's own tiles, then the partial recompute pass
+}
+
+int dsfacto_shard_partial(dsfacto_t *h, float *dst_dev, int64_t count) {
+    if (!h || !dst_dev) return DSFACTO_ERR_INVALID_ARG;
+    if (h->nshards < 2 || !h->loaded) return DSFACTO_ERR_INVALID_ARG;
+    if (count != h->n * ((int64_t)h->Kp + 2)) return DSFACTO_ERR_INVALID_ARG;
+    CU_TRY(h, cudaMemcpyAsync(dst_dev, h->d_A, sizeof(float) * (size_t)count, cudaMemcpyDeviceToDevice, h->stream));
+    CU_TRY(h, cudaStreamSynchronize(h->stream));
+    return DSFACTO_OK;
+}
+
+int dsfacto_shard_epoch_end(dsfacto_t *h, const float *summed_dev, int64_t count, double sums[4]) {
+    if (!h || !summed_dev || !sums) return DSFACTO_ERR_INVALID_ARG;
+    if (h->nshards < 2 || !h->loaded) return DSFACTO_ERR_INVALID_ARG;
+    if (count != h->n * ((int64_t)h->Kp + 2)) return DSFACTO_ERR_INVALID_ARG;
+    CU_TRY(h, cudaMemcpyAsync(h->d_A, summed_dev, sizeof(float) * (size_t)count, cudaMemcpyDeviceToDevice, h->stream));
+    const int rc = run_finish(h);
+    if (rc) return rc;
+    sums[0] = h->loss_sum; sums[1] = h->g_sum; sums[2] = h->w2; sums[3] = h->v2;
+    return DSFACTO_OK;
+}
+
+int dsfacto_bucket_host_shard(int64_t n, int32_t d, int32_t p, int32_t shard, int32_t nshards, const int64_t *indptr,
+                              const int32_t *indices, const float *values, int64_t *kept, int64_t *tile_ptr, int32_t *rows,
+                              int32_t *cols, float *vals) {
+    if (n < 1 || n >= ((int64_t)1 << 31) || d < 1 || p < 1 || p > 4096 || !indptr || !tile_ptr || !kept) return DSFACTO_ERR_INVALID_ARG;
+    if (nshards < 1 || shard < 0 || shard >= nshards || nshards > p) return DSFACTO_ERR_INVALID_ARG;
+    if (indptr[0] != 0 || indptr[n] < 0) return DSFACTO_ERR_INVALID_CSR;
+    if (indptr[n] > 0 && (!indices || !values)) return DSFACTO_ERR_INVALID_ARG;
+    int rc = validate_csr(n, d, indptr, indices, values);
+    if (rc) return rc;
+    const int32_t lo = (int32_t)(((__int128)(((int64_t)shard * p) / nshards) * d + p - 1) / p);
+    const int32_t hi = (int32_t)(((__int128)(((int64_t)(shard + 1) * p) / nshards) * d + p - 1) / p);
+    HostBuf<int64_t> fp;
+    HostBuf<int32_t> fi;
+    HostBuf<float> fv;
+    if ((rc = filter_columns(n, indptr, indices, values, lo, hi, fp, fi, fv))) return rc;
+    *kept = fp[(size_t)n];
+    return dsfacto_bucket_host(n, d, p, fp.data(), fi.data(), fv.data(), tile_ptr, rows, cols, vals);
 }
 
 int dsfacto_set_refresh_every(dsfacto_t *h, int32_t rounds) {
     if (!h || rounds < 0) return DSFACTO_ERR_INVALID_ARG;
-    if (h->loaded) return DSFACTO_ERR_INVALID_ARG;   // the tile order on the device is fixed by dsfacto_load_csr
+    if (h->loaded) return DSFACTO_ERR_INVALID_ARG;   // the launch plan is fixed by dsfacto_load_csr
+    if (rounds > 0 && h->nshards > 1) return DSFACTO_ERR_INVALID_ARG;   // column shards exchange once per epoch
     h->refresh_every = rounds;   // the launch plan built by dsfacto_load_csr is cut into segments of that many rounds
     return DSFACTO_OK;
 }

@@ -13,8 +13,12 @@ namespace dsf {
 // kEvaluate (held-out rows with labels; the quantities of the convergence figures of Section 5):
 // writes nothing per row, per-CTA fp64 partial sums {sum l_i, sum t_i} with t_i = (f_i - y_i)^2 for
 // the squared loss (RMSE) and t_i = [y_i f_i > 0] for the logistic loss (accuracy).
+// kPartial (a handle that owns only a range of columns, Section 4.2's column blocks spread over
+// workers): the sums run over the handle's own columns, so they are partial; writes a_ik, lin_i and
+// q_i per row and stops there.  The partial sums of all shards are added outside and finish_kernel
+// turns the totals into f_i, l_i and G_i.
 // ------------------------------------------------------------------------------------------
-enum { kScore = 0, kTrain = 1, kEvaluate = 2 };
+enum { kScore = 0, kTrain = 1, kEvaluate = 2, kPartial = 3 };
 struct RefreshArgs {
     int64_t n;
     const int64_t *indptr;
@@ -26,6 +30,7 @@ struct RefreshArgs {
     float *A;
     float *G;
     float *f_out;
+    float *lin_out, *q_out;  // kPartial: per-row partial sums
     double *partials;  // 2 per CTA
     float w0;
     int loss;
@@ -44,6 +49,7 @@ __global__ void __launch_bounds__(kThreads, (LG >= 8 ? 3 : 4)) refresh_kernel(co
     const float4 *V4 = reinterpret_cast<const float4 *>(a.V);
     float4 *A4 = reinterpret_cast<float4 *>(a.A);
     constexpr bool TRAIN = MODE == kTrain;
+    constexpr bool STORE_A = MODE == kTrain || MODE == kPartial;
     double loss_sum = 0.0, g_sum = 0.0;
 
     // The row pointers of the next row are requested while the current row is processed, and its
@@ -117,9 +123,18 @@ __global__ void __launch_bounds__(kThreads, (LG >= 8 ? 3 : 4)) refresh_kernel(co
         float sq = 0.f;
 #pragma unroll
         for (int v = 0; v < NV; ++v) {
-            if (TRAIN) A4[(size_t)row * KP4 + v * LG + l] = acc[v];
+            if (STORE_A) A4[(size_t)row * KP4 + v * LG + l] = acc[v];
             sq = fmaf(acc[v].x, acc[v].x, sq); sq = fmaf(acc[v].y, acc[v].y, sq);
             sq = fmaf(acc[v].z, acc[v].z, sq); sq = fmaf(acc[v].w, acc[v].w, sq);
+        }
+        if (MODE == kPartial) {
+#pragma unroll
+            for (int o = LG / 2; o > 0; o >>= 1) {
+                q += __shfl_xor_sync(gm, q, o, LG);
+                lin += __shfl_xor_sync(gm, lin, o, LG);
+            }
+            if (l == 0) { a.lin_out[row] = lin; a.q_out[row] = q; }
+            continue;
         }
         float pair = sq - q;
 #pragma unroll
@@ -154,12 +169,57 @@ __global__ void __launch_bounds__(kThreads, (LG >= 8 ? 3 : 4)) refresh_kernel(co
             }
         }
     }
-    if (MODE != kScore) {
+    if (MODE != kScore && MODE != kPartial) {
         block_sum2(loss_sum, g_sum);
         if (threadIdx.x == 0) {
             a.partials[2 * blockIdx.x] = loss_sum;
             a.partials[2 * blockIdx.x + 1] = g_sum;
         }
+    }
+}
+
+// Second half of the recompute pass for column shards: from the summed auxiliaries a_i, lin_i, q_i of all
+// shards to f_i = w0 + lin_i + 1/2 (sum_k a_ik^2 - q_i) (eq. (fm_model2)), the loss and the multiplier G_i;
+// per-CTA fp64 partial sums {sum l_i, sum G_i}.  One lane group per row.
+template <int LG, int NV>
+__global__ void __launch_bounds__(kThreads) finish_kernel(int64_t n, const float *A, const float *lin, const float *q,
+                                                          const float *y, float *G, double *partials, float w0, int loss) {
+    constexpr int GR = kThreads / LG;
+    constexpr int KP4 = LG * NV;
+    const int g = threadIdx.x / LG, l = threadIdx.x % LG;
+    const uint32_t gm = group_mask<LG>();
+    const float4 *A4 = reinterpret_cast<const float4 *>(A);
+    double loss_sum = 0.0, g_sum = 0.0;
+    for (int64_t row = (int64_t)blockIdx.x * GR + g; row < n; row += (int64_t)gridDim.x * GR) {
+        float sq = 0.f;
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const float4 x = A4[(size_t)row * KP4 + v * LG + l];
+            sq = fmaf(x.x, x.x, sq); sq = fmaf(x.y, x.y, sq); sq = fmaf(x.z, x.z, sq); sq = fmaf(x.w, x.w, sq);
+        }
+#pragma unroll
+        for (int o = LG / 2; o > 0; o >>= 1) sq += __shfl_xor_sync(gm, sq, o, LG);
+        if (l == 0) {
+            const float f = w0 + lin[row] + 0.5f * (sq - q[row]);
+            const float yy = y[row];
+            float li, gi;
+            if (loss == 0) {
+                gi = f - yy;
+                li = 0.5f * gi * gi;
+            } else {
+                const float m = yy * f;
+                li = fmaxf(-m, 0.f) + log1pf(expf(-fabsf(m)));
+                gi = -yy / (1.f + expf(m));
+            }
+            G[row] = gi;
+            loss_sum += (double)li;
+            g_sum += (double)gi;
+        }
+    }
+    block_sum2(loss_sum, g_sum);
+    if (threadIdx.x == 0) {
+        partials[2 * blockIdx.x] = loss_sum;
+        partials[2 * blockIdx.x + 1] = g_sum;
     }
 }
 

@@ -39,6 +39,15 @@ SIGNATURES = {
     "dsfacto_set_stream": (ctypes.c_int, [_vp, _vp]),
     "dsfacto_last_epoch_ms": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_float)]),
     "dsfacto_debug_set": (ctypes.c_int, [_vp, _c_i32, _c_i64]),
+    "dsfacto_create_shard": (ctypes.c_int, [ctypes.POINTER(_vp), _c_i64, _c_i32, _c_i32, _c_i32, _c_i32, _c_f32, _c_f32,
+                                            _c_f32, _c_u64, _c_i32, _c_i32]),
+    "dsfacto_shard_columns": (ctypes.c_int, [_vp, ctypes.POINTER(_c_i32), ctypes.POINTER(_c_i32)]),
+    "dsfacto_shard_partial_count": (ctypes.c_int, [_vp, ctypes.POINTER(_c_i64)]),
+    "dsfacto_shard_epoch_begin": (ctypes.c_int, [_vp]),
+    "dsfacto_shard_partial": (ctypes.c_int, [_vp, _vp, _c_i64]),
+    "dsfacto_shard_epoch_end": (ctypes.c_int, [_vp, _vp, _c_i64, ctypes.POINTER(ctypes.c_double)]),
+    "dsfacto_bucket_host_shard": (ctypes.c_int, [_c_i64, _c_i32, _c_i32, _c_i32, _c_i32, _vp, _vp, _vp,
+                                                 ctypes.POINTER(_c_i64), _vp, _vp, _vp, _vp]),
     "dsfacto_launch_count": (ctypes.c_int, [_vp, ctypes.POINTER(_c_i64)]),
     "dsfacto_last_error": (ctypes.c_char_p, [_vp]),
     "dsfacto_strerror": (ctypes.c_char_p, [ctypes.c_int]),
@@ -162,6 +171,20 @@ def dsfacto_bucket_host(n, d, p, indptr, indices, values):
     return rc, tile_ptr, rows, cols, vals
 
 
+def dsfacto_bucket_host_shard(n, d, p, shard, nshards, indptr, indices, values):
+    """Host tile bucketer of one column shard -> (status, kept, tile_ptr, rows, cols, vals); needs no GPU."""
+    nnz = int(indptr[-1])
+    tile_ptr = np.zeros(p * p + 1, np.int64)
+    rows = np.empty(max(nnz, 1), np.int32)
+    cols = np.empty(max(nnz, 1), np.int32)
+    vals = np.empty(max(nnz, 1), np.float32)
+    kept = _c_i64()
+    rc = lib().dsfacto_bucket_host_shard(n, d, p, shard, nshards, _ptr(indptr), _ptr(indices), _ptr(values),
+                                         ctypes.byref(kept), _ptr(tile_ptr), _ptr(rows), _ptr(cols), _ptr(vals))
+    k = int(kept.value)
+    return rc, k, tile_ptr, rows[:k], cols[:k], vals[:k]
+
+
 def dsfacto_score_loss_noalloc(m, d, K, loss, indptr_dev, indices_dev, values_dev, y_dev, w0, w_dev, V_dev,
                                scores_dev, sums_dev, cuda_stream=0):
     """Allocation-free scoring; every *_dev argument is a raw device address (int)."""
@@ -173,14 +196,44 @@ def dsfacto_score_loss_noalloc(m, d, K, loss, indptr_dev, indices_dev, values_de
 class DSFacto:
     """Convenience owner of one handle.  Every method is one C call plus array allocation."""
 
-    def __init__(self, n, d, K, p, loss, lambda_w, lambda_v, eta, seed):
+    def __init__(self, n, d, K, p, loss, lambda_w, lambda_v, eta, seed, shard=0, nshards=1):
         self.n, self.d, self.K, self.p = int(n), int(d), int(K), int(p)
-        rc, self._h = dsfacto_create(self.n, self.d, self.K, self.p, int(loss), float(lambda_w), float(lambda_v),
-                                     float(eta), int(seed))
+        self.shard, self.nshards = int(shard), int(nshards)
+        if self.nshards == 1:
+            rc, self._h = dsfacto_create(self.n, self.d, self.K, self.p, int(loss), float(lambda_w), float(lambda_v),
+                                         float(eta), int(seed))
+        else:
+            self._h = _vp()
+            rc = lib().dsfacto_create_shard(ctypes.byref(self._h), self.n, self.d, self.K, self.p, int(loss),
+                                            float(lambda_w), float(lambda_v), float(eta), int(seed), self.shard,
+                                            self.nshards)
         if rc != OK:
             self._h = None
             raise DSFactoError(rc, "dsfacto_create")
         self.nnz = 0
+
+    # ---- column shards (see include/dsfacto.h) ----
+    def shard_columns(self):
+        lo, hi = _c_i32(), _c_i32()
+        self._check(lib().dsfacto_shard_columns(self._h, ctypes.byref(lo), ctypes.byref(hi)), "dsfacto_shard_columns")
+        return int(lo.value), int(hi.value)
+
+    def shard_partial_count(self) -> int:
+        c = _c_i64()
+        self._check(lib().dsfacto_shard_partial_count(self._h, ctypes.byref(c)), "dsfacto_shard_partial_count")
+        return int(c.value)
+
+    def shard_epoch_begin(self):
+        self._check(lib().dsfacto_shard_epoch_begin(self._h), "dsfacto_shard_epoch_begin")
+
+    def shard_partial(self, dst_dev_ptr: int, count: int):
+        self._check(lib().dsfacto_shard_partial(self._h, ctypes.c_void_p(dst_dev_ptr), count), "dsfacto_shard_partial")
+
+    def shard_epoch_end(self, summed_dev_ptr: int, count: int):
+        sums = (ctypes.c_double * 4)()
+        self._check(lib().dsfacto_shard_epoch_end(self._h, ctypes.c_void_p(summed_dev_ptr), count, sums),
+                    "dsfacto_shard_epoch_end")
+        return [float(x) for x in sums]
 
     def _check(self, rc, where):
         if rc != OK:
@@ -214,6 +267,9 @@ class DSFacto:
             raise ValueError("indices/values shorter than indptr[-1]")
         self._check(dsfacto_load_csr(self._h, indptr, indices, values, y), "dsfacto_load_csr")
         self.nnz = int(indptr[-1])
+        if self.nshards > 1:   # a shard keeps the entries of its own columns only
+            lo, hi = self.shard_columns()
+            self.nnz = int(np.count_nonzero((indices[: self.nnz] >= lo) & (indices[: self.nnz] < hi)))
 
     def epoch(self) -> float:
         self._check(dsfacto_epoch(self._h), "dsfacto_epoch")
