@@ -166,7 +166,7 @@ int dsfacto_set_stream(dsfacto_t *h, void *cuda_stream);
 int dsfacto_last_epoch_ms(dsfacto_t *h, float ms[4]);
 
 /* Test and debugging knobs of the stratum SGD launch.
- *   DSFACTO_DEBUG_SPIN_LIMIT  polls (about 100 ns each, 1 .. 2^22, default 2^22) after which a wait for an
+ *   DSFACTO_DEBUG_SPIN_LIMIT  polls (a few hundred ns each, 1 .. 2^22, default 2^22) after which a wait for an
  *                             earlier tile of the same column block gives up; dsfacto_epoch then returns
  *                             DSFACTO_ERR_CUDA and the handle refuses further epochs until dsfacto_set_params
  *                             replaces w and V or dsfacto_load_csr loads a data set.

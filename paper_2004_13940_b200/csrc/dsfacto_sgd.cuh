@@ -13,12 +13,14 @@
 // product over m entries is (1 - ew)^m and only the count m is carried.
 //
 // During the SGD phase the column state is held in scaled form, v_j = (1 + sigma_j) u_j and
-// w_j = (1 - ew)^{m_j} uw_j with sigma_j = 0, m_j = 0 at the start of the phase.  Applying a run of
-// entries with local sums U = sum_t (b_t / P_t) a_i, W = sum_t b_t (1 - ew)^{-t}, product D and
-// length m is then
-//     u_j += U / (1 + sigma_j),  uw_j += W (1 - ew)^{-m_j},  sigma_j <- sigma_j + D + sigma_j D,  m_j += m:
-// the K-wide part is an add that nobody waits for (red.global.add; every column receives at most one
-// per tile and tiles of a column block are ordered, so the result does not depend on timing).
+// w_j = (1 - ew)^{m_j} uw_j with sigma_j = 0, m_j = 0 at the start of the phase.  A run of entries of
+// column j starts its products from the column's own scale, P_0 = 1 + sigma_j and m_0 = m_j, so its sums
+// U = sum_t (b_t / P_t) a_i and W = sum_t b_t (1 - ew)^{-m_t} need no scaling when they are applied:
+//     u_j += U,  uw_j += W,  sigma_j <- P_T - 1,  m_j <- m_T.
+// The K-wide part is an add that nobody waits for (red.global.add; every column receives at most one
+// per tile and tiles of a column block are ordered, so the result does not depend on timing).  A slice of
+// a run that is longer than a chunk cannot know the column's scale yet; it starts from P_0 = 1, m_0 = 0, and
+// the slice that joins the run's slices scales the joined sums by 1 / (1 + sigma_j) and (1 - ew)^{-m_j}.
 // sgd_finalize_* turns the state back into plain (w, V) at the end of the phase.  The scaled form
 // breaks down only if some 1 + sigma reaches zero, i.e. a step so large that a run wipes its column;
 // the parameters then become non-finite and the epoch reports divergence.
@@ -30,7 +32,7 @@ namespace dsf {
 constexpr int kSgdWarps = 1;                      // warps per CTA; every warp works on its own chunks
 constexpr int kSgdThreads = 32 * kSgdWarps;
 constexpr int kChunkMax = 512;                    // most entries a chunk may hold
-constexpr int kSgdSpinLimit = 1 << 22;            // polls (about 100 ns each) before a dependency wait gives up
+constexpr int kSgdSpinLimit = 1 << 22;            // polls (200 ns of sleep plus a read from L2 each) before a dependency wait gives up
 constexpr int kCopySpinLimit = 1 << 24;           // polls before the wait for a bulk copy into shared memory gives up
 constexpr int kTicketStop = 0x40000000;           // ticket counter value that makes every warp leave
 // Words of the launch's synchronisation array.  The ticket counter takes one atomic per chunk and the
@@ -90,10 +92,6 @@ __host__ __device__ constexpr int slice_record_floats(int Kp) { return 4 + Kp; }
 __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src) {
     const unsigned s = (unsigned)__cvta_generic_to_shared(smem_dst);
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem_src) : "memory");
-}
-__device__ __forceinline__ void cp_async4(void *smem_dst, const void *gmem_src) {
-    const unsigned s = (unsigned)__cvta_generic_to_shared(smem_dst);
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"(s), "l"(gmem_src) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N>
@@ -196,16 +194,16 @@ struct SgdArgs {
 // ------------------------------------------------------------------------------------------
 // sgd_sweep_kernel: persistent warps; each takes chunks in sweep order from a ticket counter.
 //
-// Pipeline of a warp: the ticket of chunk n+2, the descriptor of chunk n+1 and the entry records of
-// chunk n+1 (one bulk copy into shared memory, completion on an mbarrier) are under way while chunk
-// n is worked on.  A chunk is walked in passes of 32 entries, one entry per lane for the scalar
+// Pipeline of a warp: while chunk n is worked on, the ticket of chunk n+1 is drawn, its descriptor is
+// loaded and its entry records are copied into shared memory (one bulk copy, completion on an
+// mbarrier).  A chunk is walked in passes of 32 entries, one entry per lane for the scalar
 // part:
 //   scalar stage   G_i (requested one pass ahead) -> e, b; run boundaries by comparing neighbours;
 //                  segmented scan of D = P - 1 over the lanes; coefficient c = b / P and the w
 //                  coefficient; for every run that starts in the pass the scale record of its column
 //                  (requested one pass ahead).  Results go to shared memory.
 //   K-wide stage   the rows a_i of a stage (32 rows for K <= 32, fewer for wider rows; gathered with
-//                  cp.async one or two stages ahead) are added with weight c.  The run that is open at
+//                  cp.async one stage ahead) are added with weight c.  The run that is open at
 //                  the start of a stage and the run that is open at its end are spread over all lane
 //                  groups (entry u goes to group u mod GW) and the groups keep their partial sums in
 //                  registers until the run ends, then a shuffle tree joins them; runs that start and
@@ -214,8 +212,10 @@ struct SgdArgs {
 // slice of the run that finishes last joins the records in order (scalar prefix products first, then a
 // weighted sum of the K-wide parts) and applies the run.
 //
-// Order: a tile may touch column state only after the earlier tiles of its column block are done (one
-// counter per column block, bumped by the chunk that finishes a tile, after a fence).  Tickets are
+// Order: a tile may touch column state only after the earlier tiles of its column block are done: one
+// counter per column block counts finished chunks (after a fence), and a chunk waits until it has
+// reached the number of chunks of the earlier tiles.  Slices do not wait, so they are counted only by
+// the slice that joins their run, all at once, after the run has been applied.  Tickets are
 // handed out in sweep order, so every chunk a warp may wait for is already held by a warp that is
 // running: no deadlock, and no reliance on the order in which CTAs start.  The wait is bounded all
 // the same; when it runs out the error word is set, the ticket counter jumps past the end, and every
