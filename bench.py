@@ -222,6 +222,8 @@ def run_ours(args):
 
     t_gen = time.perf_counter()
     wl = W.make(args.workload, n=args.rows, p=args.p, empty=pinned_empty)
+    if args.K is not None:
+        wl.K = int(args.K)
     t_gen = time.perf_counter() - t_gen
     nnz = wl.nnz
     stream = torch.cuda.current_stream()
@@ -359,6 +361,7 @@ def main():
     ap.add_argument("--workload", default="C4")
     ap.add_argument("--rows", type=int, default=None, help="override the workload's row count (profiling)")
     ap.add_argument("--p", type=int, default=None, help="override the tile grid (profiling)")
+    ap.add_argument("--K", type=int, default=None, help="override the number of factors (profiling)")
     ap.add_argument("--refresh-every", type=int, default=0,
                     help="second schedule: recompute G, A after every R inner rounds (0: once per epoch)")
     ap.add_argument("--e2e-steps", type=int, default=3)

@@ -71,8 +71,12 @@ template <int LG, int NV>
 struct SgdCfg {
     static constexpr int GW = 32 / LG;               // lane groups per warp = rows worked on side by side
     static constexpr int KP4 = LG * NV;              // float4s per factor row
-    // rows of A gathered per stage: a whole pass for rows up to 128 bytes, at most 4 KB for wider rows
-    static constexpr int RST = KP4 <= 8 ? 32 : (KP4 <= 16 ? 16 : (KP4 <= 32 ? 8 : 4));
+    // rows of A gathered per stage: a whole pass for rows up to 128 bytes, half a pass for wider rows.  A
+    // stage has a fixed cost (commit, wait, two warp barriers, the masks of its run starts), so short stages
+    // are expensive: on the 400 M-entry workload with 512-byte rows a sweep takes 97 ms with 4-row stages,
+    // 42 ms with 8, 26 ms with 16 and 34 ms with 32 (too few resident warps); 1024-byte rows 42 ms with 8,
+    // 29 ms with 16; 256-byte rows 16 ms with 16, 20 ms with 32.
+    static constexpr int RST = KP4 <= 8 ? 32 : 16;
     static constexpr int SP = 32 / RST;              // stages per 32-entry pass
     static constexpr int NBUF = 2;                   // stages in the ring (three were no faster on any workload)
     static constexpr int PD = NBUF - 1;              // stages requested ahead
