@@ -176,9 +176,16 @@ int dsfacto_last_epoch_ms(dsfacto_t *h, float ms[4]);
  *                             failure path above can be exercised without a fault or a hang.  0 = off.
  *   DSFACTO_DEBUG_CHUNK_LEN   (takes effect at the next dsfacto_load_csr) entries per chunk, 16 .. 512, 0 = chosen
  *                             by the load; the environment variable DSFACTO_CHUNK does the same for every handle.
+ *   DSFACTO_DEBUG_COLUMN_ORDER (takes effect at the next dsfacto_load_csr) the device copy of the CSR that the
+ *                             recompute pass reads may number the columns by frequency, most frequent first, and
+ *                             the pass then reads w and V from a copy in that order (hot factor rows side by
+ *                             side in the caches; no sum changes).  0 = decided by the load (on from 2^22 stored
+ *                             entries and 1 MB of factors), 1 = always, 2 = never; the environment variable
+ *                             DSFACTO_COLUMN_ORDER=0/1 does the same for every handle.  Nothing a caller passes
+ *                             or receives is renumbered.
  * The environment variable DSFACTO_SWEEP=round (read by dsfacto_create) stores and sweeps the tiles round by
  * round, exactly Algorithm 1's order, instead of row block by row block. */
-enum { DSFACTO_DEBUG_SPIN_LIMIT = 0, DSFACTO_DEBUG_EXTRA_NEED = 1, DSFACTO_DEBUG_CHUNK_LEN = 2 };
+enum { DSFACTO_DEBUG_SPIN_LIMIT = 0, DSFACTO_DEBUG_EXTRA_NEED = 1, DSFACTO_DEBUG_CHUNK_LEN = 2, DSFACTO_DEBUG_COLUMN_ORDER = 3 };
 int dsfacto_debug_set(dsfacto_t *h, int32_t key, int64_t value);
 
 /* Number of kernels this handle has launched since creation. */

@@ -73,6 +73,17 @@ struct dsfacto {
     float4 *d_S = nullptr, *d_TS = nullptr;  // scale records of the scaled column state (zero outside the SGD phase)
     int *d_run_count = nullptr;
     int refresh_grid = 0, norm_grid = 0;
+    // Column slots of the recompute pass (per load): the device CSR holds slots (rank by frequency) instead of
+    // column indices, and the pass reads w and V from copies in slot order.
+    int column_order = 0;       // dsfacto_debug_set: 0 = decided per load, 1 = always, 2 = never
+    bool slots = false;
+    int32_t *d_column_of = nullptr;
+    float *d_Vs = nullptr;
+    // What the recompute pass reads beside V: per column (w_j, sum_k v_jk^2), by column index (d_pair) and, for
+    // the renumbered device CSR, by slot (d_pair_s, with d_Vs).  Each is rebuilt when the parameters have
+    // changed since it was made (model_version counts the changes).
+    float2 *d_pair = nullptr, *d_pair_s = nullptr;
+    int64_t model_version = 1, pair_version = 0, slot_version = 0;
 
     double loss_sum = 0, g_sum = 0, w2 = 0, v2 = 0, objective = 0;
 };
@@ -239,7 +250,9 @@ void free_data(dsfacto *h) {
     dev_free(h->d_A); dev_free(h->d_G); dev_free(h->d_y); dev_free(h->d_val); dev_free(h->d_xw);
     dev_free(h->d_indptr); dev_free(h->d_tile_ptr); dev_free(h->d_idx); dev_free(h->d_ent);
     dev_free(h->d_partials); dev_free(h->d_desc); dev_free(h->d_records); dev_free(h->d_run_count);
-    dev_free(h->d_sync);
+    dev_free(h->d_sync); dev_free(h->d_column_of); dev_free(h->d_Vs); dev_free(h->d_pair_s);
+    h->slots = false;
+    h->slot_version = 0;
     h->launch_ptr.clear();
     h->d_lin = h->d_q = nullptr;
     h->awaiting_sum = false;
@@ -507,6 +520,7 @@ int finish_sgd_plan(dsfacto *h, SgdPlanBuild &pb) {
 // The strata [L0, L1) of one epoch (inner rounds for the round sweep, row blocks for the row-block
 // sweep; the whole sweep is [0, p)), then the return from the scaled state to plain parameters.
 void run_sgd_phase(dsfacto *h, int64_t L0, int64_t L1) {
+    h->model_version += 1;   // w and V change: the views of the recompute pass are out of date
     SgdArgs a{};
     a.ent = h->d_ent; a.xw = h->d_xw; a.A = h->d_A; a.G = h->d_G; a.w = h->d_w; a.V = h->d_V;
     a.S = h->d_S; a.Tb = h->d_Tb; a.Tw = h->d_Tw; a.TS = h->d_TS; a.records = h->d_records;
@@ -548,11 +562,91 @@ void launch_finish(dsfacto *h, int grid) {
                                                             h->w0, h->loss);
 }
 
+// V and the pairs (w_j, s_j) as the recompute pass reads them: by slot for the training rows when the load
+// renumbered the columns of the device CSR, by column index otherwise (and always for rows a caller passes).
+// Rebuilt only when the parameters changed since the last time: one pass over V (4 d Kp bytes read, twice
+// that with the copy in slot order; tens of microseconds).
+void model_view(dsfacto *h, RefreshArgs &a, bool training_rows) {
+    const bool by_slot = training_rows && h->slots;
+    int64_t &version = by_slot ? h->slot_version : h->pair_version;
+    if (version != h->model_version) {
+        const int kp4 = h->Kp / 4;
+        int gs = 1;
+        while (gs < kp4 && gs < 32) gs *= 2;
+        const int64_t groups_per_cta = kThreads / gs;
+        const int grid = (int)std::min<int64_t>(((int64_t)h->d + groups_per_cta - 1) / groups_per_cta, (int64_t)h->sm_count * 16);
+        model_view_kernel<<<grid, kThreads, 0, h->stream>>>(reinterpret_cast<const float4 *>(h->d_V), h->d_w,
+                                                             by_slot ? h->d_column_of : nullptr, (int64_t)h->d, kp4, gs,
+                                                             by_slot ? reinterpret_cast<float4 *>(h->d_Vs) : nullptr,
+                                                             by_slot ? h->d_pair_s : h->d_pair);
+        h->launches += 1;
+        version = h->model_version;
+    }
+    a.V = by_slot ? h->d_Vs : h->d_V;
+    a.pair = by_slot ? h->d_pair_s : h->d_pair;
+}
+
+// Renumbers the columns of the device CSR by frequency (see the kernels).  Decided per load: it pays when
+// the factors are larger than an L1 and the pass is long enough to hide the host's sort of d counters.
+int order_columns(dsfacto *h) {
+    h->slots = false;
+    bool on = h->nnz >= ((int64_t)1 << 22) && (size_t)h->d * h->Kp * sizeof(float) >= ((size_t)1 << 20);
+    if (const char *env = std::getenv("DSFACTO_COLUMN_ORDER")) on = std::strcmp(env, "0") != 0;
+    if (h->column_order == 1) on = true;
+    if (h->column_order == 2) on = false;
+    if (!on || h->nnz == 0) return DSFACTO_OK;
+    const size_t d = (size_t)h->d;
+    int32_t *d_slot_of = nullptr;   // first the counters, then the slot of every column
+    int rc;
+    if ((rc = dev_alloc(h, &d_slot_of, d)) || (rc = dev_alloc(h, &h->d_column_of, d)) ||
+        (rc = dev_alloc(h, &h->d_Vs, d * h->Kp)) || (rc = dev_alloc(h, &h->d_pair_s, d))) {
+        dev_free(d_slot_of);
+        return rc;
+    }
+    std::vector<int32_t> count, slot_of, column_of;
+    std::vector<uint64_t> key;
+    try { count.resize(d); slot_of.resize(d); column_of.resize(d); key.resize(d); }
+    catch (const std::bad_alloc &) { dev_free(d_slot_of); return DSFACTO_ERR_OOM; }
+    auto fail = [&](cudaError_t e) {
+        h->err = std::string("column order: ") + cudaGetErrorString(e);
+        dev_free(d_slot_of);
+        return e == cudaErrorMemoryAllocation ? DSFACTO_ERR_OOM : DSFACTO_ERR_CUDA;
+    };
+    cudaError_t e;
+    const int grid = (int)std::min<int64_t>((h->nnz + kThreads - 1) / kThreads, (int64_t)h->sm_count * 16);
+    if ((e = cudaMemsetAsync(d_slot_of, 0, sizeof(int32_t) * d, h->stream)) != cudaSuccess) return fail(e);
+    column_count_kernel<<<grid, kThreads, 0, h->stream>>>(h->d_idx, h->nnz, d_slot_of);
+    if ((e = cudaMemcpyAsync(count.data(), d_slot_of, sizeof(int32_t) * d, cudaMemcpyDeviceToHost, h->stream)) != cudaSuccess ||
+        (e = cudaStreamSynchronize(h->stream)) != cudaSuccess)
+        return fail(e);
+    // most frequent first, ties by column index: one sort of 64-bit keys
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < (int64_t)d; ++j)
+        key[(size_t)j] = ((uint64_t)(0x7FFFFFFFu - (uint32_t)count[(size_t)j]) << 32) | (uint64_t)(uint32_t)j;
+    std::sort(key.begin(), key.end());
+#pragma omp parallel for schedule(static)
+    for (int64_t sl = 0; sl < (int64_t)d; ++sl) {
+        const int32_t j = (int32_t)(key[(size_t)sl] & 0xFFFFFFFFu);
+        column_of[(size_t)sl] = j;
+        slot_of[(size_t)j] = (int32_t)sl;
+    }
+    if ((e = cudaMemcpyAsync(d_slot_of, slot_of.data(), sizeof(int32_t) * d, cudaMemcpyHostToDevice, h->stream)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(h->d_column_of, column_of.data(), sizeof(int32_t) * d, cudaMemcpyHostToDevice, h->stream)) != cudaSuccess)
+        return fail(e);
+    column_rename_kernel<<<grid, kThreads, 0, h->stream>>>(h->d_idx, h->nnz, d_slot_of);
+    h->launches += 2;
+    if ((e = cudaStreamSynchronize(h->stream)) != cudaSuccess || (e = cudaGetLastError()) != cudaSuccess) return fail(e);
+    dev_free(d_slot_of);
+    h->slots = true;
+    return DSFACTO_OK;
+}
+
 // Column shard, first half of the recompute pass: a_i, lin_i, q_i over the shard's own columns.
 int run_partial_refresh(dsfacto *h) {
     RefreshArgs a{};
     a.n = h->n; a.indptr = h->d_indptr; a.idx = h->d_idx; a.val = h->d_val; a.y = h->d_y;
-    a.w = h->d_w; a.V = h->d_V; a.A = h->d_A; a.G = h->d_G; a.f_out = nullptr;
+    model_view(h, a, true);
+    a.A = h->d_A; a.G = h->d_G; a.f_out = nullptr;
     a.lin_out = h->d_lin; a.q_out = h->d_q;
     a.partials = h->d_partials; a.w0 = h->w0; a.loss = h->loss;
     DSF_DISPATCH_REFRESH(h, h, a, kPartial, h->refresh_grid);
@@ -592,7 +686,8 @@ int run_refresh(dsfacto *h, bool timed) {
     if (h->nshards > 1) return run_partial_refresh(h);
     RefreshArgs a{};
     a.n = h->n; a.indptr = h->d_indptr; a.idx = h->d_idx; a.val = h->d_val; a.y = h->d_y;
-    a.w = h->d_w; a.V = h->d_V; a.A = h->d_A; a.G = h->d_G; a.f_out = nullptr;
+    model_view(h, a, true);
+    a.A = h->d_A; a.G = h->d_G; a.f_out = nullptr;
     a.partials = h->d_partials; a.w0 = h->w0; a.loss = h->loss;
     DSF_DISPATCH_REFRESH(h, h, a, kTrain, h->refresh_grid);
     reduce2_kernel<<<1, kThreads, 0, h->stream>>>(h->d_partials, h->refresh_grid, h->d_scal);
@@ -613,6 +708,7 @@ int run_refresh(dsfacto *h, bool timed) {
 
 // V padded (d x Kp) <-> caller layout (d x K)
 int upload_V(dsfacto *h, const float *V) {
+    h->model_version += 1;
     if (h->Kp == h->K) {
         CU_TRY(h, cudaMemcpyAsync(h->d_V, V, sizeof(float) * (size_t)h->d * h->K, cudaMemcpyHostToDevice, h->stream));
     } else {
@@ -1103,7 +1199,7 @@ static int create_handle(dsfacto_t **out, int64_t n, int32_t d, int32_t K, int32
     int rc;
     if ((rc = dev_alloc(h, &h->d_w, (size_t)d)) || (rc = dev_alloc(h, &h->d_V, (size_t)d * h->Kp)) ||
         (rc = dev_alloc(h, &h->d_row_start, (size_t)p + 1)) || (rc = dev_alloc(h, &h->d_col_start, (size_t)p + 1)) ||
-        (rc = dev_alloc(h, &h->d_scal, 4)))
+        (rc = dev_alloc(h, &h->d_scal, 4)) || (rc = dev_alloc(h, &h->d_pair, (size_t)d)))
         return fail(rc);
 
     std::vector<float> V;
@@ -1154,7 +1250,7 @@ void dsfacto_destroy(dsfacto_t *h) {
     if (!h) return;
     cudaStreamSynchronize(h->stream);
     free_data(h);
-    dev_free(h->d_w); dev_free(h->d_V); dev_free(h->d_Tb); dev_free(h->d_Tw); dev_free(h->d_S); dev_free(h->d_TS); dev_free(h->d_row_start); dev_free(h->d_col_start); dev_free(h->d_scal);
+    dev_free(h->d_w); dev_free(h->d_V); dev_free(h->d_Tb); dev_free(h->d_Tw); dev_free(h->d_S); dev_free(h->d_TS); dev_free(h->d_row_start); dev_free(h->d_col_start); dev_free(h->d_scal); dev_free(h->d_pair);
     for (auto &e : h->ev)
         if (e) cudaEventDestroy(e);
     delete h;
@@ -1297,6 +1393,7 @@ static int load_validated(dsfacto_t *h, const int64_t *indptr, const int32_t *in
     CU_TRY(h, cudaMemcpyAsync(h->d_tile_ptr, h->tile_ptr.data(), sizeof(int64_t) * h->tile_ptr.size(), cudaMemcpyHostToDevice, st));
     CU_TRY(h, cudaStreamSynchronize(st));
     if ((rc = finish_sgd_plan(h, pb))) { free_data(h); return rc; }
+    if ((rc = order_columns(h))) { free_data(h); return rc; }
     h->failed = false;
     h->loaded = true;
     if (h->nshards > 1) {   // the partial sums sit right behind A, so that one buffer holds what the shards exchange
@@ -1465,6 +1562,7 @@ int dsfacto_set_params(dsfacto_t *h, const float *w0, const float *w, const floa
     if (!h) return DSFACTO_ERR_INVALID_ARG;
     if (w0) { if (!std::isfinite(*w0)) return DSFACTO_ERR_INVALID_ARG; h->w0 = *w0; }
     if (w) {
+        h->model_version += 1;
         CU_TRY(h, cudaMemcpyAsync(h->d_w, w, sizeof(float) * (size_t)h->d, cudaMemcpyHostToDevice, h->stream));
         CU_TRY(h, cudaStreamSynchronize(h->stream));
     }
@@ -1539,7 +1637,7 @@ int dsfacto_bucket_host(int64_t n, int32_t d, int32_t p, const int64_t *indptr, 
 static int score_rows(dsfacto_t *h, int mode, int64_t m, const int64_t *indptr, const int32_t *indices,
                       const float *values, const float *y, float *scores_out, double sums2[2]) {
     RefreshArgs a{};
-    a.w = h->d_w; a.V = h->d_V; a.w0 = h->w0; a.loss = h->loss; a.n = m;
+    a.w0 = h->w0; a.loss = h->loss; a.n = m;
     int64_t *d_ip = nullptr;
     int32_t *d_ix = nullptr;
     float *d_vl = nullptr, *d_f = nullptr, *d_yy = nullptr;
@@ -1550,6 +1648,7 @@ static int score_rows(dsfacto_t *h, int mode, int64_t m, const int64_t *indptr, 
         if (!h->loaded) return DSFACTO_ERR_NO_DATA;
         if (m != h->n) return DSFACTO_ERR_INVALID_ARG;
         a.indptr = h->d_indptr; a.idx = h->d_idx; a.val = h->d_val;
+        model_view(h, a, true);
     } else {
         if (indptr[0] != 0 || indptr[m] < 0) return DSFACTO_ERR_INVALID_CSR;
         const int64_t nnz = indptr[m];
@@ -1566,6 +1665,7 @@ static int score_rows(dsfacto_t *h, int mode, int64_t m, const int64_t *indptr, 
             cudaMemcpyAsync(d_vl, values, sizeof(float) * (size_t)nnz, cudaMemcpyHostToDevice, h->stream);
         }
         a.indptr = d_ip; a.idx = d_ix; a.val = d_vl;
+        model_view(h, a, false);
     }
     const int grid = refresh_grid_for(h, m);
     cudaError_t e = cudaSuccess;
@@ -1641,6 +1741,10 @@ int dsfacto_debug_set(dsfacto_t *h, int32_t key, int64_t value) {
     case DSFACTO_DEBUG_CHUNK_LEN:
         if (value != 0 && (value < 16 || value > kChunkMax)) return DSFACTO_ERR_INVALID_ARG;
         h->chunk_override = (int)value;
+        return DSFACTO_OK;
+    case DSFACTO_DEBUG_COLUMN_ORDER:
+        if (value < 0 || value > 2) return DSFACTO_ERR_INVALID_ARG;
+        h->column_order = (int)value;
         return DSFACTO_OK;
     default:
         return DSFACTO_ERR_INVALID_ARG;

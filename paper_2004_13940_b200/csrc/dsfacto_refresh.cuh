@@ -9,6 +9,9 @@ namespace dsf {
 // Recompute pass (eq. (compute_a_jk), eq. (fm_model2), multiplier G): one lane group per row.
 //   a_ik = sum_j v_jk x_ij ; lin_i = sum_j w_j x_ij ; q_i = sum_j sum_k (v_jk x_ij)^2
 //   f_i = w0 + lin_i + 1/2 (sum_k a_ik^2 - q_i)
+// q_i is taken as sum_j x_ij^2 s_j with s_j = sum_k v_jk^2, which is the same sum regrouped: s_j is computed
+// once per column after the parameters changed (model_view_kernel) and sits next to w_j, so the lane that
+// owns an entry gets both with one 8-byte load and the K-wide part of an entry is K multiply-adds.
 // MODE kScore: writes f only.  kTrain: writes A, G and per-CTA fp64 partial sums {sum l_i, sum G_i}.
 // kEvaluate (held-out rows with labels; the quantities of the convergence figures of Section 5):
 // writes nothing per row, per-CTA fp64 partial sums {sum l_i, sum t_i} with t_i = (f_i - y_i)^2 for
@@ -25,7 +28,7 @@ struct RefreshArgs {
     const int32_t *idx;
     const float *val;
     const float *y;
-    const float *w;
+    const float2 *pair;  // per column (w_j, s_j = sum_k v_jk^2)
     const float *V;
     float *A;
     float *G;
@@ -88,7 +91,11 @@ __global__ void __launch_bounds__(kThreads, (LG >= 8 ? 3 : 4)) refresh_kernel(co
             if (t0 + LG >= end) { ahead = nbeg + l; ahead_end = has_next ? nend : nbeg; }
             jn = 0; xn = 0.f;
             if (ahead < ahead_end) { jn = __ldg(a.idx + ahead); xn = __ldg(a.val + ahead); }
-            if (t0 + l < end) lin = fmaf(__ldg(a.w + jm), xm, lin);
+            if (t0 + l < end) {
+                const float2 ws = __ldg(a.pair + jm);
+                lin = fmaf(ws.x, xm, lin);
+                q = fmaf(xm * xm, ws.y, q);
+            }
             const int cnt = (int)((end - t0) < (int64_t)LG ? (end - t0) : (int64_t)LG);
             // the rows of up to UB entries are requested before any of them is used
             constexpr int UB = LG < 8 ? LG : 8 / NV;
@@ -112,9 +119,8 @@ __global__ void __launch_bounds__(kThreads, (LG >= 8 ? 3 : 4)) refresh_kernel(co
                         const float x = xs[u];
 #pragma unroll
                         for (int v = 0; v < NV; ++v) {
-                            const float px = vv[u][v].x * x, py = vv[u][v].y * x, pz = vv[u][v].z * x, pw = vv[u][v].w * x;
-                            acc[v].x += px; acc[v].y += py; acc[v].z += pz; acc[v].w += pw;
-                            q = fmaf(px, px, q); q = fmaf(py, py, q); q = fmaf(pz, pz, q); q = fmaf(pw, pw, q);
+                            acc[v].x = fmaf(vv[u][v].x, x, acc[v].x); acc[v].y = fmaf(vv[u][v].y, x, acc[v].y);
+                            acc[v].z = fmaf(vv[u][v].z, x, acc[v].z); acc[v].w = fmaf(vv[u][v].w, x, acc[v].w);
                         }
                     }
                 }
@@ -175,6 +181,57 @@ __global__ void __launch_bounds__(kThreads, (LG >= 8 ? 3 : 4)) refresh_kernel(co
             a.partials[2 * blockIdx.x] = loss_sum;
             a.partials[2 * blockIdx.x + 1] = g_sum;
         }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Column slots for the recompute pass.  The pass gathers v_j and w_j by column index, and the L1 keeps
+// whole 128-byte lines: with the columns where the data set put them, a hot 64-byte row shares its line
+// with a cold neighbour and every hot w_j takes a line of its own.  The device copy of the CSR is
+// therefore renumbered once per load, the most frequent column first (slot = rank by frequency), and the
+// pass reads a copy of V and of the pairs (w_j, s_j) in slot order: hot rows sit side by side, 16 hot pairs share one line.  The
+// order of a row's entries does not change, so neither does any sum.  The stratum SGD kernels and
+// everything a caller sees keep the column indices of the data set.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads) column_count_kernel(const int32_t *__restrict__ idx, int64_t nnz, int32_t *__restrict__ count) {
+    const int lane = (int)(threadIdx.x & 31u);
+    // the loop bound is the same for all lanes of a warp, so the warp stays converged for the match
+    for (int64_t base = (int64_t)blockIdx.x * blockDim.x + threadIdx.x - lane; base < nnz; base += (int64_t)gridDim.x * blockDim.x) {
+        const bool valid = base + lane < nnz;
+        const int32_t j = valid ? idx[base + lane] : -1;
+        // entries of the same column in one warp are counted by one lane
+        const uint32_t peers = __match_any_sync(0xFFFFFFFFu, j);
+        if (valid && lane == __ffs(peers) - 1) atomicAdd(count + j, __popc(peers));
+    }
+}
+__global__ void __launch_bounds__(kThreads) column_rename_kernel(int32_t *__restrict__ idx, int64_t nnz, const int32_t *__restrict__ slot_of) {
+    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < nnz; t += (int64_t)gridDim.x * blockDim.x)
+        idx[t] = __ldg(slot_of + idx[t]);
+}
+// The model as the recompute pass reads it: pair[s] = (w_j, sum_k v_jk^2) and, when the columns are
+// renumbered (column_of != NULL: j = column_of[s], and Vs is given), Vs[s] = V[j]; else j = s.  A group of gs
+// lanes (a power of two <= 32) takes a row of kp4 float4s.
+__global__ void __launch_bounds__(kThreads) model_view_kernel(const float4 *__restrict__ V, const float *__restrict__ w,
+                                                              const int32_t *__restrict__ column_of, int64_t d, int kp4, int gs,
+                                                              float4 *__restrict__ Vs, float2 *__restrict__ pair) {
+    const int lane = (int)(threadIdx.x & 31u), gl = lane & (gs - 1);
+    const int64_t groups = (int64_t)gridDim.x * (blockDim.x / gs);
+    const int64_t g0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / gs;
+    const int64_t rounds = (d + groups - 1) / groups;   // the same for every lane of a warp: the shuffles below stay converged
+    for (int64_t it = 0; it < rounds; ++it) {
+        const int64_t s = g0 + it * groups;
+        float sum = 0.f;
+        int64_t j = 0;
+        if (s < d) {
+            j = column_of ? (int64_t)__ldg(column_of + s) : s;
+            for (int v = gl; v < kp4; v += gs) {
+                const float4 x = V[j * kp4 + v];
+                if (Vs) Vs[s * kp4 + v] = x;
+                sum = fmaf(x.x, x.x, sum); sum = fmaf(x.y, x.y, sum); sum = fmaf(x.z, x.z, sum); sum = fmaf(x.w, x.w, sum);
+            }
+        }
+        for (int o = gs >> 1; o > 0; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
+        if (s < d && gl == 0) pair[s] = make_float2(w[j], sum);
     }
 }
 
