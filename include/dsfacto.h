@@ -62,12 +62,19 @@ int dsfacto_create(dsfacto_t **out, int64_t n, int32_t d, int32_t K, int32_t p, 
 
 /* Loads the training set X (CSR: indptr int64[n+1] with indptr[0] = 0, indices int32[nnz] strictly
  * increasing inside each row and in [0,d), values fp32[nnz] finite; stored zeros count as entries)
- * and labels y fp32[n] (finite).  Builds the p x p tile lists on the host (figure "communication
+ * and labels y fp32[n] (finite).  Builds the p x p tile lists (figure "communication
  * pattern": row block of row i is floor(i*p/n), column block of column j is floor(j*p/d); tile
  * (r,c) belongs to round s = (c-r) mod p; tiles ordered by (s, r); inside a tile entries ordered
  * by (column, row)), copies CSR and tiles to the device and runs the recompute pass once, so that
  * A, G and the objective of the initial parameters exist.  Replaces any earlier data set.
- * Loads of 2^24 stored entries and more (with p at least twice the number of host threads) are
+ * Loads of 2^24 stored entries and more are bucketed on the device itself when the packed entry layout
+ * applies (local row and column ids fit 32 bits together, tile number and local column id too) and the
+ * device has room for the buffers of a sort (about 25 bytes per stored entry for the duration of the call):
+ * the CSR copy that the recompute pass needs anyway is turned into (tile, local column) keys, sorted by a
+ * stable radix sort, packed into entry records, and a kernel cuts the chunks of the stratum SGD launch; only
+ * the CSR arrays cross the link.  DSFACTO_LOAD=device takes this way for any non-empty load that fits the
+ * layout.  Otherwise, and with any other value of DSFACTO_LOAD, the tile lists are built on the host; there,
+ * loads of 2^24 stored entries and more (with p at least twice the number of host threads) are
  * streamed: each host thread buckets one row block at a time into page-locked staging memory and
  * copies it to its place on the device while the other row blocks are being bucketed.  That staging
  * memory (two row blocks per host thread) is allocated on the first such load and kept by the process
@@ -187,6 +194,11 @@ int dsfacto_last_epoch_ms(dsfacto_t *h, float ms[4]);
  * round, exactly Algorithm 1's order, instead of row block by row block. */
 enum { DSFACTO_DEBUG_SPIN_LIMIT = 0, DSFACTO_DEBUG_EXTRA_NEED = 1, DSFACTO_DEBUG_CHUNK_LEN = 2, DSFACTO_DEBUG_COLUMN_ORDER = 3 };
 int dsfacto_debug_set(dsfacto_t *h, int32_t key, int64_t value);
+
+/* How the last dsfacto_load_csr built the tile lists: info[0] = 0 on the host with one copy, 1 on the host
+ * streamed through page-locked staging memory, 2 on the device; info[1] = bytes it copied host -> device,
+ * info[2] = bytes it copied device -> host.  DSFACTO_ERR_NO_DATA before the first load. */
+int dsfacto_last_load(dsfacto_t *h, int64_t info[3]);
 
 /* Number of kernels this handle has launched since creation. */
 int dsfacto_launch_count(dsfacto_t *h, int64_t *out);

@@ -1,8 +1,11 @@
 // Host side of the DS-FACTO C ABI (include/dsfacto.h): handle, validation, seeded initialisation,
 // the tile bucketer, device memory, the epoch driver and the copy-out calls.
 #include "dsfacto.h"
+#include "dsfacto_bucket.cuh"
 #include "dsfacto_refresh.cuh"
 #include "dsfacto_sgd.cuh"
+
+#include <cub/device/device_radix_sort.cuh>
 
 #include <omp.h>
 #include <sys/mman.h>
@@ -73,6 +76,7 @@ struct dsfacto {
     float4 *d_S = nullptr, *d_TS = nullptr;  // scale records of the scaled column state (zero outside the SGD phase)
     int *d_run_count = nullptr;
     int refresh_grid = 0, norm_grid = 0;
+    int64_t load_info[3] = {0, 0, 0};   // last load: path (0 host, 1 host streamed, 2 device), bytes H2D, bytes D2H
     // Column slots of the recompute pass (per load): the device CSR holds slots (rank by frequency) instead of
     // column indices, and the pass reads w and V from copies in slot order.
     int column_order = 0;       // dsfacto_debug_set: 0 = decided per load, 1 = always, 2 = never
@@ -349,6 +353,7 @@ struct TileDescRef {          // where the chunks of a tile sit
     int64_t first = 0;
 };
 struct SgdPlanBuild {
+    HostBuf<ChunkDesc> bulk;   // device bucketing: the chunks of all tiles as a kernel cut them, instead of the planners
     std::vector<TilePlanner> planners;
     std::vector<TileDescRef> refs;   // per tile slot
 };
@@ -457,7 +462,31 @@ int finish_sgd_plan(dsfacto *h, SgdPlanBuild &pb) {
         if (segmented) h->launch_ptr.assign((size_t)nseg + 1, 0);
     } catch (const std::bad_alloc &) { return DSFACTO_ERR_OOM; }
     h->plan_segments = segmented ? nseg : 0;
-    int64_t pos = 0, runs = 0, recs = 0, cur_run = 0, cur_rec0 = 0;
+    auto chunk_of = [&](const TileDescRef &ref, int32_t q) -> const ChunkDesc & {
+        return pb.bulk.p ? pb.bulk.p[(size_t)(ref.first + q)] : pb.planners[(size_t)ref.owner].descs[(size_t)(ref.first + q)];
+    };
+    // 1. long runs and slice records of every tile (in parallel)
+    std::vector<int32_t> tile_runs, tile_recs;
+    struct Visit { int64_t slot, pos, run0, rec0; int32_t r, c, need; bool tail; };
+    std::vector<Visit> visit;
+    try {
+        tile_runs.assign((size_t)nt, 0);
+        tile_recs.assign((size_t)nt, 0);
+        visit.reserve((size_t)nt);
+    } catch (const std::bad_alloc &) { return DSFACTO_ERR_OOM; }
+#pragma omp parallel for schedule(dynamic, 64)
+    for (int64_t slot = 0; slot < nt; ++slot) {
+        const TileDescRef &ref = pb.refs[(size_t)slot];
+        int32_t nr = 0, nrec = 0;
+        for (int32_t q = 0; q < ref.count; ++q) {
+            const ChunkDesc &d = chunk_of(ref, q);
+            if ((d.flags & kChunkSlice) && d.slice == 0) { nr += 1; nrec += d.nslices; }
+        }
+        tile_runs[(size_t)slot] = nr;
+        tile_recs[(size_t)slot] = nrec;
+    }
+    // 2. the tiles in the order the launches visit them, with what each one starts from (one thread: p^2 steps)
+    int64_t pos = 0, runs = 0, recs = 0;
     for (int64_t seg = 0; seg < nseg; ++seg) {
         const int64_t s0 = seg * every, s1 = std::min(s0 + every, p);
         if (segmented) std::fill(seen.begin(), seen.end(), 0);
@@ -478,26 +507,40 @@ int finish_sgd_plan(dsfacto *h, SgdPlanBuild &pb) {
                 tail = h->sweep == 1 && r > c;
             }
             const TileDescRef &ref = pb.refs[(size_t)slot];
-            for (int32_t q = 0; q < ref.count; ++q) {
-                ChunkDesc d = pb.planners[(size_t)ref.owner].descs[(size_t)(ref.first + q)];
-                d.row0 = (int32_t)h->row_start[(size_t)r];
-                d.col0 = h->col_start[(size_t)c];
-                d.cblock = (int32_t)c;
-                d.need = seen[(size_t)c];
-                d.tile = (int32_t)slot;
-                d.nchunks = ref.count;
-                if (tail) d.flags |= kChunkTail;
-                if (d.flags & kChunkSlice) {
-                    if (d.slice == 0) { cur_run = runs++; cur_rec0 = recs; recs += d.nslices; }
-                    d.run_id = (int32_t)cur_run;
-                    d.rec0 = (int32_t)cur_rec0;
-                }
-                all[(size_t)pos++] = d;
-            }
+            Visit v;
+            v.slot = slot; v.pos = pos; v.run0 = runs; v.rec0 = recs;
+            v.r = (int32_t)r; v.c = (int32_t)c; v.need = seen[(size_t)c]; v.tail = tail;
+            try { visit.push_back(v); } catch (const std::bad_alloc &) { return DSFACTO_ERR_OOM; }
+            pos += ref.count;
+            runs += tile_runs[(size_t)slot];
+            recs += tile_recs[(size_t)slot];
             seen[(size_t)c] += ref.count;
             if (!segmented && (slot + 1) % p == 0) h->launch_ptr[(size_t)((slot + 1) / p)] = pos;
         }
         if (segmented) h->launch_ptr[(size_t)seg + 1] = pos;
+    }
+    // 3. the descriptors (in parallel over the tiles)
+#pragma omp parallel for schedule(dynamic, 64)
+    for (int64_t vi = 0; vi < (int64_t)visit.size(); ++vi) {
+        const Visit &v = visit[(size_t)vi];
+        const TileDescRef &ref = pb.refs[(size_t)v.slot];
+        int64_t next_run = v.run0, next_rec = v.rec0, cur_run = 0, cur_rec0 = 0;
+        for (int32_t q = 0; q < ref.count; ++q) {
+            ChunkDesc d = chunk_of(ref, q);
+            d.row0 = (int32_t)h->row_start[(size_t)v.r];
+            d.col0 = h->col_start[(size_t)v.c];
+            d.cblock = v.c;
+            d.need = v.need;
+            d.tile = (int32_t)v.slot;
+            d.nchunks = ref.count;
+            if (v.tail) d.flags |= kChunkTail;
+            if (d.flags & kChunkSlice) {
+                if (d.slice == 0) { cur_run = next_run++; cur_rec0 = next_rec; next_rec += d.nslices; }
+                d.run_id = (int32_t)cur_run;
+                d.rec0 = (int32_t)cur_rec0;
+            }
+            all[(size_t)(v.pos + q)] = d;
+        }
     }
     if (recs >= ((int64_t)1 << 31)) return DSFACTO_ERR_INVALID_ARG;
     h->total_chunks = total;
@@ -596,47 +639,48 @@ int order_columns(dsfacto *h) {
     if (h->column_order == 2) on = false;
     if (!on || h->nnz == 0) return DSFACTO_OK;
     const size_t d = (size_t)h->d;
-    int32_t *d_slot_of = nullptr;   // first the counters, then the slot of every column
+    // counters -> sort keys (most frequent first) with the column indices as values -> the sorted values are
+    // the column of every slot; a stable sort, so equal counts keep the order of the column indices
+    uint32_t *d_key = nullptr, *d_key_out = nullptr;
+    int32_t *d_col = nullptr, *d_slot_of = nullptr;
+    void *tmp = nullptr;
+    auto cleanup = [&]() {
+        dev_free(d_key); dev_free(d_key_out); dev_free(d_col); dev_free(d_slot_of);
+        if (tmp) cudaFree(tmp);
+        tmp = nullptr;
+    };
     int rc;
-    if ((rc = dev_alloc(h, &d_slot_of, d)) || (rc = dev_alloc(h, &h->d_column_of, d)) ||
+    if ((rc = dev_alloc(h, &d_key, d)) || (rc = dev_alloc(h, &d_key_out, d)) || (rc = dev_alloc(h, &d_col, d)) ||
+        (rc = dev_alloc(h, &d_slot_of, d)) || (rc = dev_alloc(h, &h->d_column_of, d)) ||
         (rc = dev_alloc(h, &h->d_Vs, d * h->Kp)) || (rc = dev_alloc(h, &h->d_pair_s, d))) {
-        dev_free(d_slot_of);
+        cleanup();
         return rc;
     }
-    std::vector<int32_t> count, slot_of, column_of;
-    std::vector<uint64_t> key;
-    try { count.resize(d); slot_of.resize(d); column_of.resize(d); key.resize(d); }
-    catch (const std::bad_alloc &) { dev_free(d_slot_of); return DSFACTO_ERR_OOM; }
     auto fail = [&](cudaError_t e) {
         h->err = std::string("column order: ") + cudaGetErrorString(e);
-        dev_free(d_slot_of);
+        cudaStreamSynchronize(h->stream);
+        cleanup();
         return e == cudaErrorMemoryAllocation ? DSFACTO_ERR_OOM : DSFACTO_ERR_CUDA;
     };
     cudaError_t e;
+    size_t tmp_bytes = 0;
+    if ((e = cub::DeviceRadixSort::SortPairs(nullptr, tmp_bytes, d_key, d_key_out, d_col, h->d_column_of, (int64_t)d, 0, 32,
+                                             h->stream)) != cudaSuccess)
+        return fail(e);
+    if ((e = cudaMalloc(&tmp, tmp_bytes ? tmp_bytes : 1)) != cudaSuccess) return fail(e);
     const int grid = (int)std::min<int64_t>((h->nnz + kThreads - 1) / kThreads, (int64_t)h->sm_count * 16);
+    const int dgrid = (int)std::min<int64_t>(((int64_t)d + kThreads - 1) / kThreads, (int64_t)h->sm_count * 16);
     if ((e = cudaMemsetAsync(d_slot_of, 0, sizeof(int32_t) * d, h->stream)) != cudaSuccess) return fail(e);
     column_count_kernel<<<grid, kThreads, 0, h->stream>>>(h->d_idx, h->nnz, d_slot_of);
-    if ((e = cudaMemcpyAsync(count.data(), d_slot_of, sizeof(int32_t) * d, cudaMemcpyDeviceToHost, h->stream)) != cudaSuccess ||
-        (e = cudaStreamSynchronize(h->stream)) != cudaSuccess)
+    column_keys_kernel<<<dgrid, kThreads, 0, h->stream>>>(d_slot_of, (int64_t)d, d_key, d_col);
+    if ((e = cub::DeviceRadixSort::SortPairs(tmp, tmp_bytes, d_key, d_key_out, d_col, h->d_column_of, (int64_t)d, 0, 32,
+                                             h->stream)) != cudaSuccess)
         return fail(e);
-    // most frequent first, ties by column index: one sort of 64-bit keys
-#pragma omp parallel for schedule(static)
-    for (int64_t j = 0; j < (int64_t)d; ++j)
-        key[(size_t)j] = ((uint64_t)(0x7FFFFFFFu - (uint32_t)count[(size_t)j]) << 32) | (uint64_t)(uint32_t)j;
-    std::sort(key.begin(), key.end());
-#pragma omp parallel for schedule(static)
-    for (int64_t sl = 0; sl < (int64_t)d; ++sl) {
-        const int32_t j = (int32_t)(key[(size_t)sl] & 0xFFFFFFFFu);
-        column_of[(size_t)sl] = j;
-        slot_of[(size_t)j] = (int32_t)sl;
-    }
-    if ((e = cudaMemcpyAsync(d_slot_of, slot_of.data(), sizeof(int32_t) * d, cudaMemcpyHostToDevice, h->stream)) != cudaSuccess ||
-        (e = cudaMemcpyAsync(h->d_column_of, column_of.data(), sizeof(int32_t) * d, cudaMemcpyHostToDevice, h->stream)) != cudaSuccess)
-        return fail(e);
+    column_slots_kernel<<<dgrid, kThreads, 0, h->stream>>>(h->d_column_of, (int64_t)d, d_slot_of);
     column_rename_kernel<<<grid, kThreads, 0, h->stream>>>(h->d_idx, h->nnz, d_slot_of);
-    h->launches += 2;
+    h->launches += 4;
     if ((e = cudaStreamSynchronize(h->stream)) != cudaSuccess || (e = cudaGetLastError()) != cudaSuccess) return fail(e);
-    dev_free(d_slot_of);
+    cleanup();
     h->slots = true;
     return DSFACTO_OK;
 }
@@ -1289,6 +1333,110 @@ static int filter_columns(int64_t n, const int64_t *indptr, const int32_t *indic
     return DSFACTO_OK;
 }
 
+// ---- tile bucketing on the device (see dsfacto_bucket.cuh) ----
+// Whether this load goes that way: packed entry layout, keys of at most 32 bits, enough entries to be worth
+// it (DSFACTO_LOAD=device: any non-empty load; any other value of DSFACTO_LOAD: never), and room on the
+// device for the sort's buffers next to what the handle keeps.
+static bool device_bucketing_wanted(const dsfacto *h, int64_t nnz, const char *load_env) {
+    if (nnz <= 0 || h->wide) return false;
+    if (bits_for((int64_t)h->p * h->p) + h->jbits > 32) return false;
+    if (load_env) return std::strcmp(load_env, "device") == 0;
+    if (nnz < kStreamedLoadMinEntries) return false;
+    size_t free_b = 0, total_b = 0;
+    if (cudaMemGetInfo(&free_b, &total_b) != cudaSuccess) return false;
+    // sort buffers 2 x (4 + 8) bytes and their scratch, then entry records, A, G and the launch plan
+    const double need = (double)nnz * (24.0 + 1.0 + 8.0 + 2.0) + (double)h->n * 4.0 * (h->Kp + 2);
+    return (double)free_b > need * 1.1;
+}
+
+// d_indptr, d_idx, d_val hold the CSR arrays (copies queued on the stream), d_ent is allocated.  Fills
+// d_ent, h->tile_ptr and the per-tile pieces of the launch plan.
+static int device_bucket_tiles(dsfacto *h, int64_t nnz, SgdPlanBuild &pb) {
+    const int64_t nt = (int64_t)h->p * h->p;
+    const int kb = bits_for(nt) + h->jbits;
+    cudaStream_t st = h->stream;
+    uint32_t *key[2] = {nullptr, nullptr};
+    unsigned long long *pay[2] = {nullptr, nullptr};
+    void *tmp = nullptr;
+    int64_t *d_tp = nullptr, *d_count = nullptr, *d_first = nullptr;
+    ChunkDesc *d_out = nullptr;
+    auto cleanup = [&]() {
+        dev_free(key[0]); dev_free(key[1]); dev_free(pay[0]); dev_free(pay[1]);
+        if (tmp) cudaFree(tmp);
+        tmp = nullptr;
+        dev_free(d_tp); dev_free(d_count); dev_free(d_first); dev_free(d_out);
+    };
+    auto fail = [&](cudaError_t e) {
+        h->err = std::string("device bucketing: ") + cudaGetErrorString(e);
+        cudaStreamSynchronize(st);
+        cleanup();
+        return e == cudaErrorMemoryAllocation ? DSFACTO_ERR_OOM : DSFACTO_ERR_CUDA;
+    };
+    int rc;
+    if ((rc = dev_alloc(h, &key[0], (size_t)nnz)) || (rc = dev_alloc(h, &key[1], (size_t)nnz)) ||
+        (rc = dev_alloc(h, &pay[0], (size_t)nnz)) || (rc = dev_alloc(h, &pay[1], (size_t)nnz)) ||
+        (rc = dev_alloc(h, &d_tp, (size_t)nt + 1)) || (rc = dev_alloc(h, &d_count, (size_t)nt)) ||
+        (rc = dev_alloc(h, &d_first, (size_t)nt))) {
+        cleanup();
+        return rc;
+    }
+    cudaError_t e;
+    size_t tmp_bytes = 0;
+    if ((e = cub::DeviceRadixSort::SortPairs(nullptr, tmp_bytes, key[0], key[1], pay[0], pay[1], nnz, 0, kb, st)) != cudaSuccess)
+        return fail(e);
+    if ((e = cudaMalloc(&tmp, tmp_bytes ? tmp_bytes : 1)) != cudaSuccess) return fail(e);
+
+    const int wide_grid = h->sm_count * 16;
+    TileKeyArgs ka{};
+    ka.n = h->n; ka.indptr = h->d_indptr; ka.idx = h->d_idx; ka.val = h->d_val; ka.d = h->d; ka.p = h->p;
+    ka.sweep = h->sweep; ka.jbits = h->jbits; ka.row_start = h->d_row_start; ka.col_start = h->d_col_start;
+    ka.key = key[0]; ka.payload = pay[0];
+    tile_keys_kernel<<<wide_grid, kThreads, 0, st>>>(ka);
+    if ((e = cub::DeviceRadixSort::SortPairs(tmp, tmp_bytes, key[0], key[1], pay[0], pay[1], nnz, 0, kb, st)) != cudaSuccess)
+        return fail(e);
+    pack_entries_kernel<<<wide_grid, kThreads, 0, st>>>(nnz, key[1], pay[1], h->jbits, h->d_ent);
+    tile_bounds_kernel<<<(int)std::min<int64_t>((nt + kThreads) / kThreads, wide_grid), kThreads, 0, st>>>(nnz, key[1], h->jbits, nt, d_tp);
+    TilePlanArgs pa{};
+    pa.key = key[1]; pa.tile_ptr = d_tp; pa.ntiles = nt; pa.jbits = h->jbits; pa.chunk_len = h->chunk_len;
+    pa.count = d_count; pa.first = d_first; pa.out = nullptr;
+    plan_tiles_kernel<false><<<wide_grid, kThreads, 0, st>>>(pa);
+    h->launches += 4;
+    std::vector<int64_t> count;
+    try {
+        h->tile_ptr.assign((size_t)nt + 1, 0);
+        count.resize((size_t)nt);
+    } catch (const std::bad_alloc &) { cudaStreamSynchronize(st); cleanup(); return DSFACTO_ERR_OOM; }
+    if ((e = cudaMemcpyAsync(h->tile_ptr.data(), d_tp, sizeof(int64_t) * ((size_t)nt + 1), cudaMemcpyDeviceToHost, st)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(count.data(), d_count, sizeof(int64_t) * (size_t)nt, cudaMemcpyDeviceToHost, st)) != cudaSuccess ||
+        (e = cudaStreamSynchronize(st)) != cudaSuccess || (e = cudaGetLastError()) != cudaSuccess)
+        return fail(e);
+    // where every tile's chunks go: one planner holds them all, tile after tile
+    int64_t total = 0;
+    for (int64_t t = 0; t < nt; ++t) {
+        TileDescRef &ref = pb.refs[(size_t)t];
+        ref.owner = 0;
+        ref.first = total;
+        ref.count = (int32_t)count[(size_t)t];
+        const int64_t c = count[(size_t)t];
+        count[(size_t)t] = total;
+        total += c;
+    }
+    if (!pb.bulk.alloc((size_t)total)) { cleanup(); return DSFACTO_ERR_OOM; }
+    if (total > 0) {
+        if ((rc = dev_alloc(h, &d_out, (size_t)total))) { cleanup(); return rc; }
+        if ((e = cudaMemcpyAsync(d_first, count.data(), sizeof(int64_t) * (size_t)nt, cudaMemcpyHostToDevice, st)) != cudaSuccess)
+            return fail(e);
+        pa.out = d_out;
+        plan_tiles_kernel<true><<<wide_grid, kThreads, 0, st>>>(pa);
+        h->launches += 1;
+        if ((e = cudaMemcpyAsync(pb.bulk.data(), d_out, sizeof(ChunkDesc) * (size_t)total, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
+            return fail(e);
+    }
+    if ((e = cudaStreamSynchronize(st)) != cudaSuccess || (e = cudaGetLastError()) != cudaSuccess) return fail(e);
+    cleanup();
+    return DSFACTO_OK;
+}
+
 static int load_validated(dsfacto_t *h, const int64_t *indptr, const int32_t *indices, const float *values, const float *y);
 
 int dsfacto_load_csr(dsfacto_t *h, const int64_t *indptr, const int32_t *indices, const float *values, const float *y) {
@@ -1353,11 +1501,16 @@ static int load_validated(dsfacto_t *h, const int64_t *indptr, const int32_t *in
     if (!init_plan_build(h, pb, omp_get_max_threads())) { cudaStreamSynchronize(st); free_data(h); return DSFACTO_ERR_OOM; }
     const bool by_row_block = use_row_block_bucketer(h);
     const char *load_env = std::getenv("DSFACTO_LOAD");
-    const bool streamed = by_row_block && nnz > 0 &&
+    const bool on_device = device_bucketing_wanted(h, nnz, load_env);
+    const bool streamed = !on_device && by_row_block && nnz > 0 &&
                           (nnz >= kStreamedLoadMinEntries ||
                            (load_env && (std::strcmp(load_env, "stream") == 0 || std::strcmp(load_env, "nostaging") == 0))) &&
                           !(load_env && std::strcmp(load_env, "simple") == 0);
-    if (streamed) {
+    if (on_device) {
+        // bucketed below, once the entry array is allocated; the tile pointers get their size here
+        try { h->tile_ptr.assign((size_t)h->p * h->p + 1, 0); }
+        catch (const std::bad_alloc &) { cudaStreamSynchronize(st); free_data(h); return DSFACTO_ERR_OOM; }
+    } else if (streamed) {
         try { column_blocks(h, cb); } catch (const std::bad_alloc &) { cudaStreamSynchronize(st); free_data(h); return DSFACTO_ERR_OOM; }
         longest = count_tiles_by_row_block(h, cb, indptr, indices);
         if (longest < 0) { cudaStreamSynchronize(st); free_data(h); return DSFACTO_ERR_OOM; }
@@ -1375,7 +1528,10 @@ static int load_validated(dsfacto_t *h, const int64_t *indptr, const int32_t *in
         free_data(h);
         return rc;
     }
-    bool copy_from_host = !streamed;
+    bool copy_from_host = !streamed && !on_device;
+    if (on_device) {
+        if ((rc = device_bucket_tiles(h, nnz, pb))) { cudaStreamSynchronize(st); free_data(h); return rc; }
+    }
     if (streamed) {
         bool no_staging = false;
         rc = stream_tiles_by_row_block(h, cb, longest, indptr, indices, values, &no_staging, &pb);
@@ -1394,6 +1550,13 @@ static int load_validated(dsfacto_t *h, const int64_t *indptr, const int32_t *in
     CU_TRY(h, cudaStreamSynchronize(st));
     if ((rc = finish_sgd_plan(h, pb))) { free_data(h); return rc; }
     if ((rc = order_columns(h))) { free_data(h); return rc; }
+    {
+        const int64_t nt1 = (int64_t)h->p * h->p + 1, plan_bytes = (int64_t)sizeof(ChunkDesc) * h->total_chunks;
+        const int64_t csr_bytes = 8 * (n + 1) + 8 * nnz + 4 * n;   // indptr, idx, val, y
+        h->load_info[0] = on_device ? 2 : (copy_from_host ? 0 : 1);
+        h->load_info[1] = csr_bytes + 8 * nt1 + plan_bytes + (on_device ? 8 * (nt1 - 1) : (h->wide ? 12 : 8) * nnz);
+        h->load_info[2] = on_device ? 8 * nt1 + 8 * (nt1 - 1) + plan_bytes : 0;
+    }
     h->failed = false;
     h->loaded = true;
     if (h->nshards > 1) {   // the partial sums sit right behind A, so that one buffer holds what the shards exchange
@@ -1749,6 +1912,13 @@ int dsfacto_debug_set(dsfacto_t *h, int32_t key, int64_t value) {
     default:
         return DSFACTO_ERR_INVALID_ARG;
     }
+}
+
+int dsfacto_last_load(dsfacto_t *h, int64_t info[3]) {
+    if (!h || !info) return DSFACTO_ERR_INVALID_ARG;
+    if (!h->loaded) return DSFACTO_ERR_NO_DATA;
+    for (int k = 0; k < 3; ++k) info[k] = h->load_info[k];
+    return DSFACTO_OK;
 }
 
 int dsfacto_launch_count(dsfacto_t *h, int64_t *out) {

@@ -198,7 +198,8 @@ __global__ void __launch_bounds__(kThreads, (LG >= 8 ? 3 : 4)) refresh_kernel(co
 // Column slots for the recompute pass.  The pass gathers v_j and w_j by column index, and the L1 keeps
 // whole 128-byte lines: with the columns where the data set put them, a hot 64-byte row shares its line
 // with a cold neighbour and every hot w_j takes a line of its own.  The device copy of the CSR is
-// therefore renumbered once per load, the most frequent column first (slot = rank by frequency), and the
+// therefore renumbered once per load, the most frequent column first (slot = rank by frequency: a count
+// kernel, a stable radix sort of the d counters by cub::DeviceRadixSort, a rename kernel), and the
 // pass reads a copy of V and of the pairs (w_j, s_j) in slot order: hot rows sit side by side, 16 hot pairs share one line.  The
 // order of a row's entries does not change, so neither does any sum.  The stratum SGD kernels and
 // everything a caller sees keep the column indices of the data set.
@@ -213,6 +214,18 @@ __global__ void __launch_bounds__(kThreads) column_count_kernel(const int32_t *_
         const uint32_t peers = __match_any_sync(0xFFFFFFFFu, j);
         if (valid && lane == __ffs(peers) - 1) atomicAdd(count + j, __popc(peers));
     }
+}
+// sort key of a column: most frequent first (a column holds fewer than 2^31 entries); value: the column
+__global__ void __launch_bounds__(kThreads) column_keys_kernel(const int32_t *__restrict__ count, int64_t d, uint32_t *__restrict__ key,
+                                                               int32_t *__restrict__ column) {
+    for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < d; j += (int64_t)gridDim.x * blockDim.x) {
+        key[j] = 0x7FFFFFFFu - (uint32_t)count[j];
+        column[j] = (int32_t)j;
+    }
+}
+__global__ void __launch_bounds__(kThreads) column_slots_kernel(const int32_t *__restrict__ column_of, int64_t d, int32_t *__restrict__ slot_of) {
+    for (int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; s < d; s += (int64_t)gridDim.x * blockDim.x)
+        slot_of[column_of[s]] = (int32_t)s;
 }
 __global__ void __launch_bounds__(kThreads) column_rename_kernel(int32_t *__restrict__ idx, int64_t nnz, const int32_t *__restrict__ slot_of) {
     for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < nnz; t += (int64_t)gridDim.x * blockDim.x)

@@ -49,6 +49,7 @@ SIGNATURES = {
     "dsfacto_bucket_host_shard": (ctypes.c_int, [_c_i64, _c_i32, _c_i32, _c_i32, _c_i32, _vp, _vp, _vp,
                                                  ctypes.POINTER(_c_i64), _vp, _vp, _vp, _vp]),
     "dsfacto_launch_count": (ctypes.c_int, [_vp, ctypes.POINTER(_c_i64)]),
+    "dsfacto_last_load": (ctypes.c_int, [_vp, ctypes.POINTER(_c_i64)]),
     "dsfacto_last_error": (ctypes.c_char_p, [_vp]),
     "dsfacto_strerror": (ctypes.c_char_p, [ctypes.c_int]),
     "dsfacto_score_loss_noalloc": (ctypes.c_int, [_c_i64, _c_i32, _c_i32, _c_i32, _vp, _vp, _vp, _vp, _c_f32, _vp, _vp,
@@ -357,6 +358,12 @@ class DSFacto:
 
     def debug_set(self, key: int, value: int):
         self._check(dsfacto_debug_set(self._h, int(key), int(value)), "dsfacto_debug_set")
+
+    def last_load(self):
+        """(path, bytes host -> device, bytes device -> host) of the last load; path 0 host, 1 host streamed, 2 device."""
+        info = (_c_i64 * 3)()
+        self._check(lib().dsfacto_last_load(self._h, info), "dsfacto_last_load")
+        return int(info[0]), int(info[1]), int(info[2])
 
     def launch_count(self) -> int:
         v = _c_i64()

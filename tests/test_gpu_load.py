@@ -1,8 +1,9 @@
-"""The three ways dsfacto_load_csr builds the tile lists on the device give the same lists, bit for
-bit, as the oracle's bucketing: the plain host bucketer, the row-block bucketer, and the streamed
-load (row blocks bucketed into page-locked staging memory and copied block by block), which large
-loads take by default and which DSFACTO_LOAD=stream forces on small ones.  DSFACTO_LOAD=nostaging makes
-the streamed load behave as if no page-locked memory could be had, which must end in the row-block
+"""The ways dsfacto_load_csr builds the tile lists on the device give the same lists, bit for bit, as the
+oracle's bucketing: the plain host bucketer, the row-block bucketer, the streamed load (row blocks
+bucketed into page-locked staging memory and copied block by block; DSFACTO_LOAD=stream forces it on small
+loads), and the bucketing on the device itself (keys, a stable radix sort, the chunk plan cut by a kernel),
+which large loads take by default and DSFACTO_LOAD=device forces on small ones.  DSFACTO_LOAD=nostaging
+makes the streamed load behave as if no page-locked memory could be had, which must end in the row-block
 bucketer with one copy, not in an error."""
 import numpy as np
 import pytest
@@ -14,7 +15,7 @@ from paper_2004_13940_b200 import workloads as W
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("mode", ["stream", "nostaging", "simple", None])
+@pytest.mark.parametrize("mode", ["device", "stream", "nostaging", "simple", None])
 @pytest.mark.parametrize("name,kw", [("C3", {}), ("C4s", {}), ("C4s", {"p": 200}), ("C5s", {"p": 64}), ("C2", {"p": 40}),
                                      ("C1", {"p": 2500})])
 def test_load_paths_give_the_oracle_tiles_and_epochs(monkeypatch, mode, name, kw):
@@ -59,3 +60,34 @@ def test_streamed_load_of_the_wide_entry_layout(monkeypatch):
         assert np.array_equal(tp, o.tile_ptr) and np.array_equal(rows, o.rows) and np.array_equal(cols, o.cols)
         assert np.array_equal(v, o.vals)
         assert g.epoch() == pytest.approx(o.epoch(), rel=1e-4)
+
+
+@pytest.mark.parametrize("sweep", [None, "round"])
+@pytest.mark.parametrize("name,kw", [("C1", {}), ("C2", {}), ("C3", {}), ("C4s", {}), ("C5s", {}), ("C3", {"p": 7})])
+def test_device_bucketing_gives_the_same_bits_as_the_host(monkeypatch, sweep, name, kw):
+    # same tile lists and the same chunk plan, hence the same parameters bit for bit; also with rows and
+    # columns emptied so that tiles, rows and whole column blocks are empty
+    if sweep:
+        monkeypatch.setenv("DSFACTO_SWEEP", sweep)
+    else:
+        monkeypatch.delenv("DSFACTO_SWEEP", raising=False)
+    wl = W.make(name, **kw)
+    keep = np.ones(wl.indices.shape[0], bool)
+    rows = np.repeat(np.arange(wl.n), np.diff(wl.indptr))
+    keep[(rows % 7) == 3] = False                       # every seventh row empty
+    keep[(wl.indices * wl.p) // wl.d == wl.p // 2] = False   # one column block empty
+    indptr = np.concatenate([[0], np.cumsum(np.bincount(rows[keep], minlength=wl.n))]).astype(np.int64)
+    indices, values = wl.indices[keep], wl.values[keep]
+    res = []
+    for mode in ("device", "simple"):
+        monkeypatch.setenv("DSFACTO_LOAD", mode)
+        with D.DSFacto(wl.n, wl.d, wl.K, wl.p, wl.loss, wl.lambda_w, wl.lambda_v, wl.eta, wl.init_seed) as g:
+            g.load_csr(indptr, indices, values, wl.y)
+            tiles = g.get_tiles()
+            objs = [g.objective()] + [g.epoch() for _ in range(2)]
+            w0, w, V = g.get_params()
+        res.append((tiles, objs, w0, w, V))
+    for a, b in zip(res[0][0], res[1][0]):
+        assert np.array_equal(a, b)
+    assert res[0][1] == res[1][1] and res[0][2] == res[1][2]
+    assert np.array_equal(res[0][3], res[1][3]) and np.array_equal(res[0][4], res[1][4])
