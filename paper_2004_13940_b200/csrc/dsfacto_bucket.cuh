@@ -88,15 +88,23 @@ struct TilePlanArgs {
     const int64_t *tile_ptr;   // ntiles + 1
     int64_t ntiles;
     int jbits, chunk_len;
-    int64_t *count;            // pass 1: chunks per tile
-    const int64_t *first;      // pass 2: where the tile's chunks go
+    // kPlanCount: per tile the number of chunks, of runs longer than a chunk and of their slices
+    int64_t *count, *runs, *recs;
+    // writing passes: where the tile's chunks go; kPlanFull also: chunks of the earlier tiles of the tile's
+    // column block, number of the tile's first long run and of its first slice record, and the partition
+    const int64_t *first, *need, *run0, *rec0;
+    int p, sweep;
+    const int64_t *row_start;
+    const int32_t *col_start;
     ChunkDesc *out;
 };
+enum { kPlanCount = 0, kPlanPieces = 1, kPlanFull = 2 };
 
-// One warp per tile; everything but the key reads is the same in all lanes.  WRITE = false counts the
-// chunks of every tile, WRITE = true writes them (entry offset, length, flags, local column and slice
-// numbers; the rest of a descriptor depends on the sweep order and is filled in on the host).
-template <bool WRITE>
+// One warp per tile; everything but the key reads is the same in all lanes.  kPlanCount counts, kPlanPieces
+// writes what depends on the tile alone (entry offset, length, flags, local column and slice numbers; the
+// host fills in the rest: plans cut into segments), kPlanFull writes complete descriptors for the plain plan,
+// in which the tiles are visited in slot order.
+template <int MODE>
 __global__ void __launch_bounds__(kThreads) plan_tiles_kernel(const TilePlanArgs a) {
     const int lane = (int)(threadIdx.x & 31u);
     const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -105,17 +113,34 @@ __global__ void __launch_bounds__(kThreads) plan_tiles_kernel(const TilePlanArgs
     const int64_t L = a.chunk_len;
     for (int64_t t = warp; t < a.ntiles; t += nwarps) {
         const int64_t beg = a.tile_ptr[t], nt = a.tile_ptr[t + 1] - beg;
-        ChunkDesc *out = WRITE ? a.out + a.first[t] : nullptr;
-        int64_t emitted = 0;
+        ChunkDesc *out = MODE != kPlanCount ? a.out + a.first[t] : nullptr;
+        ChunkDesc proto{};   // what all chunks of the tile share
+        int64_t next_run = 0, next_rec = 0, cur_run = 0, cur_rec0 = 0;
+        if (MODE == kPlanFull) {
+            int64_t r, c;
+            if (a.sweep == 1) { r = a.p - 1 - t / a.p; c = t % a.p; }
+            else { r = t % a.p; c = (r + t / a.p) % a.p; }
+            proto.row0 = (int32_t)a.row_start[r];
+            proto.col0 = a.col_start[c];
+            proto.cblock = (int32_t)c;
+            proto.need = (int32_t)a.need[t];
+            proto.tile = (int32_t)t;
+            proto.nchunks = (int32_t)(a.first[t + 1] - a.first[t]);
+            proto.flags = (a.sweep == 1 && r > c) ? kChunkTail : 0;
+            next_run = a.run0[t];
+            next_rec = a.rec0[t];
+        }
+        int64_t emitted = 0, nruns = 0, nrecs = 0;
         auto emit = [&](int64_t off, int64_t len, int flags, uint32_t jl, int64_t slice, int64_t nslices) {
-            if (WRITE && lane == 0) {
-                ChunkDesc d{};
+            if (MODE != kPlanCount && lane == 0) {
+                ChunkDesc d = proto;
                 d.ent_off = beg + off;
                 d.len = (int32_t)len;
-                d.flags = flags;
+                d.flags |= flags;
                 d.jl = (int32_t)jl;
                 d.slice = (int32_t)slice;
                 d.nslices = (int32_t)nslices;
+                if (MODE == kPlanFull && (flags & kChunkSlice)) { d.run_id = (int32_t)cur_run; d.rec0 = (int32_t)cur_rec0; }
                 out[emitted] = d;
             }
             emitted += 1;
@@ -129,6 +154,11 @@ __global__ void __launch_bounds__(kThreads) plan_tiles_kernel(const TilePlanArgs
                 int64_t per = ((len + ns - 1) / ns + 31) & ~(int64_t)31;   // slices of whole passes, about equal
                 if (per > L) per = L;
                 ns = (len + per - 1) / per;
+                nruns += 1;
+                nrecs += ns;
+                cur_run = next_run++;
+                cur_rec0 = next_rec;
+                next_rec += ns;
                 for (int64_t k = 0; k < ns; ++k) {
                     const int64_t rest = len - k * per;
                     emit(prev + k * per, rest < per ? rest : per, kChunkSlice, jl, k, ns);
@@ -163,8 +193,11 @@ __global__ void __launch_bounds__(kThreads) plan_tiles_kernel(const TilePlanArgs
         }
         if (have) take_run(run_start, nt - run_start, run_jl);
         if (cur > 0) emit(cur0, cur, 0, 0u, 0, 0);
-        if (!WRITE && lane == 0) a.count[t] = emitted;
+        if (MODE == kPlanCount && lane == 0) { a.count[t] = emitted; a.runs[t] = nruns; a.recs[t] = nrecs; }
     }
 }
+
+// test knob: the first chunk of the sweep is made to wait for more finished chunks than there will ever be
+__global__ void plan_extra_need_kernel(ChunkDesc *desc, int extra) { desc[0].need += extra; }
 
 }  // namespace dsf

@@ -353,6 +353,7 @@ struct TileDescRef {          // where the chunks of a tile sit
     int64_t first = 0;
 };
 struct SgdPlanBuild {
+    bool finished = false;     // device bucketing, plain plan: the descriptors are complete and on the device already
     HostBuf<ChunkDesc> bulk;   // device bucketing: the chunks of all tiles as a kernel cut them, instead of the planners
     std::vector<TilePlanner> planners;
     std::vector<TileDescRef> refs;   // per tile slot
@@ -1358,13 +1359,13 @@ static int device_bucket_tiles(dsfacto *h, int64_t nnz, SgdPlanBuild &pb) {
     uint32_t *key[2] = {nullptr, nullptr};
     unsigned long long *pay[2] = {nullptr, nullptr};
     void *tmp = nullptr;
-    int64_t *d_tp = nullptr, *d_count = nullptr, *d_first = nullptr;
+    int64_t *d_tp = nullptr, *d_plan = nullptr, *d_in = nullptr;   // tile pointers; per-tile counts; per-tile starting values
     ChunkDesc *d_out = nullptr;
     auto cleanup = [&]() {
         dev_free(key[0]); dev_free(key[1]); dev_free(pay[0]); dev_free(pay[1]);
         if (tmp) cudaFree(tmp);
         tmp = nullptr;
-        dev_free(d_tp); dev_free(d_count); dev_free(d_first); dev_free(d_out);
+        dev_free(d_tp); dev_free(d_plan); dev_free(d_in); dev_free(d_out);
     };
     auto fail = [&](cudaError_t e) {
         h->err = std::string("device bucketing: ") + cudaGetErrorString(e);
@@ -1375,8 +1376,8 @@ static int device_bucket_tiles(dsfacto *h, int64_t nnz, SgdPlanBuild &pb) {
     int rc;
     if ((rc = dev_alloc(h, &key[0], (size_t)nnz)) || (rc = dev_alloc(h, &key[1], (size_t)nnz)) ||
         (rc = dev_alloc(h, &pay[0], (size_t)nnz)) || (rc = dev_alloc(h, &pay[1], (size_t)nnz)) ||
-        (rc = dev_alloc(h, &d_tp, (size_t)nt + 1)) || (rc = dev_alloc(h, &d_count, (size_t)nt)) ||
-        (rc = dev_alloc(h, &d_first, (size_t)nt))) {
+        (rc = dev_alloc(h, &d_tp, (size_t)nt + 1)) || (rc = dev_alloc(h, &d_plan, 3 * (size_t)nt)) ||
+        (rc = dev_alloc(h, &d_in, 4 * (size_t)nt + 1))) {
         cleanup();
         return rc;
     }
@@ -1396,41 +1397,85 @@ static int device_bucket_tiles(dsfacto *h, int64_t nnz, SgdPlanBuild &pb) {
         return fail(e);
     pack_entries_kernel<<<wide_grid, kThreads, 0, st>>>(nnz, key[1], pay[1], h->jbits, h->d_ent);
     tile_bounds_kernel<<<(int)std::min<int64_t>((nt + kThreads) / kThreads, wide_grid), kThreads, 0, st>>>(nnz, key[1], h->jbits, nt, d_tp);
+    // the chunk plan: count per tile, then write.  The plain plan visits the tiles in slot order, so the kernel
+    // can write complete descriptors straight into the handle's array; a plan cut into segments (second
+    // schedule) gets the per-tile pieces and is put in order on the host as in the host path.
+    const int64_t p = h->p;
+    const bool segmented = h->sweep == 1 && h->refresh_every > 0 && h->refresh_every < p;
     TilePlanArgs pa{};
     pa.key = key[1]; pa.tile_ptr = d_tp; pa.ntiles = nt; pa.jbits = h->jbits; pa.chunk_len = h->chunk_len;
-    pa.count = d_count; pa.first = d_first; pa.out = nullptr;
-    plan_tiles_kernel<false><<<wide_grid, kThreads, 0, st>>>(pa);
+    pa.count = d_plan; pa.runs = d_plan + nt; pa.recs = d_plan + 2 * nt;
+    pa.p = h->p; pa.sweep = h->sweep; pa.row_start = h->d_row_start; pa.col_start = h->d_col_start;
+    plan_tiles_kernel<kPlanCount><<<wide_grid, kThreads, 0, st>>>(pa);
     h->launches += 4;
-    std::vector<int64_t> count;
+    std::vector<int64_t> cnt, in;   // cnt: counts, runs, recs per tile; in: first (nt + 1), need, run0, rec0
     try {
         h->tile_ptr.assign((size_t)nt + 1, 0);
-        count.resize((size_t)nt);
+        cnt.resize(3 * (size_t)nt);
+        in.resize(4 * (size_t)nt + 1);
     } catch (const std::bad_alloc &) { cudaStreamSynchronize(st); cleanup(); return DSFACTO_ERR_OOM; }
     if ((e = cudaMemcpyAsync(h->tile_ptr.data(), d_tp, sizeof(int64_t) * ((size_t)nt + 1), cudaMemcpyDeviceToHost, st)) != cudaSuccess ||
-        (e = cudaMemcpyAsync(count.data(), d_count, sizeof(int64_t) * (size_t)nt, cudaMemcpyDeviceToHost, st)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(cnt.data(), d_plan, sizeof(int64_t) * 3 * (size_t)nt, cudaMemcpyDeviceToHost, st)) != cudaSuccess ||
         (e = cudaStreamSynchronize(st)) != cudaSuccess || (e = cudaGetLastError()) != cudaSuccess)
         return fail(e);
-    // where every tile's chunks go: one planner holds them all, tile after tile
-    int64_t total = 0;
+    int64_t *first = in.data(), *need = first + nt + 1, *run0 = need + nt, *rec0 = run0 + nt;
+    int64_t total = 0, runs = 0, recs = 0;
+    std::vector<int64_t> seen;
+    try {
+        seen.assign((size_t)p, 0);
+        if (!segmented) h->launch_ptr.assign((size_t)p + 1, 0);
+    } catch (const std::bad_alloc &) { cleanup(); return DSFACTO_ERR_OOM; }
     for (int64_t t = 0; t < nt; ++t) {
+        int64_t r, c;
+        slot_tile(h, t, r, c);
         TileDescRef &ref = pb.refs[(size_t)t];
         ref.owner = 0;
         ref.first = total;
-        ref.count = (int32_t)count[(size_t)t];
-        const int64_t c = count[(size_t)t];
-        count[(size_t)t] = total;
-        total += c;
+        ref.count = (int32_t)cnt[(size_t)t];
+        first[t] = total; need[t] = seen[(size_t)c]; run0[t] = runs; rec0[t] = recs;
+        total += cnt[(size_t)t];
+        runs += cnt[(size_t)(nt + t)];
+        recs += cnt[(size_t)(2 * nt + t)];
+        seen[(size_t)c] += cnt[(size_t)t];
+        if (!segmented && (t + 1) % p == 0) h->launch_ptr[(size_t)((t + 1) / p)] = total;
     }
-    if (!pb.bulk.alloc((size_t)total)) { cleanup(); return DSFACTO_ERR_OOM; }
-    if (total > 0) {
-        if ((rc = dev_alloc(h, &d_out, (size_t)total))) { cleanup(); return rc; }
-        if ((e = cudaMemcpyAsync(d_first, count.data(), sizeof(int64_t) * (size_t)nt, cudaMemcpyHostToDevice, st)) != cudaSuccess)
+    first[nt] = total;
+    if (total >= (int64_t)kTicketStop / 2 || recs >= ((int64_t)1 << 31)) { cleanup(); return DSFACTO_ERR_INVALID_ARG; }
+    if ((e = cudaMemcpyAsync(d_in, in.data(), sizeof(int64_t) * in.size(), cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail(e);
+    pa.first = d_in; pa.need = d_in + nt + 1; pa.run0 = pa.need + nt; pa.rec0 = pa.run0 + nt;
+    if (segmented) {
+        if (!pb.bulk.alloc((size_t)total)) { cudaStreamSynchronize(st); cleanup(); return DSFACTO_ERR_OOM; }
+        if (total > 0) {
+            if ((rc = dev_alloc(h, &d_out, (size_t)total))) { cudaStreamSynchronize(st); cleanup(); return rc; }
+            pa.out = d_out;
+            plan_tiles_kernel<kPlanPieces><<<wide_grid, kThreads, 0, st>>>(pa);
+            h->launches += 1;
+            if ((e = cudaMemcpyAsync(pb.bulk.data(), d_out, sizeof(ChunkDesc) * (size_t)total, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
+                return fail(e);
+        }
+    } else {
+        // what finish_sgd_plan does for the host paths
+        h->plan_segments = 0;
+        h->total_chunks = total;
+        h->long_runs = runs;
+        h->slice_records = recs;
+        if ((rc = dev_alloc(h, &h->d_desc, (size_t)total)) ||
+            (rc = dev_alloc(h, &h->d_records, (size_t)recs * slice_record_floats(h->Kp))) ||
+            (rc = dev_alloc(h, &h->d_run_count, (size_t)runs)) || (rc = dev_alloc(h, &h->d_sync, sync_words((int)p)))) {
+            cudaStreamSynchronize(st);
+            cleanup();
+            return rc;
+        }
+        if ((e = cudaMemsetAsync(h->d_run_count, 0, sizeof(int) * (size_t)std::max<int64_t>(runs, 1), st)) != cudaSuccess ||
+            (e = cudaMemsetAsync(h->d_sync, 0, sizeof(int) * sync_words((int)p), st)) != cudaSuccess)
             return fail(e);
-        pa.out = d_out;
-        plan_tiles_kernel<true><<<wide_grid, kThreads, 0, st>>>(pa);
-        h->launches += 1;
-        if ((e = cudaMemcpyAsync(pb.bulk.data(), d_out, sizeof(ChunkDesc) * (size_t)total, cudaMemcpyDeviceToHost, st)) != cudaSuccess)
-            return fail(e);
+        if (total > 0) {
+            pa.out = h->d_desc;
+            plan_tiles_kernel<kPlanFull><<<wide_grid, kThreads, 0, st>>>(pa);
+            h->launches += 1;
+            if (h->debug_extra_need > 0) plan_extra_need_kernel<<<1, 1, 0, st>>>(h->d_desc, h->debug_extra_need);
+        }
+        pb.finished = true;
     }
     if ((e = cudaStreamSynchronize(st)) != cudaSuccess || (e = cudaGetLastError()) != cudaSuccess) return fail(e);
     cleanup();
@@ -1548,14 +1593,17 @@ static int load_validated(dsfacto_t *h, const int64_t *indptr, const int32_t *in
     }
     CU_TRY(h, cudaMemcpyAsync(h->d_tile_ptr, h->tile_ptr.data(), sizeof(int64_t) * h->tile_ptr.size(), cudaMemcpyHostToDevice, st));
     CU_TRY(h, cudaStreamSynchronize(st));
-    if ((rc = finish_sgd_plan(h, pb))) { free_data(h); return rc; }
+    if (!pb.finished && (rc = finish_sgd_plan(h, pb))) { free_data(h); return rc; }
     if ((rc = order_columns(h))) { free_data(h); return rc; }
     {
         const int64_t nt1 = (int64_t)h->p * h->p + 1, plan_bytes = (int64_t)sizeof(ChunkDesc) * h->total_chunks;
         const int64_t csr_bytes = 8 * (n + 1) + 8 * nnz + 4 * n;   // indptr, idx, val, y
+        const int64_t nt = nt1 - 1;
         h->load_info[0] = on_device ? 2 : (copy_from_host ? 0 : 1);
-        h->load_info[1] = csr_bytes + 8 * nt1 + plan_bytes + (on_device ? 8 * (nt1 - 1) : (h->wide ? 12 : 8) * nnz);
-        h->load_info[2] = on_device ? 8 * nt1 + 8 * (nt1 - 1) + plan_bytes : 0;
+        // device bucketing: the per-tile counts come back, the per-tile starting values go out; only a plan
+        // that is cut into segments sends its descriptors to the host and back
+        h->load_info[1] = csr_bytes + 8 * nt1 + (on_device ? 8 * (4 * nt + 1) + (pb.finished ? 0 : plan_bytes) : plan_bytes + (h->wide ? 12 : 8) * nnz);
+        h->load_info[2] = on_device ? 8 * nt1 + 24 * nt + (pb.finished ? 0 : plan_bytes) : 0;
     }
     h->failed = false;
     h->loaded = true;
