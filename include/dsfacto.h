@@ -72,7 +72,8 @@ int dsfacto_create(dsfacto_t **out, int64_t n, int32_t d, int32_t K, int32_t p, 
  * device has room for the buffers of a sort (about 25 bytes per stored entry for the duration of the call):
  * the CSR copy that the recompute pass needs anyway is turned into (tile, local column) keys, sorted by a
  * stable radix sort, packed into entry records, and a kernel cuts the chunks of the stratum SGD launch; only
- * the CSR arrays cross the link.  DSFACTO_LOAD=device takes this way for any non-empty load that fits the
+ * the CSR arrays cross the link, and they are sent while the host still checks them (a data set that fails
+ * the checks leaves the handle as it was, as on every path).  DSFACTO_LOAD=device takes this way for any non-empty load that fits the
  * layout.  Otherwise, and with any other value of DSFACTO_LOAD, the tile lists are built on the host; there,
  * loads of 2^24 stored entries and more (with p at least twice the number of host threads) are
  * streamed: each host thread buckets one row block at a time into page-locked staging memory and

@@ -91,3 +91,32 @@ def test_device_bucketing_gives_the_same_bits_as_the_host(monkeypatch, sweep, na
         assert np.array_equal(a, b)
     assert res[0][1] == res[1][1] and res[0][2] == res[1][2]
     assert np.array_equal(res[0][3], res[1][3]) and np.array_equal(res[0][4], res[1][4])
+
+
+def test_a_rejected_large_load_leaves_the_handle_as_it_was():
+    # from 2^24 entries on the CSR arrays travel to the device while the host still checks them; a data set
+    # that fails the checks must not replace the one the handle holds
+    wl = W.make("C4", n=600_000, p=64)
+    assert wl.nnz >= 1 << 24
+    with D.DSFacto(wl.n, wl.d, wl.K, wl.p, wl.loss, wl.lambda_w, wl.lambda_v, wl.eta, wl.init_seed) as g, \
+            D.DSFacto(wl.n, wl.d, wl.K, wl.p, wl.loss, wl.lambda_w, wl.lambda_v, wl.eta, wl.init_seed) as ref:
+        g.load_csr(wl.indptr, wl.indices, wl.values, wl.y)
+        ref.load_csr(wl.indptr, wl.indices, wl.values, wl.y)
+        assert g.last_load()[0] == 2          # bucketed on the device
+        obj0 = g.objective()
+        bad_idx = wl.indices.copy()
+        r = wl.n // 2
+        b = wl.indptr[r]
+        bad_idx[b], bad_idx[b + 1] = bad_idx[b + 1], bad_idx[b]          # one row out of order
+        assert D.dsfacto_load_csr(g._h, wl.indptr, bad_idx, wl.values, wl.y) == D.ERR_INVALID_CSR
+        bad_val = wl.values.copy()
+        bad_val[-1] = np.nan
+        assert D.dsfacto_load_csr(g._h, wl.indptr, wl.indices, bad_val, wl.y) == D.ERR_INVALID_CSR
+        bad_ptr = wl.indptr.copy()
+        bad_ptr[5] = bad_ptr[6] + 1                                      # row pointers not monotone
+        assert D.dsfacto_load_csr(g._h, bad_ptr, wl.indices, wl.values, wl.y) == D.ERR_INVALID_CSR
+        assert g.objective() == obj0
+        assert g.epoch() == ref.epoch()
+        w0a, wa, Va = g.get_params()
+        w0b, wb, Vb = ref.get_params()
+        assert w0a == w0b and np.array_equal(wa, wb) and np.array_equal(Va, Vb)
