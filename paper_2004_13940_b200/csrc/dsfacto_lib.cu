@@ -363,9 +363,11 @@ struct SgdPlanBuild {
 // otherwise the epoch is a chain of p dependent tiles per column block and is as long as p times the
 // time one tile takes, so tiles are cut into short chunks that run side by side.
 void choose_chunk_len(dsfacto *h, int64_t nnz) {
-    // Measured on the 1.755 G-entry and the 400 M-entry workloads: 384 entries for rows up to 128 bytes (512: 3 %
-    // slower, 256: 20 % slower), 256 for wider rows, whose chunks last longer (512: 15 % slower).
-    h->chunk_len = h->Kp >= 64 ? 256 : 384;
+    // Measured on the 1.755 G-entry and the 400 M-entry workloads: 416 entries for rows up to 128 bytes (a chunk
+    // costs about 6.6 k cycles whatever its length, so longer is better up to there: 320 / 352 / 384 / 400 / 416:
+    // 30.3 / 28.9 / 28.7 / 28.5 / 28.4 ms; 432 and more are slower again, 512: +5 %), 256 for wider rows, whose
+    // chunks last longer (512: 15 % slower).
+    h->chunk_len = h->Kp >= 64 ? 256 : 416;
     if (nnz / kChunkMax < (int64_t)h->sm_count * 24 * 16) h->chunk_len = 128;
     if (h->chunk_override > 0) h->chunk_len = h->chunk_override;
     if (const char *env = std::getenv("DSFACTO_CHUNK")) {
