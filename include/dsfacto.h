@@ -184,6 +184,11 @@ int dsfacto_last_epoch_ms(dsfacto_t *h, float ms[4]);
  *                             failure path above can be exercised without a fault or a hang.  0 = off.
  *   DSFACTO_DEBUG_CHUNK_LEN   (takes effect at the next dsfacto_load_csr) entries per chunk, 16 .. 512, 0 = chosen
  *                             by the load; the environment variable DSFACTO_CHUNK does the same for every handle.
+ *   DSFACTO_DEBUG_ROW_MERGE   (takes effect at the next dsfacto_load_csr that buckets on the device) row blocks per slot of
+ *                             the device entry array, 1, 2, 4 or 8 (as many of them as the 32-bit keys and records
+ *                             allow), 0 = chosen by the load: a column's entries in consecutive row blocks follow one
+ *                             another in the stratified order, so they can be stored and swept as one run.  Same
+ *                             result up to rounding; the environment variable DSFACTO_ROW_MERGE does the same.
  *   DSFACTO_DEBUG_COLUMN_ORDER (takes effect at the next dsfacto_load_csr) the device copy of the CSR that the
  *                             recompute pass reads may number the columns by frequency, most frequent first, and
  *                             the pass then reads w and V from a copy in that order (hot factor rows side by
@@ -193,7 +198,8 @@ int dsfacto_last_epoch_ms(dsfacto_t *h, float ms[4]);
  *                             or receives is renumbered.
  * The environment variable DSFACTO_SWEEP=round (read by dsfacto_create) stores and sweeps the tiles round by
  * round, exactly Algorithm 1's order, instead of row block by row block. */
-enum { DSFACTO_DEBUG_SPIN_LIMIT = 0, DSFACTO_DEBUG_EXTRA_NEED = 1, DSFACTO_DEBUG_CHUNK_LEN = 2, DSFACTO_DEBUG_COLUMN_ORDER = 3 };
+enum { DSFACTO_DEBUG_SPIN_LIMIT = 0, DSFACTO_DEBUG_EXTRA_NEED = 1, DSFACTO_DEBUG_CHUNK_LEN = 2, DSFACTO_DEBUG_COLUMN_ORDER = 3,
+       DSFACTO_DEBUG_ROW_MERGE = 4 };
 int dsfacto_debug_set(dsfacto_t *h, int32_t key, int64_t value);
 
 /* How the last dsfacto_load_csr built the tile lists: info[0] = 0 on the host with one copy, 1 on the host

@@ -46,6 +46,7 @@ struct dsfacto {
     float ms[4] = {0, 0, 0, 0};
     int64_t launches = 0;
     int sm_count = 148, device = 0;
+    int l2_bytes = 126 << 20;   // L2 cache size of the device
     std::string err;
 
     std::vector<int64_t> row_start;  // p+1
@@ -76,6 +77,8 @@ struct dsfacto {
     float4 *d_S = nullptr, *d_TS = nullptr;  // scale records of the scaled column state (zero outside the SGD phase)
     int *d_run_count = nullptr;
     int refresh_grid = 0, norm_grid = 0;
+    int rbits = 0;              // log2 of the row blocks per slot of the device entry array (device bucketing; 0: one tile per slot)
+    int row_merge = 0;          // dsfacto_debug_set: row blocks per slot wanted (0 = chosen by the load, 1, 2, 4, 8)
     int64_t load_info[3] = {0, 0, 0};   // last load: path (0 host, 1 host streamed, 2 device), bytes H2D, bytes D2H
     // Column slots of the recompute pass (per load): the device CSR holds slots (rank by frequency) instead of
     // column indices, and the pass reads w and V from copies in slot order.
@@ -250,7 +253,52 @@ void unpack_tiles(const dsfacto *h, const std::vector<int64_t> &canon_ptr, const
     }
 }
 
+// The same for a device entry array whose slots hold several row blocks (device bucketing with merged row
+// blocks): slot (slot row sr, column block c) lists, per phase, its entries by (column, row block descending,
+// row); an entry's row block follows from its row.  canon_ptr (p*p + 1) is filled here as well.
+void unpack_merged_tiles(const dsfacto *h, const uint2 *ent, std::vector<int64_t> &canon_ptr, int32_t *rows, int32_t *cols,
+                         float *vals) {
+    const int64_t p = h->p, R = (int64_t)1 << h->rbits, slot_rows = (p + R - 1) / R, nslots = slot_rows * p;
+    const uint32_t jmask = h->jbits >= 32 ? 0xFFFFFFFFu : ((1u << h->jbits) - 1u);
+    canon_ptr.assign((size_t)(p * p) + 1, 0);
+    auto tile_of = [&](int64_t slot, uint32_t il, int64_t &i) -> int64_t {
+        const int64_t rb0 = (slot_rows - 1 - slot / p) * R, c = slot % p;
+        i = h->row_start[(size_t)rb0] + il;
+        int64_t r = rb0;
+        while (r + 1 < p && i >= h->row_start[(size_t)(r + 1)]) ++r;
+        int64_t sr = c - r;
+        if (sr < 0) sr += p;
+        return sr * p + r;
+    };
+#pragma omp parallel for schedule(dynamic, 8)
+    for (int64_t slot = 0; slot < nslots; ++slot)   // (different slots hold different tiles)
+        for (int64_t q = h->tile_ptr[slot]; q < h->tile_ptr[slot + 1]; ++q) {
+            int64_t i;
+            canon_ptr[(size_t)tile_of(slot, ent[q].x >> h->jbits, i) + 1] += 1;
+        }
+    for (int64_t t = 0; t < p * p; ++t) canon_ptr[(size_t)t + 1] += canon_ptr[(size_t)t];
+    if (!rows && !cols && !vals) return;
+#pragma omp parallel for schedule(dynamic, 8)
+    for (int64_t slot = 0; slot < nslots; ++slot) {
+        int64_t off[16] = {-1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1};   // next free place of the slot's tiles, by row block
+        const int64_t rb0 = (slot_rows - 1 - slot / p) * R, c = slot % p;
+        for (int64_t q = h->tile_ptr[slot]; q < h->tile_ptr[slot + 1]; ++q) {
+            int64_t i;
+            const int64_t tile = tile_of(slot, ent[q].x >> h->jbits, i);
+            const int64_t k = tile % p - rb0;
+            if (off[k] < 0) off[k] = canon_ptr[(size_t)tile];
+            const int64_t at = off[k]++;
+            float x;
+            std::memcpy(&x, &ent[q].y, 4);
+            if (rows) rows[at] = (int32_t)i;
+            if (cols) cols[at] = (int32_t)(h->col_start[(size_t)c] + (ent[q].x & jmask));
+            if (vals) vals[at] = x;
+        }
+    }
+}
+
 void free_data(dsfacto *h) {
+    h->rbits = 0;
     dev_free(h->d_A); dev_free(h->d_G); dev_free(h->d_y); dev_free(h->d_val); dev_free(h->d_xw);
     dev_free(h->d_indptr); dev_free(h->d_tile_ptr); dev_free(h->d_idx); dev_free(h->d_ent);
     dev_free(h->d_partials); dev_free(h->d_desc); dev_free(h->d_records); dev_free(h->d_run_count);
@@ -1232,6 +1280,8 @@ static int create_handle(dsfacto_t **out, int64_t n, int32_t d, int32_t K, int32
     h->device = dev;
     cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, dev);
     if (h->sm_count < 1) h->sm_count = 148;
+    cudaDeviceGetAttribute(&h->l2_bytes, cudaDevAttrL2CacheSize, dev);
+    if (h->l2_bytes < (1 << 20)) h->l2_bytes = 126 << 20;
 
     auto fail = [&](int rc) { dsfacto_destroy(h); return rc; };
     if (setup_partition(h)) return fail(DSFACTO_ERR_OOM);
@@ -1342,7 +1392,7 @@ static int filter_columns(int64_t n, const int64_t *indptr, const int32_t *indic
 // device for the sort's buffers next to what the handle keeps.
 static bool device_bucketing_wanted(const dsfacto *h, int64_t nnz, const char *load_env) {
     if (nnz <= 0 || h->wide) return false;
-    if (bits_for((int64_t)h->p * h->p) + h->jbits > 32) return false;
+    if (bits_for((int64_t)h->p * h->p) + 1 + h->jbits > 32) return false;   // slot, phase, local column
     if (load_env) return std::strcmp(load_env, "device") == 0;
     if (nnz < kStreamedLoadMinEntries) return false;
     size_t free_b = 0, total_b = 0;
@@ -1354,9 +1404,46 @@ static bool device_bucketing_wanted(const dsfacto *h, int64_t nnz, const char *l
 
 // d_indptr, d_idx, d_val hold the CSR arrays (copies queued on the stream), d_ent is allocated.  Fills
 // d_ent, h->tile_ptr and the per-tile pieces of the launch plan.
+// Row blocks per slot (a power of two, as log2): merged row blocks make a column's runs longer (see
+// dsfacto_bucket.cuh).  Only for the plain plan of the row-block sweep on an unsharded handle; up to 8, as
+// many as keep the auxiliary rows of a slot row (re-read by every column block) within 55 % of L2, leave at
+// least 16 slot rows, and fit the 32-bit keys and entry records.  Measured sweep times, 1 / 2 / 4 / 8 / 16 row
+// blocks per slot: 1.755 G entries, 64-byte rows (45 MB of auxiliary rows per slot row at 8): 29.3 / 28.6 /
+// 26.1 / 24.5 / 26.9 ms; 400 M entries, 512-byte rows (64 MB at 8): 26.6 / 24.7 / 23.1 / 22.1 / 24.0 ms.
+static int choose_row_merge(const dsfacto *h, int64_t nnz) {
+    const int64_t p = h->p;
+    const bool segmented = h->refresh_every > 0 && h->refresh_every < p;
+    if (h->sweep != 1 || segmented || h->nshards > 1) return 0;
+    int want = 8;
+    if (h->row_merge > 0) want = h->row_merge;
+    else if (nnz < kStreamedLoadMinEntries) want = 1;
+    if (const char *env = std::getenv("DSFACTO_ROW_MERGE")) {
+        const int v = std::atoi(env);
+        if (v >= 1 && v <= 16) want = v;
+    }
+    int rbits = 0;
+    while ((2 << rbits) <= want) {
+        const int nb = rbits + 1;
+        const int64_t R = (int64_t)1 << nb, slot_rows = (p + R - 1) / R;
+        int64_t max_rows = 0;
+        for (int64_t sr = 0; sr < slot_rows; ++sr)
+            max_rows = std::max(max_rows, h->row_start[(size_t)std::min(p, (sr + 1) * R)] - h->row_start[(size_t)(sr * R)]);
+        const bool forced = h->row_merge > 0 || std::getenv("DSFACTO_ROW_MERGE") != nullptr;
+        if (bits_for(max_rows) + h->jbits > 32) break;
+        if (bits_for(slot_rows * p) + 1 + h->jbits + nb > 32) break;
+        if (!forced && (slot_rows < 16 || (double)max_rows * h->Kp * 4.0 > 0.55 * (double)h->l2_bytes)) break;
+        if (slot_rows < 1) break;
+        rbits = nb;
+    }
+    return rbits;
+}
+
 static int device_bucket_tiles(dsfacto *h, int64_t nnz, SgdPlanBuild &pb) {
-    const int64_t nt = (int64_t)h->p * h->p;
-    const int kb = bits_for(nt) + h->jbits;
+    h->rbits = choose_row_merge(h, nnz);
+    const int64_t slot_rows = ((int64_t)h->p + ((int64_t)1 << h->rbits) - 1) >> h->rbits;
+    const int64_t nt = slot_rows * h->p;                       // slots of the device entry array
+    const int low_bits = 1 + h->jbits + h->rbits;              // key bits below the slot number: phase, local column, row block
+    const int kb = bits_for(nt) + low_bits;
     cudaStream_t st = h->stream;
     uint32_t *key[2] = {nullptr, nullptr};
     unsigned long long *pay[2] = {nullptr, nullptr};
@@ -1393,12 +1480,13 @@ static int device_bucket_tiles(dsfacto *h, int64_t nnz, SgdPlanBuild &pb) {
     TileKeyArgs ka{};
     ka.n = h->n; ka.indptr = h->d_indptr; ka.idx = h->d_idx; ka.val = h->d_val; ka.d = h->d; ka.p = h->p;
     ka.sweep = h->sweep; ka.jbits = h->jbits; ka.row_start = h->d_row_start; ka.col_start = h->d_col_start;
+    ka.rbits = h->rbits; ka.slot_rows = (int32_t)slot_rows;
     ka.key = key[0]; ka.payload = pay[0];
     tile_keys_kernel<<<wide_grid, kThreads, 0, st>>>(ka);
     if ((e = cub::DeviceRadixSort::SortPairs(tmp, tmp_bytes, key[0], key[1], pay[0], pay[1], nnz, 0, kb, st)) != cudaSuccess)
         return fail(e);
-    pack_entries_kernel<<<wide_grid, kThreads, 0, st>>>(nnz, key[1], pay[1], h->jbits, h->d_ent);
-    tile_bounds_kernel<<<(int)std::min<int64_t>((nt + kThreads) / kThreads, wide_grid), kThreads, 0, st>>>(nnz, key[1], h->jbits, nt, d_tp);
+    pack_entries_kernel<<<wide_grid, kThreads, 0, st>>>(nnz, key[1], pay[1], h->jbits, h->rbits, h->d_ent);
+    tile_bounds_kernel<<<(int)std::min<int64_t>((nt + kThreads) / kThreads, wide_grid), kThreads, 0, st>>>(nnz, key[1], low_bits, nt, d_tp);
     // the chunk plan: count per tile, then write.  The plain plan visits the tiles in slot order, so the kernel
     // can write complete descriptors straight into the handle's array; a plan cut into segments (second
     // schedule) gets the per-tile pieces and is put in order on the host as in the host path.
@@ -1406,6 +1494,7 @@ static int device_bucket_tiles(dsfacto *h, int64_t nnz, SgdPlanBuild &pb) {
     const bool segmented = h->sweep == 1 && h->refresh_every > 0 && h->refresh_every < p;
     TilePlanArgs pa{};
     pa.key = key[1]; pa.tile_ptr = d_tp; pa.ntiles = nt; pa.jbits = h->jbits; pa.chunk_len = h->chunk_len;
+    pa.rbits = h->rbits; pa.slot_rows = (int32_t)slot_rows;
     pa.count = d_plan; pa.runs = d_plan + nt; pa.recs = d_plan + 2 * nt;
     pa.p = h->p; pa.sweep = h->sweep; pa.row_start = h->d_row_start; pa.col_start = h->d_col_start;
     plan_tiles_kernel<kPlanCount><<<wide_grid, kThreads, 0, st>>>(pa);
@@ -1429,7 +1518,8 @@ static int device_bucket_tiles(dsfacto *h, int64_t nnz, SgdPlanBuild &pb) {
     } catch (const std::bad_alloc &) { cleanup(); return DSFACTO_ERR_OOM; }
     for (int64_t t = 0; t < nt; ++t) {
         int64_t r, c;
-        slot_tile(h, t, r, c);
+        if (h->rbits > 0) c = t % p;   // (merged row blocks: row-block sweep, slot = slot row x column block)
+        else slot_tile(h, t, r, c);
         TileDescRef &ref = pb.refs[(size_t)t];
         ref.owner = 0;
         ref.first = total;
@@ -1439,9 +1529,12 @@ static int device_bucket_tiles(dsfacto *h, int64_t nnz, SgdPlanBuild &pb) {
         runs += cnt[(size_t)(nt + t)];
         recs += cnt[(size_t)(2 * nt + t)];
         seen[(size_t)c] += cnt[(size_t)t];
-        if (!segmented && (t + 1) % p == 0) h->launch_ptr[(size_t)((t + 1) / p)] = total;
+        if (!segmented && h->rbits == 0 && (t + 1) % p == 0) h->launch_ptr[(size_t)((t + 1) / p)] = total;
     }
     first[nt] = total;
+    // (with merged row blocks the plain plan is one launch over everything: only its two ends are looked up)
+    if (!segmented && h->rbits > 0)
+        for (int64_t k = 1; k <= p; ++k) h->launch_ptr[(size_t)k] = total;
     if (total >= (int64_t)kTicketStop / 2 || recs >= ((int64_t)1 << 31)) { cleanup(); return DSFACTO_ERR_INVALID_ARG; }
     if ((e = cudaMemcpyAsync(d_in, in.data(), sizeof(int64_t) * in.size(), cudaMemcpyHostToDevice, st)) != cudaSuccess) return fail(e);
     pa.first = d_in; pa.need = d_in + nt + 1; pa.run0 = pa.need + nt; pa.rec0 = pa.run0 + nt;
@@ -1850,9 +1943,11 @@ int dsfacto_get_tiles(dsfacto_t *h, int64_t *tile_ptr, int32_t *rows, int32_t *c
     if (!h->loaded) return DSFACTO_ERR_NO_DATA;
     const int64_t nt = (int64_t)h->p * h->p;
     std::vector<int64_t> canon;
-    try { canon = canonical_tile_ptr(h); } catch (const std::bad_alloc &) { return DSFACTO_ERR_OOM; }
-    if (tile_ptr) std::memcpy(tile_ptr, canon.data(), sizeof(int64_t) * ((size_t)nt + 1));
-    if (!rows && !cols && !vals) return DSFACTO_OK;
+    if (h->rbits == 0) {
+        try { canon = canonical_tile_ptr(h); } catch (const std::bad_alloc &) { return DSFACTO_ERR_OOM; }
+        if (tile_ptr) std::memcpy(tile_ptr, canon.data(), sizeof(int64_t) * ((size_t)nt + 1));
+        if (!rows && !cols && !vals) return DSFACTO_OK;
+    }
     HostBuf<uint2> ent;
     HostBuf<float> xw;
     if (!ent.alloc((size_t)h->nnz) || (h->wide && !xw.alloc((size_t)h->nnz))) return DSFACTO_ERR_OOM;
@@ -1860,6 +1955,11 @@ int dsfacto_get_tiles(dsfacto_t *h, int64_t *tile_ptr, int32_t *rows, int32_t *c
         CU_TRY(h, cudaMemcpyAsync(ent.data(), h->d_ent, sizeof(uint2) * (size_t)h->nnz, cudaMemcpyDeviceToHost, h->stream));
         if (h->wide) CU_TRY(h, cudaMemcpyAsync(xw.data(), h->d_xw, sizeof(float) * (size_t)h->nnz, cudaMemcpyDeviceToHost, h->stream));
         CU_TRY(h, cudaStreamSynchronize(h->stream));
+    }
+    if (h->rbits > 0) {   // (merged row blocks: the tile sizes come from the entries themselves)
+        try { unpack_merged_tiles(h, ent.data(), canon, rows, cols, vals); } catch (const std::bad_alloc &) { return DSFACTO_ERR_OOM; }
+        if (tile_ptr) std::memcpy(tile_ptr, canon.data(), sizeof(int64_t) * ((size_t)nt + 1));
+        return DSFACTO_OK;
     }
     unpack_tiles(h, canon, ent.data(), xw.data(), rows, cols, vals);
     return DSFACTO_OK;
@@ -1999,6 +2099,10 @@ int dsfacto_debug_set(dsfacto_t *h, int32_t key, int64_t value) {
     case DSFACTO_DEBUG_CHUNK_LEN:
         if (value != 0 && (value < 16 || value > kChunkMax)) return DSFACTO_ERR_INVALID_ARG;
         h->chunk_override = (int)value;
+        return DSFACTO_OK;
+    case DSFACTO_DEBUG_ROW_MERGE:
+        if (value != 0 && value != 1 && value != 2 && value != 4 && value != 8 && value != 16) return DSFACTO_ERR_INVALID_ARG;
+        h->row_merge = (int)value;
         return DSFACTO_OK;
     case DSFACTO_DEBUG_COLUMN_ORDER:
         if (value < 0 || value > 2) return DSFACTO_ERR_INVALID_ARG;

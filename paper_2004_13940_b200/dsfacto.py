@@ -135,7 +135,7 @@ def dsfacto_set_refresh_every(h, rounds):
     return lib().dsfacto_set_refresh_every(h, rounds)
 
 
-DEBUG_SPIN_LIMIT, DEBUG_EXTRA_NEED, DEBUG_CHUNK_LEN, DEBUG_COLUMN_ORDER = 0, 1, 2, 3
+DEBUG_SPIN_LIMIT, DEBUG_EXTRA_NEED, DEBUG_CHUNK_LEN, DEBUG_COLUMN_ORDER, DEBUG_ROW_MERGE = 0, 1, 2, 3, 4
 
 
 def dsfacto_debug_set(h, key, value):

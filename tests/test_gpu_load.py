@@ -120,3 +120,45 @@ def test_a_rejected_large_load_leaves_the_handle_as_it_was():
         w0a, wa, Va = g.get_params()
         w0b, wb, Vb = ref.get_params()
         assert w0a == w0b and np.array_equal(wa, wb) and np.array_equal(Va, Vb)
+
+
+@pytest.mark.parametrize("merge", [2, 4, 8])
+@pytest.mark.parametrize("name,kw", [("C1", {"p": 16}), ("C2", {}), ("C3", {}), ("C3", {"p": 7}), ("C4s", {}), ("C5s", {})])
+def test_merged_row_blocks_on_the_device(monkeypatch, merge, name, kw):
+    # Several row blocks per slot: a column's entries of consecutive row blocks are stored and swept as one
+    # run.  The canonical tile lists that come back are still the oracle's, bit for bit; the epochs are the
+    # oracle's within the tolerance (runs are cut elsewhere, so the bits differ from the one-tile-per-slot plan).
+    monkeypatch.setenv("DSFACTO_LOAD", "device")
+    monkeypatch.delenv("DSFACTO_SWEEP", raising=False)
+    wl = W.make(name, **kw)
+    keep = np.ones(wl.indices.shape[0], bool)
+    rows = np.repeat(np.arange(wl.n), np.diff(wl.indptr))
+    keep[(rows % 11) == 5] = False                       # some rows empty
+    indptr = np.concatenate([[0], np.cumsum(np.bincount(rows[keep], minlength=wl.n))]).astype(np.int64)
+    indices, values = wl.indices[keep], wl.values[keep]
+    o = O.Oracle(wl.n, wl.d, wl.K, wl.p, wl.loss, wl.lambda_w, wl.lambda_v, wl.eta, wl.init_seed)
+    o.load_csr(indptr, indices, values, wl.y)
+    with D.DSFacto(wl.n, wl.d, wl.K, wl.p, wl.loss, wl.lambda_w, wl.lambda_v, wl.eta, wl.init_seed) as g:
+        g.debug_set(D.DEBUG_ROW_MERGE, merge)
+        g.load_csr(indptr, indices, values, wl.y)
+        assert g.last_load()[0] == 2
+        tp, r, c, v = g.get_tiles()
+        assert np.array_equal(tp, o.tile_ptr)
+        assert np.array_equal(r, o.rows) and np.array_equal(c, o.cols) and np.array_equal(v, o.vals)
+        assert g.objective() == pytest.approx(o.objective, rel=1e-5)
+        for _ in range(3):
+            assert g.epoch() == pytest.approx(o.epoch(), rel=1e-4)
+        w0, w, V = g.get_params()
+        A, G = g.get_aux()
+        # the same epochs again on a second handle: the same bits
+        with D.DSFacto(wl.n, wl.d, wl.K, wl.p, wl.loss, wl.lambda_w, wl.lambda_v, wl.eta, wl.init_seed) as g2:
+            g2.debug_set(D.DEBUG_ROW_MERGE, merge)
+            g2.load_csr(indptr, indices, values, wl.y)
+            for _ in range(3):
+                g2.epoch()
+            w0b, wb, Vb = g2.get_params()
+    assert w0 == w0b and np.array_equal(w, wb) and np.array_equal(V, Vb)
+    assert abs(w0 - o.w0) <= 1e-4 * (1 + abs(o.w0))
+    assert np.abs(w - o.w).max() <= 1e-4 * (1 + np.abs(o.w).max())
+    assert np.all(np.abs(V - o.V) <= 1e-4 * (1 + np.abs(o.V)))
+    assert np.all(np.abs(G - o.G) <= 1e-4 * (1 + np.abs(o.G)))
