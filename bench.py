@@ -35,7 +35,7 @@ ORACLE_SAMPLE_ROWS = 1_000_000
 # dram__bytes_read.sum + dram__bytes_write.sum of sgd_sweep_kernel per stored entry, by factor width K, from
 # the ncu captures summarised in profiles/ (scaled cases; DRAM traffic of the sweep grows with the entries).
 # A width without a capture of the current kernel reports traffic = null.
-SGD_DRAM_BYTES_PER_ENTRY = {16: 19.2, 128: 247.0}
+SGD_DRAM_BYTES_PER_ENTRY = {16: 22.0, 128: 186.0}
 
 
 def peaks():
