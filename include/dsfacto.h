@@ -182,8 +182,10 @@ int dsfacto_last_epoch_ms(dsfacto_t *h, float ms[4]);
  *                             wait for that many finished chunks more than its column block really has before
  *                             it; with a value larger than the number of chunks its wait runs out, so the
  *                             failure path above can be exercised without a fault or a hang.  0 = off.
- *   DSFACTO_DEBUG_CHUNK_LEN   (takes effect at the next dsfacto_load_csr) entries per chunk, 16 .. 512, 0 = chosen
+ *   DSFACTO_DEBUG_CHUNK_LEN   (takes effect at the next dsfacto_load_csr) entries per chunk, 16 .. 4096, 0 = chosen
  *                             by the load; the environment variable DSFACTO_CHUNK does the same for every handle.
+ *                             The sweep kernel reads a chunk's entries block by block; the environment variable
+ *                             DSFACTO_BLOCK (a multiple of 32, 32 .. 256) sets the entries per block.
  *   DSFACTO_DEBUG_ROW_MERGE   (takes effect at the next dsfacto_load_csr that buckets on the device) row blocks per slot of
  *                             the device entry array, 1, 2, 4 or 8 (as many of them as the 32-bit keys and records
  *                             allow), 0 = chosen by the load: a column's entries in consecutive row blocks follow one

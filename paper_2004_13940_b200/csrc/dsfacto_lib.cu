@@ -67,7 +67,8 @@ struct dsfacto {
     ChunkDesc *d_desc = nullptr;   // chunk descriptors in sweep order
     int *d_sync = nullptr;     // ticket, error word, per-column-block progress of the fused SGD launch
     int64_t total_chunks = 0, long_runs = 0, slice_records = 0;
-    int chunk_len = kChunkMax;  // most entries a chunk of the stratum SGD launches holds
+    int chunk_len = 512;        // most entries a chunk of the stratum SGD launches holds
+    int block_len = 128;        // entries per block of the kernel's entry ring
     int chunk_override = 0;     // > 0: chunk length forced by dsfacto_debug_set (tests)
     int sgd_grid = 0;           // CTAs of the persistent stratum SGD launch
     int spin_limit = kSgdSpinLimit;  // polls before a wait for an earlier tile gives up
@@ -317,7 +318,7 @@ void free_data(dsfacto *h) {
 // ---------------------------------------------------------------------------------------------
 template <int LG, int NV>
 void launch_sgd(dsfacto *h, const SgdArgs &a, int64_t chunks) {
-    const size_t bytes = (size_t)kSgdWarps * sgd_warp_smem<LG, NV>(h->wide, h->chunk_len);
+    const size_t bytes = (size_t)kSgdWarps * sgd_warp_smem<LG, NV>(h->wide, h->block_len);
     // The launch is persistent: as many CTAs as stay resident (fewer if there are fewer chunks), each warp
     // taking chunks from the ticket counter until none is left.  More than 48 KB of dynamic shared memory
     // needs an opt-in per kernel; the residency depends on the chunk length, so both are redone per load.
@@ -407,20 +408,29 @@ struct SgdPlanBuild {
     std::vector<TileDescRef> refs;   // per tile slot
 };
 
-// Chunk length: kChunkMax when the data set keeps the GPU busy for many rounds of resident warps;
+// Chunk length: long chunks when the data set keeps the GPU busy for many rounds of resident warps;
 // otherwise the epoch is a chain of p dependent tiles per column block and is as long as p times the
 // time one tile takes, so tiles are cut into short chunks that run side by side.
 void choose_chunk_len(dsfacto *h, int64_t nnz) {
-    // Measured on the 1.755 G-entry and the 400 M-entry workloads: 416 entries for rows up to 128 bytes (a chunk
-    // costs about 6.6 k cycles whatever its length, so longer is better up to there: 320 / 352 / 384 / 400 / 416:
-    // 30.3 / 28.9 / 28.7 / 28.5 / 28.4 ms; 432 and more are slower again, 512: +5 %), 256 for wider rows, whose
-    // chunks last longer (512: 15 % slower).
-    h->chunk_len = h->Kp >= 64 ? 256 : 416;
-    if (nnz / kChunkMax < (int64_t)h->sm_count * 24 * 16) h->chunk_len = 128;
+    // A chunk costs about 6.6 k cycles whatever its length (first requests, join of the lane groups, record,
+    // fence, counters), and the kernel reads a chunk's entries through a ring of blocks, so its shared memory
+    // does not limit the length.  Measured sweeps, slots of 8 row blocks: 1.755 G entries with 64-byte rows,
+    // 416 / 832 / 1248 / 1664 / 2080 / 3328 entries: 25.0 / 22.7 / 22.0 / 21.8 / 21.6 / 21.9 ms; 400 M entries
+    // with 512-byte rows, 256 / 832 / 1664 / 2496 / 3328: 29.6 / 23.4 / 21.6 / 21.5 / 21.8 ms.
+    h->chunk_len = 2048;
+    if (nnz / 512 < (int64_t)h->sm_count * 24 * 16) h->chunk_len = 128;
     if (h->chunk_override > 0) h->chunk_len = h->chunk_override;
     if (const char *env = std::getenv("DSFACTO_CHUNK")) {
         const int v = std::atoi(env);
         if (v >= 16 && v <= kChunkMax) h->chunk_len = v;
+    }
+    // the kernel streams a chunk's entries through a ring of blocks: a whole chunk per block when it is short
+    // (blocks of 96 / 128 / 192 / 256 entries with 64-byte rows: 22.5 / 22.0 / 21.7 / 22.1 ms; wide rows leave less
+    // shared memory: 64 / 96 / 128 entries with 512-byte rows: 21.5 / 21.3 / 21.8 ms)
+    h->block_len = std::min(h->Kp >= 64 ? kEntBlockWide : kEntBlockDefault, (h->chunk_len + 31) & ~31);
+    if (const char *env = std::getenv("DSFACTO_BLOCK")) {
+        const int v = std::atoi(env);
+        if (v >= 32 && v <= kEntBlockMax && v % 32 == 0) h->block_len = v;
     }
     h->sgd_grid = 0;   // residency is recomputed at the next launch
 }
@@ -619,7 +629,7 @@ void run_sgd_phase(dsfacto *h, int64_t L0, int64_t L1) {
     a.ent = h->d_ent; a.xw = h->d_xw; a.A = h->d_A; a.G = h->d_G; a.w = h->d_w; a.V = h->d_V;
     a.S = h->d_S; a.Tb = h->d_Tb; a.Tw = h->d_Tw; a.TS = h->d_TS; a.records = h->d_records;
     a.run_count = h->d_run_count;
-    a.n = h->n; a.d = h->d; a.jbits = h->jbits; a.chunk_len = h->chunk_len; a.spin_limit = h->spin_limit;
+    a.n = h->n; a.d = h->d; a.jbits = h->jbits; a.chunk_len = h->chunk_len; a.block_len = h->block_len; a.spin_limit = h->spin_limit;
     a.h = h->h; a.lambda_v = h->lambda_v;
     const double ew = (double)h->h * (double)h->lambda_w;
     const double log1m_ew = std::log1p(-ew);           // log(1 - ew); -inf / NaN for absurd steps, which then diverge

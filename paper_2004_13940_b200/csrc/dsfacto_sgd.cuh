@@ -31,7 +31,11 @@ namespace dsf {
 
 constexpr int kSgdWarps = 1;                      // warps per CTA; every warp works on its own chunks
 constexpr int kSgdThreads = 32 * kSgdWarps;
-constexpr int kChunkMax = 512;                    // most entries a chunk may hold
+constexpr int kChunkMax = 4096;                   // most entries a chunk may hold
+constexpr int kEntBlockMax = 256;                 // most entries of one block of the entry ring (a multiple of 32)
+constexpr int kEntBlockDefault = 192;             // entries per block unless the chunks are shorter
+constexpr int kEntBlockWide = 96;                 // ... for factor rows of 256 bytes and more
+constexpr int kEntSlots = 3;                      // blocks the entry ring of a warp holds
 constexpr int kSgdSpinLimit = 1 << 22;            // polls (200 ns of sleep plus a read from L2 each) before a dependency wait gives up
 constexpr int kCopySpinLimit = 1 << 24;           // polls before the wait for a bulk copy into shared memory gives up
 constexpr int kTicketStop = 0x40000000;           // ticket counter value that makes every warp leave
@@ -83,12 +87,14 @@ struct SgdCfg {
     static constexpr int ROW4 = NBUF * RST * KP4;    // float4s of the row ring
     static constexpr int DG = SP == 1 ? PD : 1;      // passes ahead at which G_i and the scale records are requested
 };
-// entries the staging buffer of one chunk holds: the copy starts and ends on multiples of 4 entries
-__host__ __device__ constexpr int sgd_ecap(int chunk_len) { return (chunk_len + 8 + 3) & ~3; }
+// entries one slot of the entry ring holds: a block of block_len entries, the four entries before it (a block
+// that is not the first of its chunk brings the entry before its first one along) and the rounding of the
+// copy's start and end to multiples of 4 entries
+__host__ __device__ constexpr int sgd_ecap(int block_len) { return (block_len + 12 + 3) & ~3; }
 template <int LG, int NV>
-__host__ __device__ constexpr size_t sgd_warp_smem(bool wide, int chunk_len) {
-    return (size_t)SgdCfg<LG, NV>::ROW4 * 16 + 32 * 8 + 32 * 4 + 40 * 4 + 16 +
-           (size_t)2 * sgd_ecap(chunk_len) * (wide ? 12 : 8);
+__host__ __device__ constexpr size_t sgd_warp_smem(bool wide, int block_len) {
+    return (size_t)SgdCfg<LG, NV>::ROW4 * 16 + 32 * 8 + 32 * 4 + 40 * 4 + 32 +
+           (size_t)kEntSlots * sgd_ecap(block_len) * (wide ? 12 : 8);
 }
 // floats of the record a slice of a long run leaves: {D, m, W, -} and the K-wide sum
 __host__ __device__ constexpr int slice_record_floats(int Kp) { return 4 + Kp; }
@@ -172,7 +178,8 @@ struct SgdArgs {
                                // launches of one sweep)
     int64_t n, d;              // rows and columns of the data set (checks of the debug build)
     int jbits;
-    int chunk_len;             // longest chunk of the plan (sizes the staging buffers)
+    int chunk_len;             // longest chunk of the plan
+    int block_len;             // entries per block of the entry ring: a multiple of 32, at most kEntBlockMax
     int spin_limit;            // polls before the wait for an earlier tile gives up
     float h, lambda_v;
     float kappa_w;             // -log2(1 - ew): (1 - ew)^{-m} = 2^(m kappa_w)
@@ -198,10 +205,12 @@ struct SgdArgs {
 // ------------------------------------------------------------------------------------------
 // sgd_sweep_kernel: persistent warps; each takes chunks in sweep order from a ticket counter.
 //
-// Pipeline of a warp: while chunk n is worked on, the ticket of chunk n+1 is drawn, its descriptor is
-// loaded and its entry records are copied into shared memory (one bulk copy, completion on an
-// mbarrier).  A chunk is walked in passes of 32 entries, one entry per lane for the scalar
-// part:
+// Pipeline of a warp: while chunk n is worked on, the ticket of chunk n+1 is drawn and its descriptor is
+// loaded.  Entry records reach shared memory block by block through a ring of three slots (one bulk copy
+// per block, completion on the slot's mbarrier): the blocks of the chunk at work two ahead of the passes,
+// then the first blocks of chunk n+1, so a chunk may be much longer than a warp's shared memory and its
+// fixed cost is spread over thousands of entries.  A chunk is walked in passes of 32 entries, one entry
+// per lane for the scalar part:
 //   scalar stage   G_i (requested one pass ahead) -> e, b; run boundaries by comparing neighbours;
 //                  segmented scan of D = P - 1 over the lanes; coefficient c = b / P and the w
 //                  coefficient; for every run that starts in the pass the scale record of its column
@@ -242,19 +251,20 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane / LG, l = lane % LG;
-    const int ecap = sgd_ecap(a.chunk_len);
-    unsigned char *wbase = smem_raw + (size_t)warp * sgd_warp_smem<LG, NV>(WIDE, a.chunk_len);
+    const int EB = a.block_len, PB = a.block_len >> 5;   // entries and passes per block of the entry ring
+    const int ecap = sgd_ecap(EB);
+    unsigned char *wbase = smem_raw + (size_t)warp * sgd_warp_smem<LG, NV>(WIDE, EB);
     float4 *rowb = reinterpret_cast<float4 *>(wbase);               // ring of row stages
     float2 *pc = reinterpret_cast<float2 *>(rowb + C::ROW4);        // per entry of the pass: {c, cw}
     uint32_t *pcol = reinterpret_cast<uint32_t *>(pc + 32);         // per entry of the pass: local column
     int *segpos = reinterpret_cast<int *>(pcol + 32);               // lane of the k-th run start of the pass (33 used)
-    uint64_t *mbar = reinterpret_cast<uint64_t *>(segpos + 40);     // one per entry buffer
-    uint2 *ebuf = reinterpret_cast<uint2 *>(mbar + 2);              // 2 x ecap entry records
-    float *xbuf = reinterpret_cast<float *>(ebuf + 2 * (size_t)ecap);  // wide layout: 2 x ecap values
+    uint64_t *mbar = reinterpret_cast<uint64_t *>(segpos + 40);     // one per slot of the entry ring (4 words reserved)
+    uint2 *ebuf = reinterpret_cast<uint2 *>(mbar + 4);              // kEntSlots x ecap entry records
+    float *xbuf = reinterpret_cast<float *>(ebuf + kEntSlots * (size_t)ecap);  // wide layout: kEntSlots x ecap values
 
     if (lane == 0) {
-        mbar_init(mbar + 0, 1);
-        mbar_init(mbar + 1, 1);
+#pragma unroll
+        for (int q = 0; q < kEntSlots; ++q) mbar_init(mbar + q, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncwarp();
@@ -276,18 +286,46 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
         if ((unsigned)tk < nch && lane < 16) v = __ldg(dints + (size_t)tk * 16 + lane);
         return v;
     };
-    auto issue_entries = [&](int64_t off, int len, int buf) {
-        const int64_t a0 = off & ~(int64_t)3;
-        const int cnt4 = (int)(((off + len + 3) & ~(int64_t)3) - a0);
+    // Entry ring.  The entries of a warp's chunks arrive as a stream of blocks of EB entries (the last block of a
+    // chunk may be shorter), each with one bulk copy into the next of kEntSlots slots, so a chunk may be far
+    // longer than the shared memory of a warp.  Block b > 0 of a chunk starts four entries early: the entry
+    // before its first one (whose column tells whether a run starts there) sits in the same slot.  Stream
+    // numbers count the blocks of this warp; q0 is the number of block 0 of the chunk at work.
+    int q0 = 0, q_fetch = -1, q_issued = 0;   // block 0 of the chunk; the block the passes read; blocks requested
+    int f_slot = 0, i_slot = 0;               // slot of the next block to read / to request
+    unsigned parity_bits = 0;                 // bit s: parity the next wait on slot s expects
+    int64_t off = 0, off1 = 0;                // first entry of the chunk at work / of the next chunk
+    int len = 0, len1 = 0, nb = 0, nb1 = 0;   // their lengths and numbers of blocks
+    bool have_next = false;                   // the next chunk's descriptor has arrived
+    auto issue_block = [&](int64_t coff, int clen, int b, int slot) {
+        const int64_t g0 = coff + (int64_t)b * EB;
+        const int blen = clen - b * EB < EB ? clen - b * EB : EB;
+        const int64_t a0 = (g0 & ~(int64_t)3) - (b > 0 ? 4 : 0);
+        const int cnt4 = (int)(((g0 + blen + 3) & ~(int64_t)3) - a0);
         if (lane == 0) {
-            mbar_expect_tx(mbar + buf, (unsigned)cnt4 * (WIDE ? 12u : 8u));
-            bulk_copy_g2s(ebuf + (size_t)buf * ecap, a.ent + a0, (unsigned)cnt4 * 8u, mbar + buf);
-            if (WIDE) bulk_copy_g2s(xbuf + (size_t)buf * ecap, a.xw + a0, (unsigned)cnt4 * 4u, mbar + buf);
+            mbar_expect_tx(mbar + slot, (unsigned)cnt4 * (WIDE ? 12u : 8u));
+            bulk_copy_g2s(ebuf + (size_t)slot * ecap, a.ent + a0, (unsigned)cnt4 * 8u, mbar + slot);
+            if (WIDE) bulk_copy_g2s(xbuf + (size_t)slot * ecap, a.xw + a0, (unsigned)cnt4 * 4u, mbar + slot);
         }
     };
-    auto wait_entries = [&](int buf, unsigned parity) -> bool {
+    // requests every block that is known (the rest of the chunk at work, then the next chunk's) and has a free
+    // slot: the slots of the blocks before q_fetch are free.  All lanes have read those blocks (callers
+    // synchronise the warp first).
+    auto pump = [&]() {
+        while (q_issued < q_fetch + kEntSlots) {
+            const int rel = q_issued - q0;
+            if (rel < nb) issue_block(off, len, rel, i_slot);
+            else if (have_next && rel - nb < nb1) issue_block(off1, len1, rel - nb, i_slot);
+            else break;
+            ++q_issued;
+            i_slot = (i_slot + 1 == kEntSlots) ? 0 : i_slot + 1;
+        }
+    };
+    auto wait_slot = [&](int slot) -> bool {
+        const unsigned parity = (parity_bits >> slot) & 1u;
+        parity_bits ^= 1u << slot;
         for (int spin = 0; spin < kCopySpinLimit; ++spin)
-            if (mbar_try_wait(mbar + buf, parity)) return true;
+            if (mbar_try_wait(mbar + slot, parity)) return true;
         return false;
     };
     auto fail = [&](int code) {
@@ -318,19 +356,15 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
     if ((unsigned)tk0 >= nch) return;
     int dc = load_desc(tk0);
     int tk1 = kTicketStop, dn = 0, tk1_raw = 0, dep_seen_next = 0, cb1 = 0;
-    int buf = 0;
-    unsigned parity_bits = 0;   // bit b: parity the next wait on buffer b expects
-    bool pending_next = false;  // a bulk copy into the other buffer is under way
     int dep_seen = 0;           // lane 0: the progress counter of the chunk's column block, read ahead
-    {
-        const int64_t off = ((int64_t)(uint32_t)__shfl_sync(FULL, dc, 0)) | ((int64_t)__shfl_sync(FULL, dc, 1) << 32);
-        issue_entries(off, __shfl_sync(FULL, dc, 2), 0);
-    }
+    bool dead = false;          // a wait for entry records ran out
 
     for (;;) {
         // ---- fields of the current chunk ----
-        const int64_t off = ((int64_t)(uint32_t)__shfl_sync(FULL, dc, 0)) | ((int64_t)__shfl_sync(FULL, dc, 1) << 32);
-        const int len = __shfl_sync(FULL, dc, 2);
+        off = ((int64_t)(uint32_t)__shfl_sync(FULL, dc, 0)) | ((int64_t)__shfl_sync(FULL, dc, 1) << 32);
+        len = __shfl_sync(FULL, dc, 2);
+        nb = (len + EB - 1) / EB;
+        have_next = false;
         const int flags = __shfl_sync(FULL, dc, 3);
         const int row0 = __shfl_sync(FULL, dc, 4);
         const int col0 = __shfl_sync(FULL, dc, 5);
@@ -341,14 +375,24 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
 
         // the ticket of the next chunk is asked for now; its descriptor and entries follow during the passes
         tk1_raw = take_ticket();
-        pending_next = false;
-        bool ok = wait_entries(buf, (parity_bits >> buf) & 1u);
-        parity_bits ^= 1u << buf;
-        if (!ok) { fail(2); break; }
 
         const int shift = (int)(off & 3);
-        const uint2 *eb = ebuf + (size_t)buf * ecap + shift;
-        const float *xb = xbuf + (size_t)buf * ecap + shift;
+        const uint2 *eb = ebuf;      // entry `at` of the chunk is eb[at] while the passes read its block
+        const float *xb = xbuf;
+        int f_next_at = 0;           // pass whose entries are the first of the next block
+        // the passes move on to the next block of the chunk: its slot is waited for, blocks further on are requested
+        auto enter_block = [&]() {
+            ++q_fetch;
+            const int b = q_fetch - q0;
+            __syncwarp();
+            pump();
+            if (!wait_slot(f_slot)) dead = true;
+            const int at0 = shift + (b > 0 ? 4 : 0) - b * EB;
+            eb = ebuf + (size_t)f_slot * ecap + at0;
+            xb = xbuf + (size_t)f_slot * ecap + at0;
+            f_slot = (f_slot + 1 == kEntSlots) ? 0 : f_slot + 1;
+            f_next_at += PB;
+        };
         const float4 *A4r = A4 + (size_t)row0 * KP4;
         const float *Gr = a.G + row0;
         float4 *U4 = reinterpret_cast<float4 *>(tail_mode ? a.Tb : a.V) + (size_t)col0 * KP4;
@@ -400,7 +444,8 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
             bool bnd = false;
             uint32_t il = 0;
             g_out = 0.f; x_out = 0.f; jl = kNoCol;
-            if (at < len) {
+            if (k == f_next_at) enter_block();
+            if (at < len && !dead) {
                 const uint2 rec = eb[at];
                 uint32_t prevj = col_init;
                 if (WIDE) { il = rec.x; jl = rec.y; x_out = xb[at]; }
@@ -468,6 +513,7 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
             il_c = il_n;
             uint32_t il_f = 0;
             if (k + DG < npass) il_f = fetch_pass(k + DG, gq[DG - 1], scq[DG - 1], mq[DG - 1], jq[DG - 1], xq[DG - 1]);
+            if (dead) break;
             if (SP > 1) il_n = il_f;
 
             // ---- scalar stage ----
@@ -613,15 +659,17 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
                 dn = load_desc(tk1);
             }
             if (k == (npass > 2 ? 2 : npass - 1) && (unsigned)tk1 < nch) {
-                const int64_t off1 = ((int64_t)(uint32_t)__shfl_sync(FULL, dn, 0)) | ((int64_t)__shfl_sync(FULL, dn, 1) << 32);
-                const int len1 = __shfl_sync(FULL, dn, 2);
+                off1 = ((int64_t)(uint32_t)__shfl_sync(FULL, dn, 0)) | ((int64_t)__shfl_sync(FULL, dn, 1) << 32);
+                len1 = __shfl_sync(FULL, dn, 2);
+                nb1 = (len1 + EB - 1) / EB;
                 cb1 = __shfl_sync(FULL, dn, 6);
+                have_next = true;
                 __syncwarp();
-                issue_entries(off1, len1, buf ^ 1);   // the other buffer's last reader was the chunk before this one
-                pending_next = true;
+                pump();   // the next chunk's first blocks, if slots are free; else they follow as the passes move on
             }
         }
         cp_async_wait<0>();
+        if (dead) { fail(2); break; }
 
         // ---- end of the chunk ----
         reduce_groups(acc, accw);
@@ -726,15 +774,20 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
         }
 
         // ---- next chunk ----
-        if ((unsigned)tk1 >= nch) { pending_next = false; break; }
+        if ((unsigned)tk1 >= nch) break;
         dc = dn;
         tk0 = tk1;
         dep_seen = dep_seen_next;
-        buf ^= 1;
+        q0 += nb;
     }
-    // leaving early: nothing may still be on its way into this warp's shared memory
+    // leaving: nothing may still be on its way into this warp's shared memory (blocks that were requested
+    // and never read: only when a wait ran out)
     cp_async_wait<0>();
-    if (pending_next) wait_entries(buf ^ 1, (parity_bits >> (buf ^ 1)) & 1u);
+    while (q_fetch + 1 < q_issued) {
+        ++q_fetch;
+        wait_slot(f_slot);
+        f_slot = (f_slot + 1 == kEntSlots) ? 0 : f_slot + 1;
+    }
 }
 
 // End of the SGD phase: back from the scaled state to plain parameters,

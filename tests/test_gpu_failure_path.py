@@ -53,7 +53,7 @@ def test_debug_knobs_reject_bad_values():
     with D.DSFacto(wl.n, wl.d, wl.K, wl.p, wl.loss, wl.lambda_w, wl.lambda_v, wl.eta, wl.init_seed) as g:
         assert D.dsfacto_debug_set(g._h, D.DEBUG_SPIN_LIMIT, 0) == D.ERR_INVALID_ARG
         assert D.dsfacto_debug_set(g._h, D.DEBUG_CHUNK_LEN, 7) == D.ERR_INVALID_ARG
-        assert D.dsfacto_debug_set(g._h, D.DEBUG_CHUNK_LEN, 513) == D.ERR_INVALID_ARG
+        assert D.dsfacto_debug_set(g._h, D.DEBUG_CHUNK_LEN, 4097) == D.ERR_INVALID_ARG
         assert D.dsfacto_debug_set(g._h, 99, 1) == D.ERR_INVALID_ARG
         assert D.dsfacto_debug_set(g._h, D.DEBUG_CHUNK_LEN, 64) == D.OK
         g.load_csr(wl.indptr, wl.indices, wl.values, wl.y)

@@ -271,13 +271,18 @@ def test_status_codes_on_device():
     g.close()
 
 
-@pytest.mark.parametrize("chunk", [16, 100, 200, 512])
+@pytest.mark.parametrize("chunk,block", [(16, 0), (100, 0), (200, 0), (512, 0), (1000, 0), (4096, 0),
+                                         (100, 32), (416, 32), (1000, 64), (2048, 256)])
 @pytest.mark.parametrize("name", ["C3", "C4s", "C5s"])
-def test_any_chunk_length_gives_the_same_epoch(monkeypatch, name, chunk):
+def test_any_chunk_length_gives_the_same_epoch(monkeypatch, name, chunk, block):
     # the chunk length of the stratum SGD launches is a tuning parameter (DSFACTO_CHUNK overrides the
     # choice made at load time): whole passes, partial passes and chunks shorter than a pass must all
-    # reproduce the oracle's epoch
+    # reproduce the oracle's epoch.  The kernel reads a chunk's entries through a ring of blocks
+    # (DSFACTO_BLOCK entries each, 192 unless the chunks are shorter): chunks of one block, of a few and of
+    # more blocks than the ring has slots, blocks of a single pass, a last block of a few entries.
     monkeypatch.setenv("DSFACTO_CHUNK", str(chunk))
+    if block:
+        monkeypatch.setenv("DSFACTO_BLOCK", str(block))
     wl = W.make(name)
     o, g = make_pair(wl)
     for _ in range(2):
