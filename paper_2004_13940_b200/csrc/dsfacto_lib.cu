@@ -411,14 +411,27 @@ struct SgdPlanBuild {
 // Chunk length: long chunks when the data set keeps the GPU busy for many rounds of resident warps;
 // otherwise the epoch is a chain of p dependent tiles per column block and is as long as p times the
 // time one tile takes, so tiles are cut into short chunks that run side by side.
-void choose_chunk_len(dsfacto *h, int64_t nnz) {
+void choose_chunk_len(dsfacto *h, int64_t nnz, int64_t slot_rows) {
     // A chunk costs about 6.6 k cycles whatever its length (first requests, join of the lane groups, record,
     // fence, counters), and the kernel reads a chunk's entries through a ring of blocks, so its shared memory
     // does not limit the length.  Measured sweeps, slots of 8 row blocks: 1.755 G entries with 64-byte rows,
     // 416 / 832 / 1248 / 1664 / 2080 / 3328 entries: 25.0 / 22.7 / 22.0 / 21.8 / 21.6 / 21.9 ms; 400 M entries
     // with 512-byte rows, 256 / 832 / 1664 / 2496 / 3328: 29.6 / 23.4 / 21.6 / 21.5 / 21.8 ms.
+    // A tile waits for the tile above it in its column block, which lies one slot row (slot_rows of them share
+    // the entries) earlier in ticket order: a slot row must hold a few times as many chunks as warps are
+    // resident, or the warps wait (scaled cases of a tenth of the entries with 2048-entry chunks: +3 % and +47 %).
     h->chunk_len = 2048;
+    {
+        const int64_t warps = (int64_t)h->sm_count * (h->Kp >= 64 ? 10 : 20);
+        const int64_t fit = (nnz / std::max<int64_t>(slot_rows, 1) / (3 * warps)) & ~(int64_t)31;
+        h->chunk_len = (int)std::min<int64_t>(2048, std::max<int64_t>(128, fit));
+    }
     if (nnz / 512 < (int64_t)h->sm_count * 24 * 16) h->chunk_len = 128;
+    // A plan cut into segments visits every row block with a fraction of its tiles, so the tiles of a column
+    // block follow one another closely in ticket order and long chunks leave the warps waiting for the tile
+    // above: 1.755 G entries in four segments, 64 / 96 / 128 / 160 / 256 / 416 / 2048 entries: 56 / 45 / 41 / 43 /
+    // 55 / 74 / 218 ms for the four launches together.
+    if (h->refresh_every > 0 && h->refresh_every < h->p) h->chunk_len = 128;
     if (h->chunk_override > 0) h->chunk_len = h->chunk_override;
     if (const char *env = std::getenv("DSFACTO_CHUNK")) {
         const int v = std::atoi(env);
@@ -1451,6 +1464,7 @@ static int choose_row_merge(const dsfacto *h, int64_t nnz) {
 static int device_bucket_tiles(dsfacto *h, int64_t nnz, SgdPlanBuild &pb) {
     h->rbits = choose_row_merge(h, nnz);
     const int64_t slot_rows = ((int64_t)h->p + ((int64_t)1 << h->rbits) - 1) >> h->rbits;
+    choose_chunk_len(h, nnz, slot_rows);   // merged row blocks: fewer and longer slot rows
     const int64_t nt = slot_rows * h->p;                       // slots of the device entry array
     const int low_bits = 1 + h->jbits + h->rbits;              // key bits below the slot number: phase, local column, row block
     const int kb = bits_for(nt) + low_bits;
@@ -1691,7 +1705,7 @@ static int load_validated(dsfacto_t *h, const int64_t *indptr, const int32_t *in
     HostBuf<float> xw;
     std::vector<int32_t> cb;
     int64_t longest = 0;
-    choose_chunk_len(h, nnz);
+    choose_chunk_len(h, nnz, h->p);
     SgdPlanBuild pb;   // the chunks of the stratum SGD launches are cut while the tiles are bucketed
     if (!init_plan_build(h, pb, omp_get_max_threads())) { cudaStreamSynchronize(st); free_data(h); return DSFACTO_ERR_OOM; }
     const bool by_row_block = use_row_block_bucketer(h);

@@ -25,6 +25,7 @@
 // breaks down only if some 1 + sigma reaches zero, i.e. a step so large that a run wipes its column;
 // the parameters then become non-finite and the epoch reports divergence.
 #pragma once
+#include <type_traits>
 #include "dsfacto_common.cuh"
 
 namespace dsf {
@@ -242,8 +243,12 @@ struct SgdArgs {
 // c, .., 0, p-1, .., c+1.  Meanwhile all entries of a row meet close together in time, so (a_i, G_i)
 // come from L2 after first touch.
 // ------------------------------------------------------------------------------------------
+// (Rows up to 128 bytes: the two copies of the pass loop would take 116 registers; held to 96, a few bytes of
+// spills, 21 instead of 17 resident warps: 22.1 -> 20.4 ms per sweep of 1.755 G entries.  Wider rows are
+// slower with that cap: 19.3 -> 20.9 ms on 400 M entries with 512-byte rows; they are held to 128 registers, as
+// more registers cost more than the few spilled bytes: 190 registers 22.5 ms.)
 template <int LG, int NV, bool WIDE>
-__global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a) {
+__global__ void __launch_bounds__(kSgdThreads, (LG * NV <= 8 ? 18 : 16)) sgd_sweep_kernel(const SgdArgs a) {
     typedef SgdCfg<LG, NV> C;
     constexpr int GW = C::GW, KP4 = C::KP4, RST = C::RST, SP = C::SP, NBUF = C::NBUF, PD = C::PD, DG = C::DG;
     constexpr unsigned FULL = 0xFFFFFFFFu;
@@ -431,67 +436,6 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
         const int npass = (len + 31) >> 5;
         const int nstage = (len + RST - 1) / RST;
         const uint32_t col_init = is_slice ? (uint32_t)__shfl_sync(FULL, dc, 14) : kNoCol;
-        // What a pass needs from global memory is requested ahead of time.  Scalars (G_i of every entry, the scale
-        // record of every column whose run starts in the pass) come DG passes ahead into a queue of registers;
-        // the rows a_i come PD stages ahead with cp.async into the row ring, one commit group per stage.
-        float gq[DG], xq[DG];
-        uint32_t jq[DG];
-        float4 scq[DG];
-        uint32_t mq[DG];                     // run starts of the pass as a lane mask
-        uint32_t il_c = 0, il_n = 0;         // local rows (one per lane) of the pass at work and of the next one
-        auto fetch_pass = [&](int k, float &g_out, float4 &sc_out, uint32_t &mask_out, uint32_t &jl, float &x_out) -> uint32_t {
-            const int at = 32 * k + lane;
-            bool bnd = false;
-            uint32_t il = 0;
-            g_out = 0.f; x_out = 0.f; jl = kNoCol;
-            if (k == f_next_at) enter_block();
-            if (at < len && !dead) {
-                const uint2 rec = eb[at];
-                uint32_t prevj = col_init;
-                if (WIDE) { il = rec.x; jl = rec.y; x_out = xb[at]; }
-                else { il = rec.x >> a.jbits; jl = rec.x & jmask; x_out = __uint_as_float(rec.y); }
-                if (at > 0) prevj = WIDE ? eb[at - 1].y : (eb[at - 1].x & jmask);
-                bnd = jl != prevj;
-                DSF_CHECK((int64_t)row0 + il < a.n, 13, il);
-                g_out = __ldg(Gr + il);
-                if (bnd) sc_out = __ldcg(Sc + jl);
-            }
-            mask_out = __ballot_sync(FULL, bnd);
-            return il;
-        };
-        // rows of stage sp of a pass whose local rows are `il`: lane group q fetches the row of entry
-        // sp*RST + it*GW + q, 16 bytes per lane (rows past the end of the chunk repeat row 0 of the block)
-        int ring_issue = 0, ring_use = 0;     // row ring: slot of the next stage to request / to work on
-        auto issue_rows = [&](uint32_t il, int sp) {
-            float4 *dst = rowb + ring_issue * (RST * KP4) + g * KP4 + l;
-#pragma unroll
-            for (int it = 0; it < RST / GW; ++it) {
-                const uint32_t ir = __shfl_sync(FULL, il, sp * RST + it * GW + g);
-#pragma unroll
-                for (int v = 0; v < NV; ++v)
-                    cp_async16(dst + it * GW * KP4 + v * LG, A4r + (size_t)ir * KP4 + v * LG + l);
-            }
-            ring_issue = (ring_issue + 1 == NBUF) ? 0 : ring_issue + 1;
-        };
-#pragma unroll
-        for (int q = 0; q < DG; ++q) {
-            gq[q] = 0.f; xq[q] = 0.f; jq[q] = kNoCol; mq[q] = 0u; scq[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-            uint32_t il = 0;
-            if (q < npass) il = fetch_pass(q, gq[q], scq[q], mq[q], jq[q], xq[q]);
-            if (q == 0) il_n = il;
-            if (SP == 1) {   // a stage is a pass: its rows are requested together with its scalars
-                if (q < nstage) issue_rows(il, 0);
-                cp_async_commit();
-            }
-        }
-        if (SP > 1) {
-#pragma unroll
-            for (int s = 0; s < PD; ++s) {   // PD <= SP: the first PD stages belong to the first pass
-                if (s < nstage) issue_rows(il_n, s);
-                cp_async_commit();
-            }
-        }
-
         float4 acc[NV];   // this lane group's share of the run that is open
         float accw = 0.f;
 #pragma unroll
@@ -501,173 +445,242 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
         float D_open = 0.f;                  // (scale of the column) x (product of the open run so far) - 1
         int m_open = 0;                      // entries of the column so far, the open run included
 
-        for (int k = 0; k < npass; ++k) {
-            const int cnt = (len - 32 * k) < 32 ? (len - 32 * k) : 32;
-            // this pass's scalars leave the queue; those of pass k + DG are requested
-            const float g_c = gq[0], x_c = xq[0];
-            const uint32_t jl_c = jq[0];
-            const float4 sc_q0 = scq[0];
-            const uint32_t mask = mq[0];
-#pragma unroll
-            for (int q = 0; q + 1 < DG; ++q) { gq[q] = gq[q + 1]; xq[q] = xq[q + 1]; jq[q] = jq[q + 1]; scq[q] = scq[q + 1]; mq[q] = mq[q + 1]; }
-            il_c = il_n;
-            uint32_t il_f = 0;
-            if (k + DG < npass) il_f = fetch_pass(k + DG, gq[DG - 1], scq[DG - 1], mq[DG - 1], jq[DG - 1], xq[DG - 1]);
-            if (dead) break;
-            if (SP > 1) il_n = il_f;
-
-            // ---- scalar stage ----
-            float D;
-            int m;
-            {
-                const bool bnd_c = (mask >> lane) & 1u;
-                float e = 0.f, b = 0.f;
-                const float4 sc_c = sc_q0;
-                if (lane < cnt) {
-                    const float gx = g_c * x_c;
-                    e = a.h * (a.lambda_v - gx * x_c);
-                    b = -a.h * gx;
+        // The passes of the chunk.  Compiled twice: SL = the chunk is a slice, i.e. lies inside one run, so no run
+        // starts, no scale record is read or written before the end of the chunk and the K-wide part has no run to
+        // close; the other copy handles chunks of whole runs.  Same arithmetic in both.
+        auto run_passes = [&](auto slice_tag) {
+            constexpr bool SL = decltype(slice_tag)::value;
+            // What a pass needs from global memory is requested ahead of time.  Scalars (G_i of every entry, the scale
+            // record of every column whose run starts in the pass) come DG passes ahead into a queue of registers;
+            // the rows a_i come PD stages ahead with cp.async into the row ring, one commit group per stage.
+            float gq[DG], xq[DG];
+            uint32_t jq[DG];
+            float4 scq[DG];
+            uint32_t mq[DG];                     // run starts of the pass as a lane mask
+            uint32_t il_c = 0, il_n = 0;         // local rows (one per lane) of the pass at work and of the next one
+            auto fetch_pass = [&](int k, float &g_out, float4 &sc_out, uint32_t &mask_out, uint32_t &jl, float &x_out) -> uint32_t {
+                const int at = 32 * k + lane;
+                bool bnd = false;
+                uint32_t il = 0;
+                g_out = 0.f; x_out = 0.f; jl = kNoCol;
+                if (k == f_next_at) enter_block();
+                if (at < len && !dead) {
+                    const uint2 rec = eb[at];
+                    if (WIDE) { il = rec.x; jl = rec.y; x_out = xb[at]; }
+                    else { il = rec.x >> a.jbits; jl = rec.x & jmask; x_out = __uint_as_float(rec.y); }
+                    if (!SL) {
+                        uint32_t prevj = col_init;
+                        if (at > 0) prevj = WIDE ? eb[at - 1].y : (eb[at - 1].x & jmask);
+                        bnd = jl != prevj;
+                    }
+                    DSF_CHECK((int64_t)row0 + il < a.n, 13, il);
+                    DSF_CHECK(!SL || jl == col_init, 14, jl);
+                    g_out = __ldg(Gr + il);
+                    if (!SL && bnd) sc_out = __ldcg(Sc + jl);
                 }
-                const uint32_t below = mask & (0xFFFFFFFFu >> (31 - lane));   // run starts at or before this lane
-                const int start = 31 - __clz(below);                              // -1: the run was open before the pass
-                const int lim = below == 0 ? lane : lane - start;                 // earlier lanes of the same run
-                // a run starts from its column's scale, so that the sums need no scaling when they are applied
-                D = bnd_c ? fmaf(sc_c.x, -e, sc_c.x - e) : -e;
+                mask_out = SL ? 0u : __ballot_sync(FULL, bnd);
+                return il;
+            };
+            // rows of stage sp of a pass whose local rows are `il`: lane group q fetches the row of entry
+            // sp*RST + it*GW + q, 16 bytes per lane (rows past the end of the chunk repeat row 0 of the block)
+            int ring_issue = 0, ring_use = 0;     // row ring: slot of the next stage to request / to work on
+            auto issue_rows = [&](uint32_t il, int sp) {
+                float4 *dst = rowb + ring_issue * (RST * KP4) + g * KP4 + l;
 #pragma unroll
-                for (int delta = 1; delta < 32; delta <<= 1) {
-                    const float up = __shfl_up_sync(FULL, D, delta);
-                    if (delta <= lim) D = fmaf(up, D, up + D);
+                for (int it = 0; it < RST / GW; ++it) {
+                    const uint32_t ir = __shfl_sync(FULL, il, sp * RST + it * GW + g);
+#pragma unroll
+                    for (int v = 0; v < NV; ++v)
+                        cp_async16(dst + it * GW * KP4 + v * LG, A4r + (size_t)ir * KP4 + v * LG + l);
                 }
-                const int mj = __shfl_sync(FULL, bnd_c ? __float_as_int(sc_c.y) : 0, start < 0 ? 0 : start);
-                m = lim + 1 + mj;
-                if (below == 0) { D = fmaf(D_open, D, D_open + D); m = lane + 1 + m_open; }
-                const float c = b * rcp_fast(1.0f + D);
-                const float cw = b * ex2_fast((float)m * a.kappa_w);
-                pc[lane] = make_float2(c, cw);
-                if (mask != 0u) {   // only passes with a run start need the rest
-                    pcol[lane] = jl_c;
-                    if (bnd_c) segpos[__popc(mask & ((1u << lane) - 1u))] = lane;
-                    if (lane == 0) segpos[__popc(mask)] = cnt;
-                    // a run that ends inside the pass leaves its column's new scale record right here
-                    if (lane + 1 < cnt && ((mask >> (lane + 1)) & 1u)) Sc[jl_c] = make_float4(D, __int_as_float(m), 0.f, 0.f);
+                ring_issue = (ring_issue + 1 == NBUF) ? 0 : ring_issue + 1;
+            };
+#pragma unroll
+            for (int q = 0; q < DG; ++q) {
+                gq[q] = 0.f; xq[q] = 0.f; jq[q] = kNoCol; mq[q] = 0u; scq[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                uint32_t il = 0;
+                if (q < npass) il = fetch_pass(q, gq[q], scq[q], mq[q], jq[q], xq[q]);
+                if (q == 0) il_n = il;
+                if (SP == 1) {   // a stage is a pass: its rows are requested together with its scalars
+                    if (q < nstage) issue_rows(il, 0);
+                    cp_async_commit();
                 }
             }
-            __syncwarp();
-
-            // ---- K-wide stages of this pass ----
+            if (SP > 1) {
 #pragma unroll
-            for (int sp = 0; sp < SP; ++sp) {
-                const int s = k * SP + sp;
-                if (s >= nstage) break;
-                if (s + PD < nstage) {
-                    if (SP == 1) issue_rows(il_f, 0);
-                    else if (sp + PD < SP) issue_rows(il_c, sp + PD);
-                    else issue_rows(il_n, sp + PD - SP);
+                for (int s = 0; s < PD; ++s) {   // PD <= SP: the first PD stages belong to the first pass
+                    if (s < nstage) issue_rows(il_n, s);
+                    cp_async_commit();
                 }
-                cp_async_commit();
-                cp_async_wait<PD>();
+            }
+
+            for (int k = 0; k < npass; ++k) {
+                const int cnt = (len - 32 * k) < 32 ? (len - 32 * k) : 32;
+                // this pass's scalars leave the queue; those of pass k + DG are requested
+                const float g_c = gq[0], x_c = xq[0];
+                const uint32_t jl_c = jq[0];
+                const float4 sc_q0 = scq[0];
+                const uint32_t mask = SL ? 0u : mq[0];
+#pragma unroll
+                for (int q = 0; q + 1 < DG; ++q) { gq[q] = gq[q + 1]; xq[q] = xq[q + 1]; jq[q] = jq[q + 1]; scq[q] = scq[q + 1]; mq[q] = mq[q + 1]; }
+                il_c = il_n;
+                uint32_t il_f = 0;
+                if (k + DG < npass) il_f = fetch_pass(k + DG, gq[DG - 1], scq[DG - 1], mq[DG - 1], jq[DG - 1], xq[DG - 1]);
+                if (dead) break;
+                if (SP > 1) il_n = il_f;
+
+                // ---- scalar stage ----
+                float D;
+                int m;
+                {
+                    const bool bnd_c = (mask >> lane) & 1u;
+                    float e = 0.f, b = 0.f;
+                    const float4 sc_c = sc_q0;
+                    if (lane < cnt) {
+                        const float gx = g_c * x_c;
+                        e = a.h * (a.lambda_v - gx * x_c);
+                        b = -a.h * gx;
+                    }
+                    const uint32_t below = mask & (0xFFFFFFFFu >> (31 - lane));   // run starts at or before this lane
+                    const int start = 31 - __clz(below);                              // -1: the run was open before the pass
+                    const int lim = below == 0 ? lane : lane - start;                 // earlier lanes of the same run
+                    // a run starts from its column's scale, so that the sums need no scaling when they are applied
+                    D = bnd_c ? fmaf(sc_c.x, -e, sc_c.x - e) : -e;
+#pragma unroll
+                    for (int delta = 1; delta < 32; delta <<= 1) {
+                        const float up = __shfl_up_sync(FULL, D, delta);
+                        if (delta <= lim) D = fmaf(up, D, up + D);
+                    }
+                    const int mj = SL ? 0 : __shfl_sync(FULL, bnd_c ? __float_as_int(sc_c.y) : 0, start < 0 ? 0 : start);
+                    m = lim + 1 + mj;
+                    if (below == 0) { D = fmaf(D_open, D, D_open + D); m = lane + 1 + m_open; }
+                    const float c = b * rcp_fast(1.0f + D);
+                    const float cw = b * ex2_fast((float)m * a.kappa_w);
+                    pc[lane] = make_float2(c, cw);
+                    if (mask != 0u) {   // only passes with a run start need the rest
+                        pcol[lane] = jl_c;
+                        if (bnd_c) segpos[__popc(mask & ((1u << lane) - 1u))] = lane;
+                        if (lane == 0) segpos[__popc(mask)] = cnt;
+                        // a run that ends inside the pass leaves its column's new scale record right here
+                        if (lane + 1 < cnt && ((mask >> (lane + 1)) & 1u)) Sc[jl_c] = make_float4(D, __int_as_float(m), 0.f, 0.f);
+                    }
+                }
                 __syncwarp();
-                const float4 *rb = rowb + ring_use * (RST * KP4);
-                ring_use = (ring_use + 1 == NBUF) ? 0 : ring_use + 1;
-                const int e0 = sp * RST;
-                const int e1 = (e0 + RST < cnt) ? e0 + RST : cnt;
-                // entries [b0, b1) of the pass, entry u to lane group (u - b0) mod GW, into (acc, accw)
-                auto add_spread = [&](int b0, int b1) {
-                    for (int u = b0 + g; u < b1; u += GW) {
-                        const float2 cf = pc[u];
+
+                // ---- K-wide stages of this pass ----
 #pragma unroll
-                        for (int v = 0; v < NV; ++v) {
-                            const float4 r = rb[(u - e0) * KP4 + v * LG + l];
-                            acc[v].x = fmaf(cf.x, r.x, acc[v].x); acc[v].y = fmaf(cf.x, r.y, acc[v].y);
-                            acc[v].z = fmaf(cf.x, r.z, acc[v].z); acc[v].w = fmaf(cf.x, r.w, acc[v].w);
-                        }
-                        accw += cf.y;
+                for (int sp = 0; sp < SP; ++sp) {
+                    const int s = k * SP + sp;
+                    if (s >= nstage) break;
+                    if (s + PD < nstage) {
+                        if (SP == 1) issue_rows(il_f, 0);
+                        else if (sp + PD < SP) issue_rows(il_c, sp + PD);
+                        else issue_rows(il_n, sp + PD - SP);
                     }
-                };
-                const uint32_t range = (e1 >= 32 ? 0xFFFFFFFFu : ((1u << e1) - 1u)) & ~((1u << e0) - 1u);
-                const uint32_t sub = mask & range;
-                if (sub == 0) {
-                    if (e1 - e0 == RST) {
-                        // a whole stage inside one run: the common case on click-log data
-#pragma unroll
-                        for (int q = 0; q < RST / GW; ++q) {
-                            const float2 cf = pc[e0 + q * GW + g];
-#pragma unroll
-                            for (int v = 0; v < NV; ++v) {
-                                const float4 r = rb[(q * GW + g) * KP4 + v * LG + l];
-                                acc[v].x = fmaf(cf.x, r.x, acc[v].x); acc[v].y = fmaf(cf.x, r.y, acc[v].y);
-                                acc[v].z = fmaf(cf.x, r.z, acc[v].z); acc[v].w = fmaf(cf.x, r.w, acc[v].w);
-                            }
-                            accw += cf.y;
-                        }
-                    } else {
-                        add_spread(e0, e1);
-                    }
-                } else {
-                    const int F = __ffs(sub) - 1, Lb = 31 - __clz(sub);
-                    // 1. what is left of the open run, then the open run ends
-                    add_spread(e0, F);
-                    if (open_valid) {
-                        reduce_groups(acc, accw);
-                        if (g == 0) {
-                            flush(open_col, acc, accw);
-                            // (a run that ends inside the pass has left its scale record in the scalar stage)
-                            if (F == 0 && l == 0) Sc[open_col] = make_float4(D_open, __int_as_float(m_open), 0.f, 0.f);
-                        }
-                    }
-#pragma unroll
-                    for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    accw = 0.f;
-                    // 2. runs that start and end inside the stage: one lane group each
-                    const int i0 = __popc(mask & ((1u << F) - 1u));
-                    const int nmid = __popc(sub) - 1;
-                    for (int i = g; i < nmid; i += GW) {
-                        const int s0 = segpos[i0 + i], s1 = segpos[i0 + i + 1];
-                        DSF_CHECK(s0 >= e0 && s1 > s0 && s1 <= e1, 11, s0 * 64 + s1);
-                        float4 tmp[NV];
-                        float tmpw = 0.f;
-#pragma unroll
-                        for (int v = 0; v < NV; ++v) tmp[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        for (int u = s0; u < s1; ++u) {
+                    cp_async_commit();
+                    cp_async_wait<PD>();
+                    __syncwarp();
+                    const float4 *rb = rowb + ring_use * (RST * KP4);
+                    ring_use = (ring_use + 1 == NBUF) ? 0 : ring_use + 1;
+                    const int e0 = sp * RST;
+                    const int e1 = (e0 + RST < cnt) ? e0 + RST : cnt;
+                    // entries [b0, b1) of the pass, entry u to lane group (u - b0) mod GW, into (acc, accw)
+                    auto add_spread = [&](int b0, int b1) {
+                        for (int u = b0 + g; u < b1; u += GW) {
                             const float2 cf = pc[u];
 #pragma unroll
                             for (int v = 0; v < NV; ++v) {
                                 const float4 r = rb[(u - e0) * KP4 + v * LG + l];
-                                tmp[v].x = fmaf(cf.x, r.x, tmp[v].x); tmp[v].y = fmaf(cf.x, r.y, tmp[v].y);
-                                tmp[v].z = fmaf(cf.x, r.z, tmp[v].z); tmp[v].w = fmaf(cf.x, r.w, tmp[v].w);
+                                fma4(acc[v], cf.x, r);
                             }
-                            tmpw += cf.y;
+                            accw += cf.y;
                         }
-                        flush(pcol[s0], tmp, tmpw);
+                    };
+                    const uint32_t range = (e1 >= 32 ? 0xFFFFFFFFu : ((1u << e1) - 1u)) & ~((1u << e0) - 1u);
+                    const uint32_t sub = mask & range;
+                    if (sub == 0) {
+                        if (e1 - e0 == RST) {
+                            // a whole stage inside one run: the common case on click-log data
+#pragma unroll
+                            for (int q = 0; q < RST / GW; ++q) {
+                                const float2 cf = pc[e0 + q * GW + g];
+#pragma unroll
+                                for (int v = 0; v < NV; ++v) {
+                                    const float4 r = rb[(q * GW + g) * KP4 + v * LG + l];
+                                    fma4(acc[v], cf.x, r);
+                                }
+                                accw += cf.y;
+                            }
+                        } else {
+                            add_spread(e0, e1);
+                        }
+                    } else {
+                        const int F = __ffs(sub) - 1, Lb = 31 - __clz(sub);
+                        // 1. what is left of the open run, then the open run ends
+                        add_spread(e0, F);
+                        if (open_valid) {
+                            reduce_groups(acc, accw);
+                            if (g == 0) {
+                                flush(open_col, acc, accw);
+                                // (a run that ends inside the pass has left its scale record in the scalar stage)
+                                if (F == 0 && l == 0) Sc[open_col] = make_float4(D_open, __int_as_float(m_open), 0.f, 0.f);
+                            }
+                        }
+#pragma unroll
+                        for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        accw = 0.f;
+                        // 2. runs that start and end inside the stage: one lane group each
+                        const int i0 = __popc(mask & ((1u << F) - 1u));
+                        const int nmid = __popc(sub) - 1;
+                        for (int i = g; i < nmid; i += GW) {
+                            const int s0 = segpos[i0 + i], s1 = segpos[i0 + i + 1];
+                            DSF_CHECK(s0 >= e0 && s1 > s0 && s1 <= e1, 11, s0 * 64 + s1);
+                            float4 tmp[NV];
+                            float tmpw = 0.f;
+#pragma unroll
+                            for (int v = 0; v < NV; ++v) tmp[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+                            for (int u = s0; u < s1; ++u) {
+                                const float2 cf = pc[u];
+#pragma unroll
+                                for (int v = 0; v < NV; ++v) {
+                                    const float4 r = rb[(u - e0) * KP4 + v * LG + l];
+                                    fma4(tmp[v], cf.x, r);
+                                }
+                                tmpw += cf.y;
+                            }
+                            flush(pcol[s0], tmp, tmpw);
+                        }
+                        __syncwarp();
+                        // 3. the run that is open at the end of the stage
+                        add_spread(Lb, e1);
+                        open_valid = true;
+                        open_col = pcol[Lb];
                     }
                     __syncwarp();
-                    // 3. the run that is open at the end of the stage
-                    add_spread(Lb, e1);
-                    open_valid = true;
-                    open_col = pcol[Lb];
                 }
-                __syncwarp();
-            }
-            // the open run up to the end of this pass
-            D_open = __shfl_sync(FULL, D, cnt - 1);
-            m_open = __shfl_sync(FULL, m, cnt - 1);
+                // the open run up to the end of this pass
+                D_open = __shfl_sync(FULL, D, cnt - 1);
+                m_open = __shfl_sync(FULL, m, cnt - 1);
 
-            // the next chunk: its descriptor after the first pass, its entries a little later, so that neither
-            // request is waited for
-            if (k == 0) {
-                tk1 = __shfl_sync(FULL, tk1_raw, 0);
-                dn = load_desc(tk1);
+                // the next chunk: its descriptor after the first pass, its entries a little later, so that neither
+                // request is waited for
+                if (k == 0) {
+                    tk1 = __shfl_sync(FULL, tk1_raw, 0);
+                    dn = load_desc(tk1);
+                }
+                if (k == (npass > 2 ? 2 : npass - 1) && (unsigned)tk1 < nch) {
+                    off1 = ((int64_t)(uint32_t)__shfl_sync(FULL, dn, 0)) | ((int64_t)__shfl_sync(FULL, dn, 1) << 32);
+                    len1 = __shfl_sync(FULL, dn, 2);
+                    nb1 = (len1 + EB - 1) / EB;
+                    cb1 = __shfl_sync(FULL, dn, 6);
+                    have_next = true;
+                    __syncwarp();
+                    pump();   // the next chunk's first blocks, if slots are free; else they follow as the passes move on
+                }
             }
-            if (k == (npass > 2 ? 2 : npass - 1) && (unsigned)tk1 < nch) {
-                off1 = ((int64_t)(uint32_t)__shfl_sync(FULL, dn, 0)) | ((int64_t)__shfl_sync(FULL, dn, 1) << 32);
-                len1 = __shfl_sync(FULL, dn, 2);
-                nb1 = (len1 + EB - 1) / EB;
-                cb1 = __shfl_sync(FULL, dn, 6);
-                have_next = true;
-                __syncwarp();
-                pump();   // the next chunk's first blocks, if slots are free; else they follow as the passes move on
-            }
-        }
+        };
+        if (is_slice) run_passes(std::integral_constant<bool, true>{});
+        else run_passes(std::integral_constant<bool, false>{});
         cp_async_wait<0>();
         if (dead) { fail(2); break; }
 
@@ -734,8 +747,7 @@ __global__ void __launch_bounds__(kSgdThreads) sgd_sweep_kernel(const SgdArgs a)
 #pragma unroll
                             for (int v = 0; v < NV; ++v) {
                                 const float4 r = __ldcg(rbase + (size_t)(base + kk) * (KP4 + 1) + 1 + v * LG + l);
-                                ut[v].x = fmaf(s_, r.x, ut[v].x); ut[v].y = fmaf(s_, r.y, ut[v].y);
-                                ut[v].z = fmaf(s_, r.z, ut[v].z); ut[v].w = fmaf(s_, r.w, ut[v].w);
+                                fma4(ut[v], s_, r);
                             }
                         }
                     }
