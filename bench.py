@@ -307,10 +307,12 @@ def run_ours(args):
     # Stratum SGD, algorithmic bytes per epoch.  Row-block sweep (default): every array once - the 8-byte
     # entry records, A and G once (all entries of a row meet in one launch), w and V read + written.
     # Round sweep: the p tiles of a round own disjoint row blocks, so every entry re-reads G_i and a_i.
-    sweep = "round" if args.refresh_every > 0 else os.environ.get("DSFACTO_SWEEP", "rowblock")
+    # A plan cut into segments (--refresh-every) keeps the row-block sweep: one launch per segment, each of
+    # which reads A and G of all rows and reads and writes w and V once.
+    sweep = os.environ.get("DSFACTO_SWEEP", "rowblock")
     segments = -(-p // args.refresh_every) if 0 < args.refresh_every < p else 1
     sgd_gather = nnz * (8 + 4 * K + 4) + 8 * d * (K + 1)
-    sgd_floor = 8 * nnz + 4 * n * (K + 1) + 8 * d * (K + 1)
+    sgd_floor = 8 * nnz + segments * (4 * n * (K + 1) + 8 * d * (K + 1))
     sgd_bytes = sgd_gather if sweep == "round" else sgd_floor
     ref_bytes = 8 * nnz + 8 * (n + 1) + 4 * d * (K + 2) + 4 * n * K + 8 * n
     sgd_s, ref_s = phase[1] * 1e-3, phase[2] * 1e-3
@@ -322,7 +324,8 @@ def run_ours(args):
             "peak_kind": "of " + peak_kind, "traffic": traffic,
             "algorithmic_bytes_per_launch": sgd_bytes / segments, "avg_launch_us": 1e6 * sgd_s / segments,
             "model": ("gather: nnz*(8+4K+4) + 8d(K+1)" if sweep == "round" else "stream floor: 8nnz + 4n(K+1) + 8d(K+1)")
-                     + "; one launch covers the whole sweep",
+                     + ("; one launch covers the whole sweep" if segments == 1 else
+                        "; %d launches per sweep, A, G, w, V once per launch" % segments),
             # bytes the sweep asks its caches for when nothing is reused in registers; most of them are served
             # by L2, so this rate is NOT a fraction of the HBM peak and is given for context only
             "cache_request_model": {"bytes_per_step": sgd_gather, "rate_GBps": sgd_gather / sgd_s / 1e9},
