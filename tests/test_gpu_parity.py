@@ -191,7 +191,13 @@ def test_degenerate_shapes():
             g.close()
 
 
-def test_wide_entry_layout_on_device():
+@pytest.mark.parametrize("chunk,block", [(0, 0), (1000, 64), (2048, 192)])
+def test_wide_entry_layout_on_device(monkeypatch, chunk, block):
+    # local row and column need 17 bits each: entry records of {row, column} plus a value array of their own;
+    # with long chunks the kernel reads both arrays block by block through its entry ring
+    if chunk:
+        monkeypatch.setenv("DSFACTO_CHUNK", str(chunk))
+        monkeypatch.setenv("DSFACTO_BLOCK", str(block))
     n = d = 1 << 17
     indptr, indices, values, y = W.generate(n=n, d=d, seed=5, structure=W.UNIFORM, len_min=3, len_max=3,
                                             label_kind=W.L_REGRESSION, noise=0.1)
