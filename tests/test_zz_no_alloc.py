@@ -5,13 +5,15 @@ memory belongs to someone else's pool, or the thread must not touch the driver's
 keeps its reduction scratch in a fixed array inside the library, shared by every call, so this test
 runs it twice in a row on different inputs: the second result must not be coloured by what the
 first call left behind.  Reference values come from the handle-based path (dsfacto_predict for the
-scores, dsfacto_get_stats for the two sums), with the tolerances the other GPU tests use.
+scores, dsfacto_get_stats for the two sums), with the tolerances the other GPU tests use, and the
+scores and the loss sum are also held against the CPU oracle's own evaluation of the same rows.
 
 The file name sorts last on purpose: if this extra entry point breaks, a run that stops at the
 first failure has already gone through every other test."""
 import numpy as np
 import pytest
 
+from oracle import dsfacto_oracle as O
 from paper_2004_13940_b200 import dsfacto as D
 from paper_2004_13940_b200 import workloads as W
 
@@ -54,6 +56,12 @@ def _check(wl, seed):
     np.testing.assert_allclose(scores, ref_scores, rtol=0, atol=2e-5 * (1 + np.abs(ref_scores).max()))
     assert loss_sum == pytest.approx(ref_loss, rel=1e-5, abs=1e-6)
     assert g_sum == pytest.approx(ref_g, rel=1e-4, abs=1e-3)
+    # the oracle: scores by eq. (fm_model2) in fp64, mean loss over the same rows
+    w64, V64 = w.astype(np.float64), V.astype(np.float64)
+    want = O.score(wl.indptr, wl.indices, wl.values, w0, w64, V64)
+    np.testing.assert_allclose(scores, want, rtol=0, atol=2e-5 * (1 + np.abs(want).max()))
+    mean_loss, _ = O.evaluate(wl.loss, wl.indptr, wl.indices, wl.values, wl.y, w0, w64, V64)
+    assert loss_sum == pytest.approx(mean_loss * wl.n, rel=1e-4)
 
 
 def test_two_calls_in_a_row_match_the_handle_based_path():
