@@ -107,6 +107,19 @@ namespace {
         }                                                                                   \
     } while (0)
 
+// the same inside dsfacto_load_csr: a failed call leaves no half-built data set behind (free_data is declared below)
+void free_data(dsfacto *h);
+#define CU_TRY_LOAD(h, call)                                                                \
+    do {                                                                                    \
+        cudaError_t e_ = (call);                                                            \
+        if (e_ != cudaSuccess) {                                                            \
+            (h)->err = std::string(#call) + ": " + cudaGetErrorString(e_);                 \
+            cudaStreamSynchronize((h)->stream);                                             \
+            free_data(h);                                                                   \
+            return e_ == cudaErrorMemoryAllocation ? DSFACTO_ERR_OOM : DSFACTO_ERR_CUDA;    \
+        }                                                                                   \
+    } while (0)
+
 template <typename T>
 int dev_alloc(dsfacto *h, T **ptr, size_t count) {
     *ptr = nullptr;
@@ -1689,12 +1702,12 @@ static int load_validated(dsfacto_t *h, const int64_t *indptr, const int32_t *in
             free_data(h);
             return rc;
         }
-        CU_TRY(h, cudaMemcpyAsync(h->d_indptr, indptr, sizeof(int64_t) * ((size_t)n + 1), cudaMemcpyHostToDevice, st));
+        CU_TRY_LOAD(h, cudaMemcpyAsync(h->d_indptr, indptr, sizeof(int64_t) * ((size_t)n + 1), cudaMemcpyHostToDevice, st));
         if (nnz > 0) {
-            CU_TRY(h, cudaMemcpyAsync(h->d_idx, indices, sizeof(int32_t) * (size_t)nnz, cudaMemcpyHostToDevice, st));
-            CU_TRY(h, cudaMemcpyAsync(h->d_val, values, sizeof(float) * (size_t)nnz, cudaMemcpyHostToDevice, st));
+            CU_TRY_LOAD(h, cudaMemcpyAsync(h->d_idx, indices, sizeof(int32_t) * (size_t)nnz, cudaMemcpyHostToDevice, st));
+            CU_TRY_LOAD(h, cudaMemcpyAsync(h->d_val, values, sizeof(float) * (size_t)nnz, cudaMemcpyHostToDevice, st));
         }
-        CU_TRY(h, cudaMemcpyAsync(h->d_y, y, sizeof(float) * (size_t)n, cudaMemcpyHostToDevice, st));
+        CU_TRY_LOAD(h, cudaMemcpyAsync(h->d_y, y, sizeof(float) * (size_t)n, cudaMemcpyHostToDevice, st));
     }
 
     // Tile lists.  With enough row blocks (row-block sweep) a row block is the unit of work; large
@@ -1752,11 +1765,11 @@ static int load_validated(dsfacto_t *h, const int64_t *indptr, const int32_t *in
         if (rc) { cudaStreamSynchronize(st); free_data(h); return rc; }
     }
     if (copy_from_host && nnz > 0) {
-        CU_TRY(h, cudaMemcpyAsync(h->d_ent, ent.data(), sizeof(uint2) * (size_t)nnz, cudaMemcpyHostToDevice, st));
-        if (h->wide) CU_TRY(h, cudaMemcpyAsync(h->d_xw, xw.data(), sizeof(float) * (size_t)nnz, cudaMemcpyHostToDevice, st));
+        CU_TRY_LOAD(h, cudaMemcpyAsync(h->d_ent, ent.data(), sizeof(uint2) * (size_t)nnz, cudaMemcpyHostToDevice, st));
+        if (h->wide) CU_TRY_LOAD(h, cudaMemcpyAsync(h->d_xw, xw.data(), sizeof(float) * (size_t)nnz, cudaMemcpyHostToDevice, st));
     }
-    CU_TRY(h, cudaMemcpyAsync(h->d_tile_ptr, h->tile_ptr.data(), sizeof(int64_t) * h->tile_ptr.size(), cudaMemcpyHostToDevice, st));
-    CU_TRY(h, cudaStreamSynchronize(st));
+    CU_TRY_LOAD(h, cudaMemcpyAsync(h->d_tile_ptr, h->tile_ptr.data(), sizeof(int64_t) * h->tile_ptr.size(), cudaMemcpyHostToDevice, st));
+    CU_TRY_LOAD(h, cudaStreamSynchronize(st));
     if (!pb.finished && (rc = finish_sgd_plan(h, pb))) { free_data(h); return rc; }
     if ((rc = order_columns(h))) { free_data(h); return rc; }
     {
