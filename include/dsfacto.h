@@ -67,14 +67,16 @@ int dsfacto_create(dsfacto_t **out, int64_t n, int32_t d, int32_t K, int32_t p, 
  * (r,c) belongs to round s = (c-r) mod p; tiles ordered by (s, r); inside a tile entries ordered
  * by (column, row)), copies CSR and tiles to the device and runs the recompute pass once, so that
  * A, G and the objective of the initial parameters exist.  Replaces any earlier data set.
- * Loads of 2^24 stored entries and more are bucketed on the device itself when the packed entry layout
+ * Non-empty loads are bucketed on the device itself when the packed entry layout
  * applies (local row and column ids fit 32 bits together, tile number and local column id too) and the
  * device has room for the buffers of a sort (about 25 bytes per stored entry for the duration of the call):
  * the CSR copy that the recompute pass needs anyway is turned into (tile, local column) keys, sorted by a
  * stable radix sort, packed into entry records, and a kernel cuts the chunks of the stratum SGD launch; only
- * the CSR arrays cross the link, and they are sent while the host still checks them (a data set that fails
- * the checks leaves the handle as it was, as on every path).  DSFACTO_LOAD=device takes this way for any non-empty load that fits the
- * layout.  Otherwise, and with any other value of DSFACTO_LOAD, the tile lists are built on the host; there,
+ * the CSR arrays cross the link, and from 2^24 stored entries on they are sent while the host still checks them
+ * (a data set that fails the checks leaves the handle as it was, as on every path).  On this path the
+ * row-block sweep stores several consecutive row blocks of a column block as one slot (up to 8, for loads of
+ * fewer than 2^24 entries up to 16; see DSFACTO_DEBUG_ROW_MERGE).  DSFACTO_LOAD=device asks for this way
+ * explicitly.  Otherwise, and with any other value of DSFACTO_LOAD, the tile lists are built on the host; there,
  * loads of 2^24 stored entries and more (with p at least twice the number of host threads) are
  * streamed: each host thread buckets one row block at a time into page-locked staging memory and
  * copies it to its place on the device while the other row blocks are being bucketed.  That staging
@@ -187,7 +189,7 @@ int dsfacto_last_epoch_ms(dsfacto_t *h, float ms[4]);
  *                             The sweep kernel reads a chunk's entries block by block; the environment variable
  *                             DSFACTO_BLOCK (a multiple of 32, 32 .. 256) sets the entries per block.
  *   DSFACTO_DEBUG_ROW_MERGE   (takes effect at the next dsfacto_load_csr that buckets on the device) row blocks per slot of
- *                             the device entry array, 1, 2, 4 or 8 (as many of them as the 32-bit keys and records
+ *                             the device entry array, 1, 2, 4, 8 or 16 (as many of them as the 32-bit keys and records
  *                             allow), 0 = chosen by the load: a column's entries in consecutive row blocks follow one
  *                             another in the stratified order, so they can be stored and swept as one run.  Same
  *                             result up to rounding; the environment variable DSFACTO_ROW_MERGE does the same.

@@ -2,7 +2,7 @@
 oracle's bucketing: the plain host bucketer, the row-block bucketer, the streamed load (row blocks
 bucketed into page-locked staging memory and copied block by block; DSFACTO_LOAD=stream forces it on small
 loads), and the bucketing on the device itself (keys, a stable radix sort, the chunk plan cut by a kernel),
-which large loads take by default and DSFACTO_LOAD=device forces on small ones.  DSFACTO_LOAD=nostaging
+which loads take by default when the packed entry layout applies (DSFACTO_LOAD=device asks for it by name).  DSFACTO_LOAD=nostaging
 makes the streamed load behave as if no page-locked memory could be had, which must end in the row-block
 bucketer with one copy, not in an error."""
 import numpy as np
@@ -79,6 +79,7 @@ def test_device_bucketing_gives_the_same_bits_as_the_host(monkeypatch, sweep, na
     indptr = np.concatenate([[0], np.cumsum(np.bincount(rows[keep], minlength=wl.n))]).astype(np.int64)
     indices, values = wl.indices[keep], wl.values[keep]
     res = []
+    monkeypatch.setenv("DSFACTO_ROW_MERGE", "1")   # (slots of several row blocks, which only the device builds, round differently)
     for mode in ("device", "simple"):
         monkeypatch.setenv("DSFACTO_LOAD", mode)
         with D.DSFacto(wl.n, wl.d, wl.K, wl.p, wl.loss, wl.lambda_w, wl.lambda_v, wl.eta, wl.init_seed) as g:
