@@ -179,6 +179,7 @@ inline float init_factor(uint64_t seed, uint64_t e) {
     return (float)(0.01 * z);
 }
 
+constexpr int kMaxRowMerge = 16;   // most row blocks per slot of the device entry array (32 and 64 were no faster on any data set)
 constexpr int64_t kStreamedLoadMinEntries = (int64_t)1 << 24;   // smaller loads are not worth the staging set-up
 
 inline int bits_for(int64_t count) {  // bits needed for values in [0, count)
@@ -294,7 +295,8 @@ void unpack_merged_tiles(const dsfacto *h, const uint2 *ent, std::vector<int64_t
     if (!rows && !cols && !vals) return;
 #pragma omp parallel for schedule(dynamic, 8)
     for (int64_t slot = 0; slot < nslots; ++slot) {
-        int64_t off[16] = {-1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1};   // next free place of the slot's tiles, by row block
+        int64_t off[kMaxRowMerge];   // next free place of the slot's tiles, by row block
+        for (int k = 0; k < kMaxRowMerge; ++k) off[k] = -1;
         const int64_t rb0 = (slot_rows - 1 - slot / p) * R, c = slot % p;
         for (int64_t q = h->tile_ptr[slot]; q < h->tile_ptr[slot + 1]; ++q) {
             int64_t i;
@@ -1456,11 +1458,11 @@ static int choose_row_merge(const dsfacto *h, int64_t nnz) {
     // blocks per slot as there may be (3.7 M entries, p = 64, 1 / 2 / 4 / 8 / 16 per slot: 0.90 / 0.48 / 0.29 / 0.21 /
     // 0.15 ms per sweep; 650 k entries, p = 16: 0.068 -> 0.039 ms; 20 k entries, p = 4: 0.040 -> 0.024 ms).
     const bool small = nnz < kStreamedLoadMinEntries;
-    int want = small ? 16 : 8;
+    int want = small ? kMaxRowMerge : 8;
     if (h->row_merge > 0) want = h->row_merge;
     if (const char *env = std::getenv("DSFACTO_ROW_MERGE")) {
         const int v = std::atoi(env);
-        if (v >= 1 && v <= 16) want = v;
+        if (v >= 1 && v <= kMaxRowMerge) want = v;
     }
     int rbits = 0;
     while ((2 << rbits) <= want) {
@@ -2143,7 +2145,7 @@ int dsfacto_debug_set(dsfacto_t *h, int32_t key, int64_t value) {
         h->chunk_override = (int)value;
         return DSFACTO_OK;
     case DSFACTO_DEBUG_ROW_MERGE:
-        if (value != 0 && value != 1 && value != 2 && value != 4 && value != 8 && value != 16) return DSFACTO_ERR_INVALID_ARG;
+        if (value != 0 && value != 1 && value != 2 && value != 4 && value != 8 && value != kMaxRowMerge) return DSFACTO_ERR_INVALID_ARG;
         h->row_merge = (int)value;
         return DSFACTO_OK;
     case DSFACTO_DEBUG_COLUMN_ORDER:

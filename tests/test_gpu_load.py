@@ -123,7 +123,7 @@ def test_a_rejected_large_load_leaves_the_handle_as_it_was():
         assert w0a == w0b and np.array_equal(wa, wb) and np.array_equal(Va, Vb)
 
 
-@pytest.mark.parametrize("merge", [2, 4, 8])
+@pytest.mark.parametrize("merge", [2, 4, 8, 16])
 @pytest.mark.parametrize("name,kw", [("C1", {"p": 16}), ("C2", {}), ("C3", {}), ("C3", {"p": 7}), ("C4s", {}), ("C5s", {})])
 def test_merged_row_blocks_on_the_device(monkeypatch, merge, name, kw):
     # Several row blocks per slot: a column's entries of consecutive row blocks are stored and swept as one
