@@ -283,7 +283,7 @@ int dsfacto_bucket_host_shard(int64_t n, int32_t d, int32_t p, int32_t shard, in
  * process exits).  Anything outside these limits returns DSFACTO_ERR_INVALID_ARG.
  * V_dev must be 16-byte aligned and none of the pointers may be NULL (DSFACTO_ERR_INVALID_ARG otherwise).
  * The first call on each device looks up that array's device address (a host-side query, once per
- * device).  All calls on a device share the array: it keeps the last call's
+ * device), so make that first call before any stream capture begins.  All calls on a device share the array: it keeps the last call's
  * contents, every call overwrites the slots it uses before reading them (nothing needs clearing),
  * and two calls that overlap on the GPU (different streams or threads) race on it - serialise them.
  * The call performs no cudaMalloc/cudaFree and returns after its work on the stream has finished. */
